@@ -1,0 +1,150 @@
+/* wkv.h -- C ABI of the WeightedKV decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library keeps, for every lane = (layer, sequence, kv-head), a key/value cache of at most
+ * `budget` entries and runs one iteration of the paper's Algorithm 1 ("WeightedKV") per incoming
+ * token: append k_t, v_t; single-query softmax attention over the cache (Background section:
+ * A_t = softmax(q_t^T K_t), o_t = A_t^T V_t); fold A_t into the accumulated scores a; once the cache
+ * holds more than `budget` entries, pick the entry with the smallest average score a/n outside the
+ * protected regions, merge its value into the right neighbour by the score-weighted convex
+ * combination, and drop its key.  Lanes are independent (the paper omits the batch and head
+ * dimensions for that reason).  Every step of that path runs in CUDA kernels of this library; there
+ * is no CPU fallback.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device addresses on the context's GPU; "host" pointers are ordinary
+ *     (preferably page-locked) host addresses.  The library never takes ownership of caller buffers.
+ *   - q, k, v, out hold elements of the context's storage type (fp32 or bf16); scores are fp32.
+ *   - All calls on one context must be issued from one host thread at a time and run on the
+ *     context's stream; device-pointer calls are asynchronous with respect to the host.
+ *   - Every function returning int returns WKV_OK (0) or a negative wkv_error; no exceptions cross the
+ *     boundary.  wkv_last_error() gives a text for the most recent failure on that context.
+ */
+#ifndef WKV_H_
+#define WKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wkv_ctx wkv_ctx; /* opaque, library-owned */
+
+typedef enum { WKV_F32 = 0, WKV_BF16 = 1 } wkv_dtype;
+
+typedef enum {
+  WKV_OK = 0,
+  WKV_ERR_INVALID = -1, /* bad configuration or argument                                   */
+  WKV_ERR_ALLOC = -2,   /* the memory provider returned NULL                               */
+  WKV_ERR_CUDA = -3,    /* a CUDA runtime call or launch failed (text in wkv_last_error)    */
+  WKV_ERR_STATE = -4,   /* call order misuse, or exported bookkeeping found inconsistent    */
+  WKV_ERR_TIMEOUT = -5  /* a bounded device-side wait gave up (device status word)          */
+} wkv_error;
+
+/* Device memory provider.  alloc returns a device address aligned to at least 256 bytes, or NULL. */
+typedef void* (*wkv_alloc_fn)(size_t bytes, void* user);
+typedef void (*wkv_release_fn)(void* ptr, void* user);
+
+typedef struct {
+  int32_t n_layers;   /* >= 1                                                                          */
+  int32_t batch;      /* sequences per call, >= 1                                                      */
+  int32_t n_q_heads;  /* query heads; a multiple of n_kv_heads; group = n_q_heads/n_kv_heads in {1,2,4,8} */
+  int32_t n_kv_heads; /* key/value heads                                                               */
+  int32_t head_dim;   /* 64 or 128                                                                     */
+  int32_t budget;     /* m of Algorithm 1: entries kept per lane after a step; 1 <= m < 2^20           */
+  int32_t window;     /* W >= 1: the W newest entries are never picked (W = 1 is Algorithm 1's range
+                         {0..m-1}; the Experiments section keeps 508 / 124 recent tokens)              */
+  int32_t sink;       /* S >= 0: the S first tokens are never picked (Experiments section keeps 4);
+                         budget >= sink + window is required                                           */
+  int32_t dtype;      /* wkv_dtype: storage type of q, k, v, out and the cache                         */
+  float scale;        /* softmax scale; 0 selects 1/sqrt(head_dim) (Ideal Merging section)             */
+  int32_t merge;      /* 1: WeightedKV; 0: the "Eviction" variant of the Ablation Study (value dropped) */
+  int32_t n_splits;   /* CTAs that share one lane's cache scan; 0 = choose from the shape; max 64      */
+  void* stream;       /* cudaStream_t of the caller; NULL = the legacy default stream                  */
+  wkv_alloc_fn alloc; /* NULL = cudaMalloc / cudaFree                                                  */
+  wkv_release_fn release;
+  void* user;
+} wkv_config;
+
+/* Host-only check of a configuration: NULL if wkv_create would accept it, else a static text naming the
+ * first violated rule.  Touches no GPU. */
+const char* wkv_config_error(const wkv_config* cfg);
+
+/* Validates cfg, allocates the cache and bookkeeping for n_layers*batch*n_kv_heads lanes on the current
+ * CUDA device through the provider and clears them.  *out is NULL on failure.  (Algorithm 1: "a, n are
+ * empty lists".) */
+int wkv_create(const wkv_config* cfg, wkv_ctx** out);
+
+/* Releases everything obtained from the provider.  NULL is accepted. */
+void wkv_destroy(wkv_ctx* ctx);
+
+/* Empties every lane (all caches, scores, positions); asynchronous on the stream. */
+int wkv_reset(wkv_ctx* ctx);
+
+/* Changes the stream later calls are issued on.  The caller orders work across streams. */
+int wkv_set_stream(wkv_ctx* ctx, void* stream);
+
+/* One iteration of Algorithm 1 for every sequence of one layer, one kernel launch, asynchronous.
+ *   q    device [batch, n_q_heads, head_dim]   query of the new token
+ *   k, v device [batch, n_kv_heads, head_dim]  its key and value, appended to the cache first
+ *                                              (Background: K_t = [K_{t-1}, k_t], V_t = [V_{t-1}, v_t])
+ *   out  device [batch, n_q_heads, head_dim]   o_t = A_t^T V_t over the cache including the new token and
+ *                                              before this step's merge
+ *   evicted_pos device [batch, n_kv_heads] int32, or NULL: original 0-based position of the token whose
+ *                                              key was dropped this step, -1 when the lane did not compress
+ *   probs device [batch, n_q_heads, budget+1] fp32, or NULL: A_t in slot order (slot -> position through
+ *                                              wkv_export_slots); slots beyond the lane's length get 0
+ * Errors: WKV_ERR_INVALID (NULL ctx/q/k/v/out, layer out of range), WKV_ERR_CUDA (launch failure). */
+int wkv_decode_step(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                    int32_t* evicted_pos, float* probs);
+
+/* The same step from HOST buffers: copies q, k, v to library-owned device staging, runs the step, copies
+ * out (and evicted_pos if not NULL) back and waits for the stream.  Shapes as in wkv_decode_step. */
+int wkv_decode_step_host(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                         int32_t* evicted_pos);
+
+/* Consumes a prompt exactly as Algorithm 1 does: token by token, compressing as soon as a lane exceeds
+ * the budget (the algorithm has no separate prompt phase).  One kernel launch per token, asynchronous.
+ *   Q    device [batch, T_max, n_q_heads, head_dim], K, V device [batch, T_max, n_kv_heads, head_dim]
+ *   seq_lens device [batch] int32 or NULL: sequence b consumes tokens 0..seq_lens[b]-1 (NULL = T_max each)
+ *   out  device [batch, T_max, n_q_heads, head_dim] or NULL (outputs discarded into internal staging)
+ *   evicted_pos device [batch, T_max, n_kv_heads] int32 or NULL */
+int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                int32_t T_max, void* out, int32_t* evicted_pos);
+
+/* Copies one lane to HOST memory in position order and checks its bookkeeping (links form one chain of
+ * `len` entries with strictly increasing positions); waits for the stream.  Any destination may be NULL.
+ *   len, tokens : entries held / tokens consumed so far
+ *   pos [len] int32 original positions; a [len] fp32 accumulated scores (n_i = tokens - pos_i);
+ *   K, V [len, head_dim] storage type.  Buffers must have room for budget entries.
+ * Returns WKV_ERR_STATE if the bookkeeping is inconsistent. */
+int wkv_export_state(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, int32_t* len, int32_t* tokens,
+                     int32_t* pos, float* a, void* K, void* V);
+
+/* Slot-order view of one lane for interpreting `probs`: slot_pos [budget+1] int32 on the HOST, -1 for a
+ * free slot.  Waits for the stream. */
+int wkv_export_slots(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, int32_t* slot_pos);
+
+/* Replaces one lane by the given position-ordered HOST state (len <= budget, pos strictly increasing and
+ * < tokens).  Waits for the stream. */
+int wkv_import_state(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, int32_t len, int32_t tokens,
+                     const int32_t* pos, const float* a, const void* K, const void* V);
+
+/* Reads and clears the device status word (waits for the stream): WKV_OK, or WKV_ERR_TIMEOUT if a bounded
+ * wait inside a kernel gave up since the last call. */
+int wkv_status(wkv_ctx* ctx);
+
+/* Number of kernels this context has launched so far, and bytes it obtained from the provider. */
+int64_t wkv_launch_count(const wkv_ctx* ctx);
+int64_t wkv_device_bytes(const wkv_ctx* ctx);
+/* The number of CTAs per lane the context uses (after resolving n_splits = 0). */
+int32_t wkv_splits(const wkv_ctx* ctx);
+
+const char* wkv_strerror(int code);
+const char* wkv_last_error(const wkv_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WKV_H_ */

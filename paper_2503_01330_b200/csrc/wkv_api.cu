@@ -1,0 +1,433 @@
+// Host side of the C ABI declared in include/wkv.h: configuration checks, device state, launches,
+// export / import of lanes.  All arithmetic of the method lives in wkv_kernels.cuh.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/wkv.h"
+#include "wkv_kernels.cuh"
+
+struct wkv_ctx {
+  wkv_config cfg;
+  int device = 0;
+  int lanes_per_layer = 0;
+  long long lanes_total = 0;
+  int cap = 0;            // slots per lane
+  int group = 1;
+  int n_splits = 1;
+  float scale = 0.f;
+  size_t elem = 2;
+  cudaStream_t stream = nullptr;
+  // device memory (provider-owned)
+  void* Kc = nullptr;
+  void* Vc = nullptr;
+  float* a = nullptr;
+  int32_t* pos = nullptr;
+  int32_t* next = nullptr;
+  int32_t* prev = nullptr;
+  int32_t* lane_state = nullptr;
+  float* logits = nullptr;
+  float* part = nullptr;
+  uint32_t* ticket = nullptr;
+  uint32_t* status = nullptr;
+  // staging for the host-buffer entry point and for discarded prefill outputs
+  void* stage_q = nullptr;
+  void* stage_k = nullptr;
+  void* stage_v = nullptr;
+  void* stage_out = nullptr;
+  int32_t* stage_ev = nullptr;
+  std::vector<void*> owned;
+  long long device_bytes = 0;
+  long long launches = 0;
+  std::string last_error;
+};
+
+namespace {
+
+int fail(wkv_ctx* c, int code, const std::string& msg) {
+  if (c) c->last_error = msg;
+  return code;
+}
+int cuda_fail(wkv_ctx* c, cudaError_t e, const char* what) {
+  return fail(c, WKV_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+#define WKV_CUDA(ctx, expr)                                   \
+  do {                                                        \
+    cudaError_t e_ = (expr);                                  \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #expr);  \
+  } while (0)
+
+void* default_alloc(size_t bytes, void*) {
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+  return p;
+}
+void default_release(void* p, void*) { cudaFree(p); }
+
+template <typename P>
+int take(wkv_ctx* c, P** dst, size_t bytes) {
+  bytes = (bytes + 255) & ~(size_t)255;
+  void* p = c->cfg.alloc(bytes, c->cfg.user);
+  if (!p) return fail(c, WKV_ERR_ALLOC, "device memory provider returned NULL for " + std::to_string(bytes) + " bytes");
+  c->owned.push_back(p);
+  c->device_bytes += (long long)bytes;
+  *dst = reinterpret_cast<P*>(p);
+  return WKV_OK;
+}
+
+const char* check_config(const wkv_config* c) {
+  if (!c) return "config is NULL";
+  if (c->n_layers < 1 || c->batch < 1) return "n_layers and batch must be >= 1";
+  if (c->n_kv_heads < 1 || c->n_q_heads < 1 || c->n_q_heads % c->n_kv_heads) return "n_q_heads must be a positive multiple of n_kv_heads";
+  const int g = c->n_q_heads / c->n_kv_heads;
+  if (g != 1 && g != 2 && g != 4 && g != 8) return "n_q_heads / n_kv_heads must be 1, 2, 4 or 8";
+  if (c->head_dim != 64 && c->head_dim != 128) return "head_dim must be 64 or 128";
+  if (c->dtype != WKV_F32 && c->dtype != WKV_BF16) return "dtype must be WKV_F32 or WKV_BF16";
+  if (c->budget < 1 || c->budget >= (1 << 20)) return "budget must be in [1, 2^20)";
+  if (c->window < 1) return "window must be >= 1 (the newest entry has no right neighbour)";
+  if (c->sink < 0) return "sink must be >= 0";
+  if ((long long)c->sink + c->window > c->budget) return "budget must be >= sink + window";
+  if (c->merge != 0 && c->merge != 1) return "merge must be 0 or 1";
+  if (c->n_splits < 0 || c->n_splits > wkv::kMaxSplits) return "n_splits must be in [0, 64]";
+  if (!(c->scale >= 0.f) || std::isinf(c->scale)) return "scale must be finite and >= 0";
+  if ((c->alloc == nullptr) != (c->release == nullptr)) return "alloc and release must both be set or both be NULL";
+  if ((long long)c->batch * c->n_kv_heads * wkv::kMaxSplits > 0x7fffffffLL) return "batch * n_kv_heads too large";
+  return nullptr;
+}
+
+int auto_splits(const wkv_config& c) {
+  const int lanes = c.batch * c.n_kv_heads;
+  const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+  int s = (3552 + lanes - 1) / lanes;                 // about eight waves of 148 SMs x 3 CTAs
+  const int max_by_work = (tiles + 3) / 4;            // at least ~4 tiles per CTA
+  if (s > max_by_work) s = max_by_work;
+  if (s > wkv::kMaxSplits) s = wkv::kMaxSplits;
+  if (s < 1) s = 1;
+  return s;
+}
+
+template <typename T, int D, int G>
+cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, cudaStream_t stream) {
+  using C = wkv::Cfg<T, D, G>;
+  static bool attr_done[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev >= 0 && dev < 64 && !attr_done[dev]) {
+    cudaError_t e = cudaFuncSetAttribute(wkv::decode_step_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_done[dev] = true;
+  }
+  wkv::decode_step_kernel<T, D, G><<<n_ctas, wkv::kThreads, C::kSmemBytes, stream>>>(P);
+  return cudaGetLastError();
+}
+
+template <typename T, int D>
+cudaError_t launch_by_group(int G, const wkv::StepParams& P, int n_ctas, cudaStream_t s) {
+  switch (G) {
+    case 1: return launch_step<T, D, 1>(P, n_ctas, s);
+    case 2: return launch_step<T, D, 2>(P, n_ctas, s);
+    case 4: return launch_step<T, D, 4>(P, n_ctas, s);
+    case 8: return launch_step<T, D, 8>(P, n_ctas, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P) {
+  const int n_ctas = c->lanes_per_layer * c->n_splits;
+  if (c->cfg.dtype == WKV_BF16) {
+    return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n_ctas, c->stream)
+                                  : launch_by_group<__nv_bfloat16, 64>(c->group, P, n_ctas, c->stream);
+  }
+  return c->cfg.head_dim == 128 ? launch_by_group<float, 128>(c->group, P, n_ctas, c->stream)
+                                : launch_by_group<float, 64>(c->group, P, n_ctas, c->stream);
+}
+
+wkv::StepParams base_params(const wkv_ctx* c, int layer) {
+  wkv::StepParams P;
+  std::memset(&P, 0, sizeof(P));
+  P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
+  P.lane_state = c->lane_state; P.logits = c->logits; P.part = c->part; P.ticket = c->ticket; P.status = c->status;
+  P.lane0 = layer * c->lanes_per_layer;
+  P.n_kv_heads = c->cfg.n_kv_heads;
+  P.cap = c->cap;
+  P.budget = c->cfg.budget; P.window = c->cfg.window; P.sink = c->cfg.sink;
+  P.n_splits = c->n_splits;
+  P.merge = c->cfg.merge;
+  P.scale = c->scale;
+  return P;
+}
+
+int run_reset(wkv_ctx* c) {
+  wkv::reset_kernel<<<592, 256, 0, c->stream>>>(c->lane_state, c->pos, c->a, c->next, c->prev, c->lanes_total, c->cap,
+                                                c->ticket, c->lanes_per_layer, c->status);
+  c->launches++;
+  WKV_CUDA(c, cudaGetLastError());
+  return WKV_OK;
+}
+
+int check_lane(wkv_ctx* c, int layer, int b, int h) {
+  if (!c) return WKV_ERR_INVALID;
+  if (layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || h < 0 || h >= c->cfg.n_kv_heads)
+    return fail(c, WKV_ERR_INVALID, "layer / sequence / kv_head out of range");
+  return WKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* wkv_config_error(const wkv_config* cfg) { return check_config(cfg); }
+
+int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
+  if (!out) return WKV_ERR_INVALID;
+  *out = nullptr;
+  if (check_config(cfg) != nullptr) return WKV_ERR_INVALID;
+  wkv_ctx* c = new (std::nothrow) wkv_ctx;
+  if (!c) return WKV_ERR_ALLOC;
+  c->cfg = *cfg;
+  if (!c->cfg.alloc) { c->cfg.alloc = default_alloc; c->cfg.release = default_release; c->cfg.user = nullptr; }
+  cudaError_t e = cudaGetDevice(&c->device);
+  if (e != cudaSuccess) { delete c; return WKV_ERR_CUDA; }
+  c->group = cfg->n_q_heads / cfg->n_kv_heads;
+  c->lanes_per_layer = cfg->batch * cfg->n_kv_heads;
+  c->lanes_total = (long long)cfg->n_layers * c->lanes_per_layer;
+  c->cap = (cfg->budget + 1 + 3) & ~3;
+  c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg);
+  c->scale = cfg->scale != 0.f ? cfg->scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
+  c->elem = cfg->dtype == WKV_BF16 ? 2 : 4;
+  c->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
+
+  const size_t D = cfg->head_dim, cap = c->cap, G = c->group;
+  const size_t row = D * c->elem;
+  int rc = WKV_OK;
+  auto T = [&](int r) { if (rc == WKV_OK) rc = r; };
+  T(take(c, &c->Kc, (size_t)c->lanes_total * cap * row));
+  T(take(c, &c->Vc, (size_t)c->lanes_total * cap * row));
+  T(take(c, &c->a, (size_t)c->lanes_total * cap * 4));
+  T(take(c, &c->pos, (size_t)c->lanes_total * cap * 4));
+  T(take(c, &c->next, (size_t)c->lanes_total * cap * 4));
+  T(take(c, &c->prev, (size_t)c->lanes_total * cap * 4));
+  T(take(c, &c->lane_state, (size_t)c->lanes_total * wkv::LS_STRIDE * 4));
+  T(take(c, &c->logits, (size_t)c->lanes_per_layer * G * cap * 4));
+  T(take(c, &c->part, (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
+  T(take(c, &c->ticket, (size_t)c->lanes_per_layer * 4));
+  T(take(c, &c->status, 256));
+  T(take(c, &c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * row));
+  T(take(c, &c->stage_k, (size_t)c->lanes_per_layer * row));
+  T(take(c, &c->stage_v, (size_t)c->lanes_per_layer * row));
+  T(take(c, &c->stage_out, (size_t)cfg->batch * cfg->n_q_heads * row));
+  T(take(c, &c->stage_ev, (size_t)c->lanes_per_layer * 4));
+  if (rc == WKV_OK) rc = run_reset(c);
+  if (rc != WKV_OK) {
+    wkv_destroy(c);
+    return rc;
+  }
+  *out = c;
+  return WKV_OK;
+}
+
+void wkv_destroy(wkv_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  for (void* p : c->owned) c->cfg.release(p, c->cfg.user);
+  delete c;
+}
+
+int wkv_reset(wkv_ctx* c) {
+  if (!c) return WKV_ERR_INVALID;
+  return run_reset(c);
+}
+
+int wkv_set_stream(wkv_ctx* c, void* stream) {
+  if (!c) return WKV_ERR_INVALID;
+  c->stream = reinterpret_cast<cudaStream_t>(stream);
+  return WKV_OK;
+}
+
+int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                    int32_t* evicted_pos, float* probs) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
+  wkv::StepParams P = base_params(c, layer);
+  const long long D = c->cfg.head_dim;
+  P.q = q; P.k = k; P.v = v; P.out = out; P.evicted = evicted_pos; P.probs = probs;
+  P.q_bs = (long long)c->cfg.n_q_heads * D;
+  P.kv_bs = (long long)c->cfg.n_kv_heads * D;
+  P.out_bs = P.q_bs;
+  P.ev_bs = c->cfg.n_kv_heads;
+  P.seq_lens = nullptr;
+  P.tok_idx = 0;
+  cudaError_t e = launch_any(c, P);
+  c->launches++;
+  if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch");
+  return WKV_OK;
+}
+
+int wkv_decode_step_host(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                         int32_t* evicted_pos) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
+  const size_t row = (size_t)c->cfg.head_dim * c->elem;
+  const size_t qb = (size_t)c->cfg.batch * c->cfg.n_q_heads * row, kb = (size_t)c->lanes_per_layer * row;
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_q, q, qb, cudaMemcpyHostToDevice, c->stream));
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_k, k, kb, cudaMemcpyHostToDevice, c->stream));
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_v, v, kb, cudaMemcpyHostToDevice, c->stream));
+  int rc = wkv_decode_step(c, layer, c->stage_q, c->stage_k, c->stage_v, c->stage_out, c->stage_ev, nullptr);
+  if (rc != WKV_OK) return rc;
+  WKV_CUDA(c, cudaMemcpyAsync(out, c->stage_out, qb, cudaMemcpyDeviceToHost, c->stream));
+  if (evicted_pos)
+    WKV_CUDA(c, cudaMemcpyAsync(evicted_pos, c->stage_ev, (size_t)c->lanes_per_layer * 4, cudaMemcpyDeviceToHost, c->stream));
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  return WKV_OK;
+}
+
+int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                int32_t T_max, void* out, int32_t* evicted_pos) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!Q || !K || !V) return fail(c, WKV_ERR_INVALID, "Q, K and V must not be NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
+  if (T_max < 0) return fail(c, WKV_ERR_INVALID, "T_max must be >= 0");
+  const long long D = c->cfg.head_dim, Hq = c->cfg.n_q_heads, Hk = c->cfg.n_kv_heads;
+  wkv::StepParams P = base_params(c, layer);
+  P.seq_lens = seq_lens;
+  P.q_bs = (long long)T_max * Hq * D;
+  P.kv_bs = (long long)T_max * Hk * D;
+  P.out_bs = out ? P.q_bs : Hq * D;
+  P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
+  for (int t = 0; t < T_max; ++t) {
+    P.tok_idx = t;
+    P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
+    P.k = (const char*)K + (size_t)t * Hk * D * c->elem;
+    P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
+    P.out = out ? (void*)((char*)out + (size_t)t * Hq * D * c->elem) : c->stage_out;
+    P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
+    cudaError_t e = launch_any(c, P);
+    c->launches++;
+    if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (prefill)");
+  }
+  return WKV_OK;
+}
+
+int wkv_export_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* len, int32_t* tokens, int32_t* pos,
+                     float* a, void* K, void* V) {
+  int rc = check_lane(c, layer, b, kv_head);
+  if (rc != WKV_OK) return rc;
+  const long long lane = ((long long)layer * c->cfg.batch + b) * c->cfg.n_kv_heads + kv_head;
+  const int cap = c->cap, D = c->cfg.head_dim;
+  const size_t row = (size_t)D * c->elem;
+  int32_t st[wkv::LS_STRIDE];
+  std::vector<int32_t> hpos(cap), hnext(cap), hprev(cap);
+  std::vector<float> ha(cap);
+  std::vector<char> hK, hV;
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  WKV_CUDA(c, cudaMemcpy(st, c->lane_state + lane * wkv::LS_STRIDE, sizeof(st), cudaMemcpyDeviceToHost));
+  WKV_CUDA(c, cudaMemcpy(hpos.data(), c->pos + lane * cap, cap * 4, cudaMemcpyDeviceToHost));
+  WKV_CUDA(c, cudaMemcpy(hnext.data(), c->next + lane * cap, cap * 4, cudaMemcpyDeviceToHost));
+  WKV_CUDA(c, cudaMemcpy(hprev.data(), c->prev + lane * cap, cap * 4, cudaMemcpyDeviceToHost));
+  WKV_CUDA(c, cudaMemcpy(ha.data(), c->a + lane * cap, cap * 4, cudaMemcpyDeviceToHost));
+  if (K) { hK.resize(cap * row); WKV_CUDA(c, cudaMemcpy(hK.data(), (char*)c->Kc + lane * cap * row, cap * row, cudaMemcpyDeviceToHost)); }
+  if (V) { hV.resize(cap * row); WKV_CUDA(c, cudaMemcpy(hV.data(), (char*)c->Vc + lane * cap * row, cap * row, cudaMemcpyDeviceToHost)); }
+  const int n = st[wkv::LS_LEN];
+  if (n < 0 || n > c->cfg.budget) return fail(c, WKV_ERR_STATE, "lane length out of range");
+  if (len) *len = n;
+  if (tokens) *tokens = st[wkv::LS_T];
+  // walk the chain: exactly n entries, consistent back links, strictly increasing positions
+  int s = st[wkv::LS_HEAD], prev_slot = -1, last_pos = -1;
+  for (int i = 0; i < n; ++i) {
+    if (s < 0 || s >= cap) return fail(c, WKV_ERR_STATE, "chain leaves the slot range");
+    if (hprev[s] != prev_slot) return fail(c, WKV_ERR_STATE, "back link does not match");
+    if (hpos[s] <= last_pos || hpos[s] >= st[wkv::LS_T]) return fail(c, WKV_ERR_STATE, "positions not strictly increasing");
+    if (pos) pos[i] = hpos[s];
+    if (a) a[i] = ha[s];
+    if (K) std::memcpy((char*)K + i * row, hK.data() + s * row, row);
+    if (V) std::memcpy((char*)V + i * row, hV.data() + s * row, row);
+    last_pos = hpos[s];
+    prev_slot = s;
+    s = hnext[s];
+  }
+  if (n > 0 && (s != -1 || prev_slot != st[wkv::LS_TAIL])) return fail(c, WKV_ERR_STATE, "chain does not end at the tail");
+  if (n == 0 && st[wkv::LS_HEAD] != -1) return fail(c, WKV_ERR_STATE, "empty lane with a head");
+  return WKV_OK;
+}
+
+int wkv_export_slots(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* slot_pos) {
+  int rc = check_lane(c, layer, b, kv_head);
+  if (rc != WKV_OK) return rc;
+  if (!slot_pos) return fail(c, WKV_ERR_INVALID, "slot_pos must not be NULL");
+  const long long lane = ((long long)layer * c->cfg.batch + b) * c->cfg.n_kv_heads + kv_head;
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  WKV_CUDA(c, cudaMemcpy(slot_pos, c->pos + lane * c->cap, (size_t)(c->cfg.budget + 1) * 4, cudaMemcpyDeviceToHost));
+  return WKV_OK;
+}
+
+int wkv_import_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int32_t len, int32_t tokens,
+                     const int32_t* pos, const float* a, const void* K, const void* V) {
+  int rc = check_lane(c, layer, b, kv_head);
+  if (rc != WKV_OK) return rc;
+  if (len < 0 || len > c->cfg.budget || tokens < len) return fail(c, WKV_ERR_INVALID, "len / tokens out of range");
+  if (len > 0 && (!pos || !a || !K || !V)) return fail(c, WKV_ERR_INVALID, "pos, a, K, V must not be NULL");
+  for (int i = 0; i < len; ++i)
+    if (pos[i] < 0 || pos[i] >= tokens || (i > 0 && pos[i] <= pos[i - 1]))
+      return fail(c, WKV_ERR_INVALID, "pos must be strictly increasing and < tokens");
+  const long long lane = ((long long)layer * c->cfg.batch + b) * c->cfg.n_kv_heads + kv_head;
+  const int cap = c->cap;
+  const size_t row = (size_t)c->cfg.head_dim * c->elem;
+  std::vector<int32_t> hpos(cap, -1), hnext(cap, -1), hprev(cap, -1);
+  std::vector<float> ha(cap, 0.f);
+  for (int i = 0; i < len; ++i) {
+    hpos[i] = pos[i];
+    ha[i] = a[i];
+    hnext[i] = i + 1 < len ? i + 1 : -1;
+    hprev[i] = i - 1;
+  }
+  int32_t st[wkv::LS_STRIDE] = {len, tokens, len > 0 ? 0 : -1, len > 0 ? len - 1 : -1, len, 0, 0, 0};
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  WKV_CUDA(c, cudaMemcpy(c->pos + lane * cap, hpos.data(), cap * 4, cudaMemcpyHostToDevice));
+  WKV_CUDA(c, cudaMemcpy(c->next + lane * cap, hnext.data(), cap * 4, cudaMemcpyHostToDevice));
+  WKV_CUDA(c, cudaMemcpy(c->prev + lane * cap, hprev.data(), cap * 4, cudaMemcpyHostToDevice));
+  WKV_CUDA(c, cudaMemcpy(c->a + lane * cap, ha.data(), cap * 4, cudaMemcpyHostToDevice));
+  if (len > 0) {
+    WKV_CUDA(c, cudaMemcpy((char*)c->Kc + lane * cap * row, K, len * row, cudaMemcpyHostToDevice));
+    WKV_CUDA(c, cudaMemcpy((char*)c->Vc + lane * cap * row, V, len * row, cudaMemcpyHostToDevice));
+  }
+  WKV_CUDA(c, cudaMemcpy(c->lane_state + lane * wkv::LS_STRIDE, st, sizeof(st), cudaMemcpyHostToDevice));
+  return WKV_OK;
+}
+
+int wkv_status(wkv_ctx* c) {
+  if (!c) return WKV_ERR_INVALID;
+  uint32_t w = 0;
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  WKV_CUDA(c, cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost));
+  if (w) {
+    WKV_CUDA(c, cudaMemset(c->status, 0, 4));
+    if (w & wkv::kStatusWaitTimeout) return fail(c, WKV_ERR_TIMEOUT, "a bounded wait inside a kernel gave up");
+    return fail(c, WKV_ERR_STATE, "a kernel found inconsistent slot links");
+  }
+  return WKV_OK;
+}
+
+int64_t wkv_launch_count(const wkv_ctx* c) { return c ? c->launches : 0; }
+int64_t wkv_device_bytes(const wkv_ctx* c) { return c ? c->device_bytes : 0; }
+int32_t wkv_splits(const wkv_ctx* c) { return c ? c->n_splits : 0; }
+
+const char* wkv_strerror(int code) {
+  switch (code) {
+    case WKV_OK: return "ok";
+    case WKV_ERR_INVALID: return "invalid configuration or argument";
+    case WKV_ERR_ALLOC: return "device memory provider failed";
+    case WKV_ERR_CUDA: return "CUDA runtime error";
+    case WKV_ERR_STATE: return "inconsistent state or call order";
+    case WKV_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown error";
+}
+
+const char* wkv_last_error(const wkv_ctx* c) { return c ? c->last_error.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,620 @@
+// Device code of the WeightedKV decode step for sm_100a.
+//
+// One launch runs one iteration of the paper's Algorithm 1 for every lane (sequence, kv-head) of a layer.
+// grid = lanes * n_splits CTAs (the splits of a lane are adjacent).  The CTAs of a lane split the lane's slots into contiguous chunks; each CTA
+// streams its K and V rows through a shared-memory ring filled by bulk asynchronous copies (one elected
+// producer thread, mbarrier completion), computes the logits, an online-softmax partial of the attention
+// output, and parks the logits in scratch.  The CTA that finishes last for a lane (atomic ticket: nobody
+// waits for anybody) combines the partials into o_t, turns the logits into the probabilities A_t with the
+// reproducible binary32 arithmetic below, folds them into the accumulated scores, picks the eviction
+// victim, merges its value into the right neighbour, and relinks the slot bookkeeping.
+//
+// Slots are not kept in position order.  A lane owns budget+1 slots; each holds one cache entry
+// (K row, V row, accumulated score a, original position pos) and is chained to its position neighbours
+// through next/prev, so "the right adjacent entry" of Algorithm 1 is next[j] and freeing an entry never
+// moves cache rows.  n of Algorithm 1 is not stored: n_i = t - pos_i + 1.
+//
+// Reproducible binary32 score path (decides the eviction index, therefore specified operation by operation;
+// all operations IEEE round-to-nearest-even, explicit intrinsics so the compiler neither contracts nor
+// reassociates):
+//   dot   : 16 partial sums over contiguous channel blocks of head_dim/16, fma chain from +0, then a
+//           butterfly p_r + p_{r^off}, off = 8,4,2,1; logit = scale * p.
+//   exp   : 0 below -87; n = rint(x*LOG2E); Cody-Waite reduction with LN2_HI/LN2_LO; degree-7 Taylor
+//           polynomial in Horner form with fma; exact scaling by 2^n.
+//   sum   : Z = float(sum_i trunc(e_i * 2^40)) * 2^-40 -- an integer sum, hence order-free.
+//   prob  : e_i / Z; group mean (((p0+p1)+p2)+...)*(1/G); a += pbar; abar = a / float(n).
+//   pick  : minimum of (abar, pos) lexicographically == minimum of (bits(abar) << 32 | pos).
+//   merge : D = abar_j + abar_r; w_j = abar_j/D; w_r = abar_r/D; v = fma(w_j, v_j, w_r*v_r), rounded to T.
+// The attention output o_t is not part of that chain and uses fast exp2 with an online softmax.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace wkv {
+
+constexpr int kTileSlots = 32;        // cache entries per pipeline stage
+constexpr int kConsumerWarps = 4;     // each owns 8 rows of a tile
+constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
+constexpr int kMaxSplits = 64;
+constexpr uint32_t kSpinLimit = 1u << 22;             // bounded mbarrier polling (each poll sleeps briefly)
+
+enum StatusBits : uint32_t { kStatusWaitTimeout = 1u, kStatusBadLink = 2u };
+
+// lane_state[lane][8]
+enum { LS_LEN = 0, LS_T = 1, LS_HEAD = 2, LS_TAIL = 3, LS_FREE = 4, LS_STRIDE = 8 };
+
+struct StepParams {
+  void* Kc;              // [lanes_total][cap][D] storage type
+  void* Vc;
+  float* a;              // [lanes_total][cap]
+  int32_t* pos;          // [lanes_total][cap]
+  int32_t* next;         // [lanes_total][cap]
+  int32_t* prev;         // [lanes_total][cap]
+  int32_t* lane_state;   // [lanes_total][LS_STRIDE]
+  float* logits;         // scratch [lanes_per_layer*G][cap]
+  float* part;           // scratch [lanes_per_layer][n_splits][G][D+2] : m, l, o[D]
+  uint32_t* ticket;      // scratch [lanes_per_layer], zero between launches
+  uint32_t* status;      // device status word
+  const void* q;         // [B][..][Hq][D]   batch stride q_bs elements
+  const void* k;         // [B][..][Hkv][D]  batch stride kv_bs elements
+  const void* v;
+  void* out;             // batch stride out_bs elements
+  int32_t* evicted;      // or nullptr; batch stride ev_bs
+  float* probs;          // or nullptr; [B][Hq][budget+1]
+  const int32_t* seq_lens;   // or nullptr
+  long long q_bs, kv_bs, out_bs, ev_bs;
+  int tok_idx;           // index of this token inside the prefill call (activity test against seq_lens)
+  int lane0;             // first global lane of this layer
+  int n_kv_heads;
+  int cap;               // slots per lane (>= budget+1, multiple of 4)
+  int budget, window, sink;
+  int n_splits;
+  int merge;
+  float scale;
+};
+
+// ------------------------------------------------------------------------------------------------
+// small PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls, records it in the status word and returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
+  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 64) __nanosleep(64);
+  }
+  atomicOr(status, kStatusWaitTimeout);
+  return false;
+}
+// Bulk asynchronous copy global -> this CTA's shared memory, completion counted in bytes on an mbarrier.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ------------------------------------------------------------------------------------------------
+// storage-type helpers: a lane's EPL = D/16 contiguous channels of a row, widened to fp32
+// ------------------------------------------------------------------------------------------------
+template <int EPL>
+__device__ __forceinline__ void load_chunk(const float* p, float (&x)[EPL]) {
+#pragma unroll
+  for (int i = 0; i < EPL; i += 4) {
+    float4 t = *reinterpret_cast<const float4*>(p + i);
+    x[i] = t.x; x[i + 1] = t.y; x[i + 2] = t.z; x[i + 3] = t.w;
+  }
+}
+template <int EPL>
+__device__ __forceinline__ void load_chunk(const __nv_bfloat16* p, float (&x)[EPL]) {
+  if constexpr (EPL == 4) {
+    uint2 t = *reinterpret_cast<const uint2*>(p);
+    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xffff0000u);
+    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xffff0000u);
+  } else {
+#pragma unroll
+    for (int i = 0; i < EPL; i += 8) {
+      uint4 t = *reinterpret_cast<const uint4*>(p + i);
+      x[i + 0] = __uint_as_float(t.x << 16); x[i + 1] = __uint_as_float(t.x & 0xffff0000u);
+      x[i + 2] = __uint_as_float(t.y << 16); x[i + 3] = __uint_as_float(t.y & 0xffff0000u);
+      x[i + 4] = __uint_as_float(t.z << 16); x[i + 5] = __uint_as_float(t.z & 0xffff0000u);
+      x[i + 6] = __uint_as_float(t.w << 16); x[i + 7] = __uint_as_float(t.w & 0xffff0000u);
+    }
+  }
+}
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// ------------------------------------------------------------------------------------------------
+// reproducible exp (see the header comment)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float repro_exp(float x) {
+  if (x < -87.0f) return 0.0f;
+  const float LOG2E = __uint_as_float(0x3fb8aa3bu);
+  const float NLN2_HI = -__uint_as_float(0x3f317000u);
+  const float NLN2_LO = -__uint_as_float(0x3805fdf4u);
+  const float n = rintf(__fmul_rn(x, LOG2E));
+  float f = __fmaf_rn(n, NLN2_HI, x);
+  f = __fmaf_rn(n, NLN2_LO, f);
+  float r = __uint_as_float(0x39500d01u);                  // 1/5040
+  r = __fmaf_rn(r, f, __uint_as_float(0x3ab60b61u));       // 1/720
+  r = __fmaf_rn(r, f, __uint_as_float(0x3c088889u));       // 1/120
+  r = __fmaf_rn(r, f, __uint_as_float(0x3d2aaaabu));       // 1/24
+  r = __fmaf_rn(r, f, __uint_as_float(0x3e2aaaabu));       // 1/6
+  r = __fmaf_rn(r, f, 0.5f);
+  r = __fmaf_rn(r, f, 1.0f);
+  r = __fmaf_rn(r, f, 1.0f);
+  return __fmul_rn(r, __int_as_float(((int)n + 127) << 23));
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long x) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+  return x;
+}
+__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long x) {
+#pragma unroll
+  for (int off = 16; off >= 1; off >>= 1) {
+    unsigned long long y = __shfl_xor_sync(0xffffffffu, x, off);
+    x = y < x ? y : x;
+  }
+  return x;
+}
+
+// ------------------------------------------------------------------------------------------------
+// shared memory layout
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+struct Cfg {
+  static constexpr int EPL = D / 16;                        // channels per thread of a 16-thread row group
+  static constexpr int kRowBytes = D * (int)sizeof(T);
+  static constexpr int kTileBytes = kTileSlots * kRowBytes; // one of K or V
+  static constexpr int kStages = (kTileBytes * 2 * 4 <= 64 * 1024) ? 4 : (kTileBytes * 2 * 3 <= 96 * 1024 ? 3 : 2);
+  static constexpr int kRingBytes = kStages * 2 * kTileBytes;
+  // after the ring: per-warp partials [warps][G][D+2], new k/v rows, barriers, epilogue scalars
+  static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
+  static constexpr int kSmemBytes = kRingBytes + kWarpPartFloats * 4 + 2 * kRowBytes + 2 * kStages * 8 +
+                                    (G * kMaxSplits + 32 + 64) * 4 + 64 * 8 + 128;
+};
+
+// ------------------------------------------------------------------------------------------------
+// the fused decode step
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams P) {
+  using C = Cfg<T, D, G>;
+  constexpr int EPL = C::EPL;
+  constexpr int kStages = C::kStages;
+  const float kLog2e = 1.4426950408889634f;
+
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  unsigned char* ring = smem_raw;                                        // [stage][K tile | V tile]
+  float* warp_part = reinterpret_cast<float*>(ring + C::kRingBytes);    // [warp][G][D+2]
+  T* new_k = reinterpret_cast<T*>(warp_part + C::kWarpPartFloats);      // [D]
+  T* new_v = new_k + D;                                                 // [D]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(new_v + D);          // [kStages]
+  uint64_t* empty_bar = full_bar + kStages;                             // [kStages]
+  float* ep_w = reinterpret_cast<float*>(empty_bar + kStages);          // [G][kMaxSplits] split weights
+  float* ep_M = ep_w + G * kMaxSplits;                                  // [G] global max logit (8 reserved each)
+  float* ep_linv = ep_M + 8;                                            // [G]
+  float* ep_Z = ep_linv + 8;                                            // [G]
+  float* ep_misc = ep_Z + 8;                                            // [8] w_j, w_r
+  int* ep_int = reinterpret_cast<int*>(ep_misc + 8);                    // [64] flags, j, r
+  unsigned long long* ep_u64 = reinterpret_cast<unsigned long long*>(ep_int + 64);  // [64] reduction scratch
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
+  const int split = blockIdx.x % P.n_splits;
+  const int lane_local = blockIdx.x / P.n_splits;    // (b, kv head) of this layer
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed (ragged prefill)
+    if (split == 0 && tid == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
+    return;
+  }
+  const long long lane = (long long)P.lane0 + lane_local;
+  int* st = P.lane_state + lane * LS_STRIDE;
+  const int len = st[LS_LEN], t = st[LS_T], new_slot = st[LS_FREE];
+  const int L = len + 1;                             // entries attended this step (new token included)
+
+  const T* Kl = reinterpret_cast<const T*>(P.Kc) + lane * (long long)P.cap * D;
+  const T* Vl = reinterpret_cast<const T*>(P.Vc) + lane * (long long)P.cap * D;
+  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
+  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+
+  const int tiles_total = (L + kTileSlots - 1) / kTileSlots;
+  const int tps = (tiles_total + P.n_splits - 1) / P.n_splits;
+  const int tile_begin = split * tps;
+  const int tile_end = min(tiles_total, tile_begin + tps);
+  const int n_my_tiles = max(0, tile_end - tile_begin);
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // the new token's rows: kept in shared memory for the scan (the cache copy of that slot may still be
+  // in flight) and written to the cache by the CTA whose chunk owns the slot
+  for (int c = tid; c < D; c += kThreads) {
+    new_k[c] = k_in[c];
+    new_v[c] = v_in[c];
+  }
+  {
+    const int nt = new_slot / kTileSlots;
+    if (nt >= tile_begin && nt < tile_end) {
+      T* Kw = const_cast<T*>(Kl) + (long long)new_slot * D;
+      T* Vw = const_cast<T*>(Vl) + (long long)new_slot * D;
+      for (int c = tid; c < D; c += kThreads) {
+        Kw[c] = k_in[c];
+        Vw[c] = v_in[c];
+      }
+    }
+  }
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    // ---------------- producer: one thread keeps the ring full ----------------
+    if (lane_id == 0) {
+      for (int i = 0; i < n_my_tiles; ++i) {
+        const int s = i % kStages;
+        if (i >= kStages) mbar_wait(&empty_bar[s], ((i / kStages) - 1) & 1, P.status);
+        const int slot0 = (tile_begin + i) * kTileSlots;
+        const uint32_t bytes = (uint32_t)min(kTileSlots, L - slot0) * C::kRowBytes;
+        unsigned char* dst = ring + (size_t)s * 2 * C::kTileBytes;
+        mbar_expect_tx(&full_bar[s], 2 * bytes);
+        bulk_g2s(dst, Kl + (long long)slot0 * D, bytes, &full_bar[s]);
+        bulk_g2s(dst + C::kTileBytes, Vl + (long long)slot0 * D, bytes, &full_bar[s]);
+      }
+    }
+  } else {
+    // ---------------- consumers: 4 warps x (2 rows per pass, 16 threads per row) ----------------
+    const int half = lane_id >> 4, l16 = lane_id & 15;
+    float qf[G][EPL];
+#pragma unroll
+    for (int g = 0; g < G; ++g) load_chunk<EPL>(q_in + g * D + l16 * EPL, qf[g]);
+    float m_run[G], l_run[G], o_acc[G][EPL];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      m_run[g] = -INFINITY;
+      l_run[g] = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) o_acc[g][e] = 0.f;
+    }
+    float* logit_base = P.logits + (long long)lane_local * G * P.cap;
+
+    for (int i = 0; i < n_my_tiles; ++i) {
+      const int s = i % kStages;
+      mbar_wait(&full_bar[s], (i / kStages) & 1, P.status);
+      const T* tK = reinterpret_cast<const T*>(ring + (size_t)s * 2 * C::kTileBytes);
+      const T* tV = reinterpret_cast<const T*>(ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      const int slot0 = (tile_begin + i) * kTileSlots;
+
+      float sv[G][4];
+      bool valid[4];
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        const int row = warp * 8 + it * 2 + half;
+        const int slot = slot0 + row;
+        valid[it] = slot < L;
+        const T* krow = (slot == new_slot) ? new_k : tK + row * D;
+        float kf[EPL];
+        load_chunk<EPL>(krow + l16 * EPL, kf);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float acc = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc = __fmaf_rn(qf[g][e], kf[e], acc);
+#pragma unroll
+          for (int off = 8; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+          const float sc = __fmul_rn(P.scale, acc);
+          sv[g][it] = valid[it] ? sc : -INFINITY;
+        }
+      }
+      // park the logits: thread (half, l16 = it) owns row warp*8 + it*2 + half
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float mine = l16 == 0 ? sv[g][0] : l16 == 1 ? sv[g][1] : l16 == 2 ? sv[g][2] : sv[g][3];
+        const int slot = slot0 + warp * 8 + l16 * 2 + half;
+        if (l16 < 4 && slot < L) logit_base[(long long)g * P.cap + slot] = mine;
+      }
+      // online softmax update, one rescale per tile
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float mt = fmaxf(fmaxf(sv[g][0], sv[g][1]), fmaxf(sv[g][2], sv[g][3]));
+        const float m_new = fmaxf(m_run[g], mt);
+        const float m_use = m_new == -INFINITY ? 0.f : m_new;
+        const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
+        m_run[g] = m_new;
+        l_run[g] *= corr;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o_acc[g][e] *= corr;
+#pragma unroll
+        for (int it = 0; it < 4; ++it) sv[g][it] = fast_exp2((sv[g][it] - m_use) * kLog2e);   // now probabilities
+      }
+#pragma unroll
+      for (int it = 0; it < 4; ++it) {
+        const int row = warp * 8 + it * 2 + half;
+        const T* vrow = (slot0 + row == new_slot) ? new_v : tV + row * D;
+        float vf[EPL];
+        load_chunk<EPL>(vrow + l16 * EPL, vf);
+        if (valid[it]) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            l_run[g] += sv[g][it];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o_acc[g][e] = fmaf(sv[g][it], vf[e], o_acc[g][e]);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane_id == 0) mbar_arrive(&empty_bar[s]);
+    }
+
+    // fold the two row groups of the warp, then leave the warp's partial in shared memory
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], 16);
+      const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], 16);
+      const float m_new = fmaxf(m_run[g], m_o);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
+      const float l_new = l_run[g] * c_me + l_o * c_o;
+      float* wp = warp_part + (warp * G + g) * (D + 2);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][e], 16);
+        const float o_new = o_acc[g][e] * c_me + o_o * c_o;
+        if (half == 0) wp[2 + l16 * EPL + e] = o_new;
+      }
+      if (lane_id == 0) { wp[0] = m_new; wp[1] = l_new; }
+    }
+  }
+  __syncthreads();
+
+  // ---------------- CTA partial -> global scratch ----------------
+  float* my_part = P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2);
+  for (int idx = tid; idx < G * D; idx += kThreads) {
+    const int g = idx / D, c = idx % D;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; ++w) mx = fmaxf(mx, warp_part[(w * G + g) * (D + 2)]);
+    const float m_use = mx == -INFINITY ? 0.f : mx;
+    float o = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kConsumerWarps; ++w) {
+      const float* wp = warp_part + (w * G + g) * (D + 2);
+      const float cw = fast_exp2((wp[0] - m_use) * kLog2e);
+      o += wp[2 + c] * cw;
+      l += wp[1] * cw;
+    }
+    my_part[g * (D + 2) + 2 + c] = o;
+    if (c == 0) { my_part[g * (D + 2)] = mx; my_part[g * (D + 2) + 1] = l; }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const uint32_t prev = atomicAdd(&P.ticket[lane_local], 1u);
+    ep_int[0] = (prev == (uint32_t)P.n_splits - 1) ? 1 : 0;
+  }
+  __syncthreads();
+  if (!ep_int[0]) return;
+  __threadfence();
+
+  // =====================================================================================
+  // Epilogue, run by the last CTA of the lane.
+  // =====================================================================================
+  // (1) split weights and the global max / normaliser of every query head
+  if (tid < G) {
+    const int g = tid;
+    const float* pg = P.part + (long long)lane_local * P.n_splits * G * (D + 2) + g * (D + 2);
+    float M = -INFINITY;
+    for (int s = 0; s < P.n_splits; ++s) M = fmaxf(M, __ldcg(pg + (long long)s * G * (D + 2)));
+    float lsum = 0.f;
+    for (int s = 0; s < P.n_splits; ++s) {
+      const float w = fast_exp2((__ldcg(pg + (long long)s * G * (D + 2)) - M) * kLog2e);
+      ep_w[g * kMaxSplits + s] = w;
+      lsum += w * __ldcg(pg + (long long)s * G * (D + 2) + 1);
+    }
+    ep_M[g] = M;                       // max of the reproducible logits: exact, order-free
+    ep_linv[g] = 1.f / lsum;
+  }
+  __syncthreads();
+  // (2) o_t = A_t^T V_t  (Background section), V as it was before this step's merge
+  {
+    T* out = reinterpret_cast<T*>(P.out) + b * P.out_bs + (long long)hk * G * D;
+    for (int idx = tid; idx < G * D; idx += kThreads) {
+      const int g = idx / D, c = idx % D;
+      const float* pg = P.part + (long long)lane_local * P.n_splits * G * (D + 2) + g * (D + 2) + 2 + c;
+      float o = 0.f;
+      for (int s = 0; s < P.n_splits; ++s) o += ep_w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
+      out[idx] = from_f32<T>(o * ep_linv[g]);
+    }
+  }
+  // (3) Z_g = sum_i exp(s_i - M_g) as an exact integer sum
+  const float* lg = P.logits + (long long)lane_local * G * P.cap;
+  {
+    unsigned long long zl[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) zl[g] = 0ull;
+    for (int i = tid; i < L; i += kThreads) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float e = repro_exp(__fsub_rn(__ldcg(lg + (long long)g * P.cap + i), ep_M[g]));
+        zl[g] += __float2ull_rz(__fmul_rn(e, 1099511627776.0f));
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const unsigned long long w = warp_sum_u64(zl[g]);
+      if (lane_id == 0) ep_u64[g * 8 + warp] = w;
+    }
+    __syncthreads();
+    if (tid < G) {
+      unsigned long long z = 0ull;
+      for (int w = 0; w < kThreads / 32; ++w) z += ep_u64[tid * 8 + w];
+      ep_Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
+    }
+    __syncthreads();
+  }
+  // (4) A_t, a = [a,0] + A_t, abar = a/n, candidate key  (Algorithm 1)
+  float* a_l = P.a + lane * P.cap;
+  int32_t* pos_l = P.pos + lane * P.cap;
+  const bool compress = L > P.budget;                 // "length of V_t exceeds m"
+  unsigned long long best = ~0ull, bmin = ~0ull;
+  int best_slot = -1;
+  for (int i = tid; i < L; i += kThreads) {
+    float pbar;
+    {
+      float pg[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float e = repro_exp(__fsub_rn(__ldcg(lg + (long long)g * P.cap + i), ep_M[g]));
+        pg[g] = __fdiv_rn(e, ep_Z[g]);
+        if (P.probs) P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = pg[g];
+      }
+      pbar = pg[0];
+#pragma unroll
+      for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pg[g]);
+      if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
+    }
+    const bool is_new = i == new_slot;
+    const float a_new = __fadd_rn(is_new ? 0.f : a_l[i], pbar);
+    const int pos_i = is_new ? t : pos_l[i];
+    a_l[i] = a_new;
+    if (is_new) pos_l[i] = t;
+    if (compress && pos_i >= P.sink && pos_i <= t - P.window) {
+      const float abar = __fdiv_rn(a_new, __int2float_rn(t - pos_i + 1));
+      const unsigned long long key = ((unsigned long long)__float_as_uint(abar) << 32) | (uint32_t)pos_i;
+      if (key < best) { best = key; best_slot = i; }
+    }
+  }
+  if (P.probs) {
+    for (int i = L + tid; i < P.budget + 1; i += kThreads)
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = 0.f;
+  }
+  {
+    const unsigned long long wmin = warp_min_u64(best);
+    if (lane_id == 0) ep_u64[32 + warp] = wmin;
+    __syncthreads();                                     // also publishes a_l / pos_l written above to the block
+    bmin = ep_u64[32];
+    for (int w = 1; w < kThreads / 32; ++w) bmin = ep_u64[32 + w] < bmin ? ep_u64[32 + w] : bmin;
+    if (tid == 0) ep_int[1] = -1;
+    __syncthreads();
+    if (compress && best == bmin && best_slot >= 0) ep_int[1] = best_slot;   // positions are unique: one owner
+    __syncthreads();
+  }
+  // (5) link the new entry as the chain's tail; unlink the victim; merge weights
+  int32_t* next_l = P.next + lane * P.cap;
+  int32_t* prev_l = P.prev + lane * P.cap;
+  if (tid == 0) {
+    int head = st[LS_HEAD], tail = st[LS_TAIL];
+    next_l[new_slot] = -1;
+    prev_l[new_slot] = tail;
+    if (tail >= 0) next_l[tail] = new_slot; else head = new_slot;
+    tail = new_slot;
+    int ev_pos = -1, new_len = L, new_free = L;          // while growing, slots fill in arrival order
+    ep_int[2] = -1;
+    if (compress) {
+      const int j = ep_int[1];
+      const int r = next_l[j];
+      if (j < 0 || r < 0 || r >= P.cap) {
+        atomicOr(P.status, kStatusBadLink);              // cannot happen with budget >= sink + window
+      } else {
+        const float abar_j = __uint_as_float((uint32_t)(bmin >> 32));
+        const int pos_r = pos_l[r];
+        const float abar_r = __fdiv_rn(a_l[r], __int2float_rn(t - pos_r + 1));
+        const float Dn = __fadd_rn(abar_j, abar_r);
+        float wj = 0.5f, wr = 0.5f;
+        if (Dn != 0.f) { wj = __fdiv_rn(abar_j, Dn); wr = __fdiv_rn(abar_r, Dn); }
+        ep_misc[0] = wj;
+        ep_misc[1] = wr;
+        ep_int[2] = j;
+        ep_int[3] = r;
+        ev_pos = (int)(uint32_t)(bmin & 0xffffffffull);
+        // Algorithm 1: remove K[j], a[j], n[j]; the neighbour keeps its own key, a and n
+        const int pv = prev_l[j];
+        if (pv >= 0) next_l[pv] = r; else head = r;
+        prev_l[r] = pv;
+        pos_l[j] = -1;
+        new_len = P.budget;
+        new_free = j;
+      }
+    }
+    st[LS_LEN] = new_len;
+    st[LS_T] = t + 1;
+    st[LS_HEAD] = head;
+    st[LS_TAIL] = tail;
+    st[LS_FREE] = new_free;
+    if (P.evicted) P.evicted[b * P.ev_bs + hk] = ev_pos;
+    P.ticket[lane_local] = 0u;                            // ready for the next launch
+  }
+  __syncthreads();
+  // (6) V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r)   (Algorithm 1), stored in T
+  if (compress && P.merge && ep_int[2] >= 0) {
+    const int j = ep_int[2], r = ep_int[3];
+    const float wj = ep_misc[0], wr = ep_misc[1];
+    T* Vw = const_cast<T*>(Vl);
+    for (int c = tid; c < D; c += kThreads) {
+      // the row of this step's token may have been written to the cache by another CTA: take it from shared memory
+      const float vj = to_f32(j == new_slot ? new_v[c] : __ldcg(Vw + (long long)j * D + c));
+      const float vr = to_f32(r == new_slot ? new_v[c] : __ldcg(Vw + (long long)r * D + c));
+      Vw[(long long)r * D + c] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
+    }
+  }
+}
+
+// Clears a context: every lane empty, chain heads/tails unset, slot 0 free.
+__global__ void reset_kernel(int32_t* lane_state, int32_t* pos, float* a, int32_t* next, int32_t* prev, long long lanes,
+                             int cap, uint32_t* ticket, int n_ticket, uint32_t* status) {
+  const long long n = lanes * cap;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+    pos[i] = -1;
+    a[i] = 0.f;
+    next[i] = -1;
+    prev[i] = -1;
+  }
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < lanes; i += (long long)gridDim.x * blockDim.x) {
+    int32_t* st = lane_state + i * LS_STRIDE;
+    st[LS_LEN] = 0; st[LS_T] = 0; st[LS_HEAD] = -1; st[LS_TAIL] = -1; st[LS_FREE] = 0;
+    st[5] = 0; st[6] = 0; st[7] = 0;
+  }
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_ticket; i += (long long)gridDim.x * blockDim.x)
+    ticket[i] = 0u;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;
+}
+
+}  // namespace wkv

@@ -122,7 +122,7 @@ class TokenStream:
             s = d ** -0.5
             q, k, v = q * s, k * s, v * s
         dt = wl.torch_dtype
-        return q.to(dt), k.to(dt), v.to(dt)
+        return q.to(dt).contiguous(), k.to(dt).contiguous(), v.to(dt).contiguous()
 
     def tokens(self, t0: int, n: int):
         """n consecutive tokens, token-major per sequence: q [n_layers, B, n, Hq, d], k, v [n_layers, B, n, Hkv, d]."""

@@ -1,0 +1,164 @@
+"""CUDA library vs CPU oracle on the same seeded inputs, through the C ABI.  Eviction positions, retained
+positions and accumulated scores are compared bit for bit; attention outputs and merged values within the
+tolerances stated in parity_util."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_01330_b200 import binding
+from paper_2503_01330_b200.synth import WORKLOADS, Workload
+
+from parity_util import Parity, assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name="s", layers=1, batch=2, hq=4, hkv=4, d=64, dtype="f32", m=40, W=4, S=0, rank=0):
+    return Workload(name, layers, batch, hq, hkv, d, dtype, m, W, S, 0, 0, 0, rank, 0.05, rank == 0)
+
+
+def test_tiny_config_every_step():
+    """1 layer, batch 1, 4 heads x 64, fp32, budget 128, window 16: 256 prefill tokens, 256 decode steps."""
+    wl = WORKLOADS["tiny"]
+    p = Parity(wl)
+    p.prefill(wl.prefill, chunk=64)
+    p.compare_state()
+    p.decode(wl.decode)
+    p.compare_state()
+    assert p.n_evictions == wl.lanes * (wl.prefill + wl.decode - wl.budget)
+    p.close()
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,m,W,S,splits,steps", [
+    ("f32", 64, 4, 4, 40, 4, 0, 0, 120),       # several tiles, ragged tail (41 = 32 + 9)
+    ("f32", 128, 2, 2, 70, 1, 0, 3, 150),      # Algorithm 1's own range (window 1), 3 tiles over 3 CTAs
+    ("bf16", 128, 4, 4, 100, 8, 4, 2, 220),    # sinks
+    ("bf16", 64, 4, 4, 33, 5, 2, 5, 100),      # more splits than tiles
+    ("bf16", 128, 8, 4, 64, 16, 0, 2, 160),    # group of 2
+    ("bf16", 128, 8, 2, 95, 16, 1, 0, 200),    # group of 4
+    ("f32", 64, 8, 1, 31, 3, 0, 1, 90),        # group of 8, exactly one tile
+    ("f32", 64, 2, 2, 1, 1, 0, 0, 20),         # smallest possible cache
+    ("bf16", 128, 2, 2, 8, 8, 0, 0, 40),       # window == budget: a single candidate
+    ("bf16", 128, 2, 2, 200, 32, 0, 64, 260),  # maximum split count
+])
+def test_shapes_every_step(dtype, d, hq, hkv, m, W, S, splits, steps):
+    wl = small(batch=3, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=W, S=S, rank=16 if dtype == "bf16" else 0)
+    p = Parity(wl, seed=17 + m, n_splits=splits)
+    p.decode(steps)
+    p.compare_state()
+    assert p.n_evictions == wl.lanes * max(0, steps - m)
+    p.close()
+
+
+def test_split_count_does_not_change_results():
+    """The same stream under 1, 2, 5 and 16 CTAs per lane: identical eviction sequences and bit-identical a."""
+    wl = small(batch=2, d=128, dtype="bf16", m=150, W=8, rank=16)
+    states = []
+    for splits in (1, 2, 5, 16):
+        p = Parity(wl, seed=5, n_splits=splits)
+        assert p.ctx.wkv_splits() == splits
+        p.decode(230)
+        states.append([p.ctx.wkv_export_state(*ln) for ln in p.lanes])
+        p.close()
+    for other in states[1:]:
+        for s0, s1 in zip(states[0], other):
+            assert torch.equal(s0["pos"], s1["pos"]) and torch.equal(s0["a"], s1["a"]) and torch.equal(s0["V"], s1["V"])
+
+
+def test_ragged_prefill_then_decode():
+    """Per-sequence prompt lengths, one shorter than the budget so that lane is still growing during decode."""
+    wl = small(layers=2, batch=4, d=128, dtype="bf16", m=96, W=8, rank=16)
+    p = Parity(wl, seed=9, ragged=[150, 40, 97, 96])
+    p.prefill(150, chunk=50)
+    p.compare_state()
+    p.decode(80)
+    p.compare_state()
+    p.close()
+
+
+def test_probabilities_output():
+    wl = small(batch=1, hq=4, hkv=2, d=64, dtype="f32", m=20, W=2)
+    p = Parity(wl, seed=3, check_probs=True)
+    p.decode(45)
+    p.close()
+
+
+def test_eviction_ablation():
+    wl = small(batch=2, d=64, dtype="f32", m=30, W=4)
+    p = Parity(wl, seed=4, merge=0)
+    p.decode(100)
+    p.compare_state()
+    p.close()
+
+
+def test_host_buffer_entry_point():
+    wl = small(layers=2, batch=2, d=128, dtype="bf16", m=50, W=4, rank=16)
+    p = Parity(wl, seed=6)
+    p.decode(30)
+    p.decode(60, host_entry=True)
+    p.compare_state()
+    p.close()
+
+
+def test_export_import_roundtrip_and_continue():
+    wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=24, W=3)
+    p = Parity(wl, seed=8)
+    p.decode(60)
+    snap = [p.ctx.wkv_export_state(*ln) for ln in p.lanes]
+    p.ctx.wkv_reset()
+    for ln in p.lanes:
+        assert p.ctx.wkv_export_state(*ln)["len"] == 0
+    for ln, s in zip(p.lanes, snap):
+        p.ctx.wkv_import_state(*ln, tokens=s["tokens"], pos=s["pos"], a=s["a"], K=s["K"], V=s["V"])
+    p.compare_state()
+    p.decode(40)           # the imported (compacted) layout must keep matching the oracle
+    p.compare_state()
+    p.close()
+
+
+def test_large_budget_is_full_attention():
+    """budget >= tokens: nothing is ever removed and the output is plain softmax attention (torch, fp64)."""
+    wl = small(batch=2, hq=4, hkv=4, d=64, dtype="f32", m=300, W=4)
+    p = Parity(wl, seed=10)
+    ks, vs = [], []
+    from paper_2503_01330_b200.synth import TokenStream
+    st = TokenStream(wl, 10, "cuda:0")
+    for t in range(70):
+        q, k, v = st.token(t)
+        ks.append(k[0].double())
+        vs.append(v[0].double())
+        p.decode(1)
+        K, V = torch.stack(ks, 2), torch.stack(vs, 2)           # [B, H, t, d]
+        att = torch.softmax(torch.einsum("bhd,bhtd->bht", q[0].double(), K) / 8.0, -1)
+        want = torch.einsum("bht,bhtd->bhd", att, V)
+        assert_close(p.out[0].cpu().numpy(), want.cpu().numpy(), "f32", f"full attention step {t}")
+        assert (p.ev == -1).all()
+    p.close()
+
+
+def test_argument_errors_leave_context_usable():
+    ctx = binding.Context(1, 1, 2, 2, 64, 16, 2, dtype=binding.WKV_F32)
+    q = torch.zeros(1, 2, 64, device="cuda")
+    with pytest.raises(binding.WkvError) as e:
+        ctx.wkv_decode_step(3, q, q, q, q)
+    assert e.value.code == binding.WKV_ERR_INVALID
+    with pytest.raises(binding.WkvError):
+        ctx.wkv_decode_step(0, None, q, q, q)
+    with pytest.raises(binding.WkvError):
+        ctx.wkv_export_state(0, 5, 0)
+    ctx.wkv_decode_step(0, q, q, q, torch.empty_like(q))
+    assert ctx.wkv_status() == 0 and ctx.wkv_export_state(0, 0, 1)["len"] == 1
+    assert ctx.wkv_launch_count() == 2      # the reset at creation and one step
+    ctx.close()
+
+
+def test_llama7b_layer_config_all_lanes():
+    """One Llama-2-7B-shaped layer (32 heads x 128, bf16, budget 2048, window 64): every lane, every step of a
+    prefill that fills the cache and runs 300 compressions, then 64 decode steps."""
+    wl = WORKLOADS["llama7b_layer"]
+    p = Parity(wl)
+    p.prefill(wl.budget + 300, chunk=128)
+    p.decode(64)
+    mism = p.compare_state()
+    assert p.n_evictions == wl.lanes * 364
+    p.close()
