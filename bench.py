@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Decode-step benchmark of the WeightedKV CUDA library.
+
+One *step* = one new token for every sequence of the batch through all layers: n_layers calls of
+wkv_decode_step (one kernel launch each), compression and value merge included.  Prints one JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl wkv|reference]
+
+N > 1 is launched by torch.distributed.run, one rank per GPU; every rank decodes its own batch (the lanes of
+Algorithm 1 are independent, so there is no data-path collective) and the time is the maximum over ranks.
+`--impl reference` times the CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2503_01330_b200.synth import BASE_SEED, WORKLOADS, TokenStream, sequence_lengths  # noqa: E402
+
+METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------------------------------
+def algorithmic_bytes_per_launch(wl) -> int:
+    """Bytes one layer launch must move at a full cache (L = budget + 1 entries per lane):
+    K and V rows read once, a read + written, pos read, plus q, the appended k and v, out and the merge rows."""
+    L, d, e, G = wl.budget + 1, wl.head_dim, wl.elem_bytes, wl.group
+    per_lane = L * (2 * d * e + 12) + (2 * G + 5) * d * e
+    return wl.batch * wl.n_kv_heads * per_lane
+
+
+def hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------------
+def oracle_lane_steps_per_s(wl, n_lanes: int, steps: int, warmup: int, seed: int):
+    """Times the CPU oracle as it stands on `n_lanes` lanes of the workload's shape at a full cache.
+    Returns (lane-steps per second, threads used)."""
+    import numpy as np
+    import oracle
+    oracle.build()
+    sub = wl.scaled(n_layers=1, batch=1, n_kv_heads=n_lanes, n_q_heads=n_lanes * wl.group)
+    ref = oracle.Oracle(n_lanes, wl.head_dim, wl.budget, window=wl.window, sink=wl.sink, group=wl.group,
+                        dtype=oracle.F32 if wl.dtype == "f32" else oracle.BF16, mode=oracle.MODE_PINNED)
+    stream = TokenStream(sub, seed, "cpu")
+    # fill the cache first (growth only: cheap), then time steps that attend budget+1 entries and compress
+    t = 0
+    for t in range(wl.budget + warmup):
+        q, k, v = stream.token(t)
+        ref.step(q[0, 0].float().numpy().reshape(n_lanes, wl.group, -1), k[0, 0].float().numpy(), v[0, 0].float().numpy())
+    toks = [stream.token(wl.budget + warmup + i) for i in range(steps)]
+    toks = [(q[0, 0].float().numpy().reshape(n_lanes, wl.group, -1), k[0, 0].float().numpy(), v[0, 0].float().numpy())
+            for q, k, v in toks]
+    t0 = time.perf_counter()
+    for q, k, v in toks:
+        ref.step(q, k, v)
+    dt = time.perf_counter() - t0
+    ref.close()
+    return n_lanes * steps / dt, min(n_lanes, os.cpu_count() or 1)
+
+
+def run_reference(args, wl):
+    """The reference arm: the CPU oracle on the host cores; each step is a bounded sample of the workload."""
+    cores = os.cpu_count() or 1
+    n_lanes = cores
+    lane_rate, used = oracle_lane_steps_per_s(wl, n_lanes, args.steps, args.warmup, BASE_SEED)
+    value = lane_rate / wl.lanes
+    sample = (f"{n_lanes} of {wl.lanes} lanes at a full cache ({wl.budget + 1} entries attended), {args.steps} timed steps "
+              f"after {wl.budget + args.warmup} filling steps; full-workload rate = lane-steps/s / lanes (lanes are independent)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 / value, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(wl, args, None),
+            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": used, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl, args, splits):
+    return {"workload": wl.name, "n_layers": wl.n_layers, "batch_per_gpu": wl.batch, "n_q_heads": wl.n_q_heads,
+            "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "budget": wl.budget, "window": wl.window,
+            "sink": wl.sink, "prefill_tokens": args.prefill_tokens if args.prefill_tokens else wl.budget + 64,
+            "prefill": "streamed through wkv_prefill until every cache is full and compressing",
+            "n_splits": splits, "l2": "inputs larger than L2 (cache rows streamed once per step)",
+            "parallelism": f"lanes replicated per GPU x{args.gpus}, no collective"}
+
+
+# ------------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="serving_b16", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="wkv", choices=["wkv", "reference"])
+    ap.add_argument("--prefill-tokens", type=int, default=0, help="0 = budget + 64")
+    ap.add_argument("--n-splits", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            if args.steps > 64:
+                args.steps = 16          # keep the whole run within a few minutes
+            run_reference(args, wl)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation of the path")
+    if args.warmup < 3:
+        args.warmup = 3
+    from paper_2503_01330_b200 import binding
+    from paper_2503_01330_b200.build import build_library
+    if rank == 0:
+        build_library()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+
+    seed = BASE_SEED + 3 + 1000 * rank
+    dt_code = binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16
+    ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window, wl.sink,
+                          dt_code, n_splits=args.n_splits, device=dev)
+    stream = TokenStream(wl, seed, dev)
+    n_prefill = args.prefill_tokens if args.prefill_tokens else wl.budget + 64
+    # ragged prompt lengths in the last 32 tokens of the (shortened) prefill: every cache ends up full
+    lens = sequence_lengths(wl.scaled(prefill=n_prefill, prefill_min=max(1, n_prefill - 32)), seed).to(dev)
+    t = 0
+    chunk = 16
+    while t < n_prefill:
+        tc = min(chunk, n_prefill - t)
+        Q, K, V = stream.tokens(t, tc)
+        rel = (lens - t).clamp(min=0, max=tc).to(torch.int32)
+        for layer in range(wl.n_layers):
+            ctx.wkv_prefill(layer, Q[layer], K[layer], V[layer], rel)
+        t += tc
+    torch.cuda.synchronize()
+    del Q, K, V
+
+    total = args.warmup + args.steps
+    toks = [stream.token(n_prefill + i) for i in range(total)]
+    out = torch.empty(wl.n_layers, wl.batch, wl.n_q_heads, wl.head_dim, dtype=wl.torch_dtype, device=dev)
+    ev = torch.empty(wl.n_layers, wl.batch, wl.n_kv_heads, dtype=torch.int32, device=dev)
+
+    def step(i):
+        q, k, v = toks[i]
+        for layer in range(wl.n_layers):
+            ctx.wkv_decode_step(layer, q[layer], k[layer], v[layer], out[layer], ev[layer])
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.wkv_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    e1.record()
+    torch.cuda.synchronize()
+    elapsed_ms = e0.elapsed_time(e1)
+    launches = ctx.wkv_launch_count() - launches0
+    clocks = sampler.stop()
+    if dist is not None:
+        tt = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+        dist.barrier()
+    assert ctx.wkv_status() == 0, "device status word reports an error"
+    assert int((ev >= 0).sum()) == ev.numel(), "every lane must compress in the timed region"
+    value = world * args.steps / (elapsed_ms * 1e-3)
+
+    # ---- end to end: host buffers through wkv_decode_step_host, copies inside the timed region ----
+    n_e2e = max(1, min(args.e2e_steps, args.steps))
+    host = [tuple(x.cpu().pin_memory() for x in toks[args.warmup + i]) for i in range(n_e2e)]
+    out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
+    ev_h = torch.empty(ev.shape, dtype=ev.dtype).pin_memory()
+    for layer in range(wl.n_layers):                                   # warm the path once
+        ctx.wkv_decode_step_host(layer, host[0][0][layer], host[0][1][layer], host[0][2][layer], out_h[layer], ev_h[layer])
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for q, k, v in host:
+        for layer in range(wl.n_layers):
+            ctx.wkv_decode_step_host(layer, q[layer], k[layer], v[layer], out_h[layer], ev_h[layer])
+    h1.record()
+    torch.cuda.synchronize()
+    e2e_ms = h0.elapsed_time(h1)
+    if dist is not None:
+        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+    h2d = sum(x.numel() * x.element_size() for x in host[0])
+    d2h = out_h.numel() * out_h.element_size() + ev_h.numel() * ev_h.element_size()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = hbm_peak()
+    bytes_launch = algorithmic_bytes_per_launch(wl)
+    launch_ms = elapsed_ms / max(1, launches // 1)
+    achieved = bytes_launch / (launch_ms * 1e-3) / 1e9
+    traffic = None      # DRAM bytes per launch from an ncu capture; see profiles/
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get(wl.name)
+        except Exception:
+            traffic = None
+    line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": workload_config(wl, args, ctx.wkv_splits()),
+            "gpu_launches": launches, "clocks": clocks,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_8000_nominal": achieved / 8000.0,
+                         "kernel": "decode_step_kernel", "algorithmic_bytes_per_launch": bytes_launch,
+                         "launch_ms": launch_ms},
+            "e2e": {"value": e2e_value, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": n_e2e}}
+    if not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        n_lanes, n_steps = cores, 8
+        lane_rate, used = oracle_lane_steps_per_s(wl, n_lanes, n_steps, 2, BASE_SEED)
+        line["cpu_baseline"] = {"value": lane_rate / wl.lanes, "unit": "steps/s", "cores": used, "kind": "oracle",
+                                "sample": f"{n_lanes} of {wl.lanes} lanes at a full cache, {n_steps} timed steps; "
+                                          f"full-workload rate = lane-steps/s / lanes (lanes are independent)"}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
