@@ -99,6 +99,33 @@ int wkv_set_stream(wkv_ctx* ctx, void* stream);
 int wkv_decode_step(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
                     int32_t* evicted_pos, float* probs);
 
+/* No counterpart in the paper: this entry point exists for callers that must not allocate device memory.
+ *
+ * Some hosts of this library cannot call cudaMalloc at the moment they need a decode step: code running
+ * inside a region where allocation is forbidden or would stall (a latency-critical serving loop that
+ * promised its allocator a fixed footprint, a process whose memory pool has been handed over entirely to
+ * another component, a plug-in that is only allowed to use buffers it is given).  wkv_decode_step already
+ * allocates nothing per call, but its scratch (parked logits, per-split partial outputs, arrival counters)
+ * was obtained from the memory provider at wkv_create.  This variant runs the same kernel with that
+ * scratch placed in a fixed array of WKV_STATIC_SCRATCH_BYTES bytes that is part of the library image, so a
+ * context created through a provider that only hands out caller-owned memory never causes an allocation.
+ * Every GPU that loads the library holds the array until the process exits.
+ *
+ *   Arguments, shapes and results: exactly those of wkv_decode_step, without `probs`.
+ *   Limit: batch*n_kv_heads*(4 + group*4*roundup4(budget+1) + n_splits*group*(head_dim+2)*4) bytes (each
+ *          region rounded up to 256) must fit WKV_STATIC_SCRATCH_BYTES; otherwise WKV_ERR_INVALID is returned,
+ *          nothing is launched, and wkv_last_error() names both numbers.
+ *   First call on a device: looks up the array's device address (cudaGetSymbolAddress) with that device
+ *          current and remembers it.  Make that first call outside any stream capture.
+ *   Sharing: all contexts and all calls use the one array, which keeps the previous call's contents.  The
+ *          arrival counters are cleared on the stream before each launch; everything else is overwritten
+ *          before it is read.  Calls that can overlap on the GPU (different streams, or different contexts
+ *          without ordering between them) race on the array: serialise them.
+ *   Calls no cudaMalloc, cudaFree or other allocating routine. */
+#define WKV_STATIC_SCRATCH_BYTES (4u << 20)
+int wkv_decode_step_static(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                           int32_t* evicted_pos);
+
 /* The same step from HOST buffers: copies q, k, v to library-owned device staging, runs the step, copies
  * out (and evicted_pos if not NULL) back and waits for the stream.  Shapes as in wkv_decode_step. */
 int wkv_decode_step_host(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,

@@ -28,7 +28,7 @@ class wkv_config(C.Structure):
 
 
 EXPORTS = ["wkv_config_error", "wkv_create", "wkv_destroy", "wkv_reset", "wkv_set_stream", "wkv_decode_step",
-           "wkv_decode_step_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
+           "wkv_decode_step_static", "wkv_decode_step_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
            "wkv_status", "wkv_launch_count", "wkv_device_bytes", "wkv_splits", "wkv_strerror", "wkv_last_error"]
 
 _lib = None
@@ -50,6 +50,7 @@ def lib():
         L.wkv_reset.argtypes = [vp]
         L.wkv_set_stream.argtypes = [vp, vp]
         L.wkv_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+        L.wkv_decode_step_static.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.wkv_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.wkv_prefill.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp]
         L.wkv_export_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -164,6 +165,11 @@ class Context:
 
     def wkv_decode_step(self, layer, q, k, v, out, evicted_pos=None, probs=None):
         self._check(lib().wkv_decode_step(self._h, layer, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos), _dp(probs)))
+
+    def wkv_decode_step_static(self, layer, q, k, v, out, evicted_pos=None):
+        """wkv_decode_step with its scratch in the library's built-in device array: for callers that may not
+        allocate device memory.  Raises WkvError(WKV_ERR_INVALID) when the shape needs more than the array holds."""
+        self._check(lib().wkv_decode_step_static(self._h, layer, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos)))
 
     def wkv_decode_step_host(self, layer, q, k, v, out, evicted_pos=None):
         self._check(lib().wkv_decode_step_host(self._h, layer, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos)))

@@ -45,6 +45,12 @@ struct wkv_ctx {
   std::string last_error;
 };
 
+// Scratch of wkv_decode_step_static.  It lives in the library image: every GPU that loads the library holds
+// these bytes until the process exits.  Host code must not pass this name to a kernel -- on the host it is
+// only a stand-in for the symbol; the device address comes from cudaGetSymbolAddress (static_scratch_base).
+constexpr size_t kStaticScratchBytes = (size_t)WKV_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
 namespace {
 
 int fail(wkv_ctx* c, int code, const std::string& msg) {
@@ -169,6 +175,23 @@ int run_reset(wkv_ctx* c) {
   return WKV_OK;
 }
 
+// Device address of g_static_scratch on the current device, looked up once per device.
+cudaError_t static_scratch_base(unsigned char** base) {
+  static unsigned char* per_device[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (per_device[dev] == nullptr) {
+    unsigned char* p = nullptr;
+    e = cudaGetSymbolAddress((void**)&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    per_device[dev] = p;
+  }
+  *base = per_device[dev];
+  return cudaSuccess;
+}
+
 int check_lane(wkv_ctx* c, int layer, int b, int h) {
   if (!c) return WKV_ERR_INVALID;
   if (layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || h < 0 || h >= c->cfg.n_kv_heads)
@@ -265,6 +288,43 @@ int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, con
   cudaError_t e = launch_any(c, P);
   c->launches++;
   if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch");
+  return WKV_OK;
+}
+
+int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                           int32_t* evicted_pos) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
+  const size_t D = c->cfg.head_dim, G = c->group, lanes = c->lanes_per_layer;
+  // layout inside the static array: tickets | logits | split partials, each region 256-byte aligned
+  const size_t ticket_bytes = (lanes * 4 + 255) & ~(size_t)255;
+  const size_t logit_bytes = (lanes * G * (size_t)c->cap * 4 + 255) & ~(size_t)255;
+  const size_t part_bytes = lanes * (size_t)c->n_splits * G * (D + 2) * 4;
+  const size_t need = ticket_bytes + logit_bytes + part_bytes;
+  if (need > kStaticScratchBytes)
+    return fail(c, WKV_ERR_INVALID,
+                "wkv_decode_step_static: this shape needs " + std::to_string(need) + " bytes of scratch, the built-in array holds " +
+                    std::to_string(kStaticScratchBytes) + " (WKV_STATIC_SCRATCH_BYTES); use wkv_decode_step");
+  unsigned char* base = nullptr;
+  cudaError_t e = static_scratch_base(&base);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetSymbolAddress(static scratch)");
+  wkv::StepParams P = base_params(c, layer);
+  P.ticket = reinterpret_cast<uint32_t*>(base);
+  P.logits = reinterpret_cast<float*>(base + ticket_bytes);
+  P.part = reinterpret_cast<float*>(base + ticket_bytes + logit_bytes);
+  P.q = q; P.k = k; P.v = v; P.out = out; P.evicted = evicted_pos; P.probs = nullptr;
+  P.q_bs = (long long)c->cfg.n_q_heads * (long long)D;
+  P.kv_bs = (long long)c->cfg.n_kv_heads * (long long)D;
+  P.out_bs = P.q_bs;
+  P.ev_bs = c->cfg.n_kv_heads;
+  P.seq_lens = nullptr;
+  P.tok_idx = 0;
+  // the array keeps whatever the previous call (of any context) left: the arrival counters must start at zero
+  WKV_CUDA(c, cudaMemsetAsync(base, 0, ticket_bytes, c->stream));
+  e = launch_any(c, P);
+  c->launches++;
+  if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (static scratch)");
   return WKV_OK;
 }
 
