@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
+from paper_2503_01330_b200.multi import aggregate_steps_per_s, max_over_ranks, rank_seed  # noqa: E402
 from paper_2503_01330_b200.synth import BASE_SEED, WORKLOADS, TokenStream, sequence_lengths  # noqa: E402
 
 METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
@@ -144,7 +145,8 @@ def workload_config(wl, args, splits):
     return {"workload": wl.name, "n_layers": wl.n_layers, "batch_per_gpu": wl.batch, "n_q_heads": wl.n_q_heads,
             "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "budget": wl.budget, "window": wl.window,
             "sink": wl.sink, "prefill_tokens": args.prefill_tokens if args.prefill_tokens else wl.budget + 64,
-            "prefill": "streamed through wkv_prefill until every cache is full and compressing",
+            "prefill": "streamed through wkv_prefill until every cache is full and compressing" if args.init == "prefill"
+            else "synthetic full caches through wkv_import_state (profiling only)",
             "n_splits": splits, "l2": "inputs larger than L2 (cache rows streamed once per step)",
             "parallelism": f"lanes replicated per GPU x{args.gpus}, no collective"}
 
@@ -161,8 +163,14 @@ def main():
     ap.add_argument("--n-splits", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling captures)")
+    ap.add_argument("--init", default="prefill", choices=["prefill", "import"],
+                    help="import: fill every cache through wkv_import_state with one synthetic full lane instead of "
+                         "streaming a prompt (profiling captures: no launches before the steps)")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
+    if args.layers > 0:
+        wl = wl.scaled(n_layers=args.layers)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -190,7 +198,7 @@ def main():
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
 
-    seed = BASE_SEED + 3 + 1000 * rank
+    seed = rank_seed(BASE_SEED, rank)
     dt_code = binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16
     ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window, wl.sink,
                           dt_code, n_splits=args.n_splits, device=dev)
@@ -200,6 +208,19 @@ def main():
     lens = sequence_lengths(wl.scaled(prefill=n_prefill, prefill_min=max(1, n_prefill - 32)), seed).to(dev)
     t = 0
     chunk = 16
+    if args.init == "import":
+        g = torch.Generator().manual_seed(seed)
+        m = wl.budget
+        K1 = torch.randn(m, wl.head_dim, generator=g).to(wl.torch_dtype)
+        V1 = torch.randn(m, wl.head_dim, generator=g).to(wl.torch_dtype)
+        a1 = torch.rand(m, generator=g) + 0.1
+        p1 = torch.arange(m, dtype=torch.int32)
+        for layer in range(wl.n_layers):
+            for b in range(wl.batch):
+                for h in range(wl.n_kv_heads):
+                    ctx.wkv_import_state(layer, b, h, m, p1, a1, K1, V1)
+        n_prefill = m
+        t = n_prefill
     while t < n_prefill:
         tc = min(chunk, n_prefill - t)
         Q, K, V = stream.tokens(t, tc)
@@ -208,7 +229,7 @@ def main():
             ctx.wkv_prefill(layer, Q[layer], K[layer], V[layer], rel)
         t += tc
     torch.cuda.synchronize()
-    del Q, K, V
+    Q = K = V = None
 
     total = args.warmup + args.steps
     toks = [stream.token(n_prefill + i) for i in range(total)]
@@ -238,14 +259,12 @@ def main():
     elapsed_ms = e0.elapsed_time(e1)
     launches = ctx.wkv_launch_count() - launches0
     clocks = sampler.stop()
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     if dist is not None:
-        tt = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
         dist.barrier()
     assert ctx.wkv_status() == 0, "device status word reports an error"
     assert int((ev >= 0).sum()) == ev.numel(), "every lane must compress in the timed region"
-    value = world * args.steps / (elapsed_ms * 1e-3)
+    value = aggregate_steps_per_s(world, args.steps, elapsed_ms)
 
     # ---- end to end: host buffers through wkv_decode_step_host, copies inside the timed region ----
     n_e2e = max(1, min(args.e2e_steps, args.steps))
@@ -265,11 +284,8 @@ def main():
     h1.record()
     torch.cuda.synchronize()
     e2e_ms = h0.elapsed_time(h1)
-    if dist is not None:
-        tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
-    e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+    e2e_ms = max_over_ranks(e2e_ms, dist, dev)
+    e2e_value = aggregate_steps_per_s(world, n_e2e, e2e_ms)
     h2d = sum(x.numel() * x.element_size() for x in host[0])
     d2h = out_h.numel() * out_h.element_size() + ev_h.numel() * ev_h.element_size()
 

@@ -1,0 +1,32 @@
+"""Parity at the full shapes of the large workloads (all layers, full batch, full budget) in the launch
+configuration bench.py times, on sampled lanes the oracle computes one by one.  The streamed prompt is shortened
+to budget + 160 tokens: every cache is then full and has compressed 160 times, which is the state the decode phase
+runs in."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_01330_b200.synth import WORKLOADS
+
+from parity_util import Parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,n_sample,decode", [("llama7b_b8", 12, 16), ("serving_b16", 12, 12), ("gqa_b32", 10, 8)])
+def test_full_shape_sampled_lanes(name, n_sample, decode):
+    wl = WORKLOADS[name]
+    n_prefill = wl.budget + 160
+    rng = np.random.default_rng(11)
+    lens = rng.integers(n_prefill - 60, n_prefill + 1, wl.batch)       # ragged prompt ends, all beyond the budget
+    lens[0] = n_prefill
+    lens[-1] = n_prefill - 60
+    p = Parity(wl, sample=n_sample, ragged=lens.tolist())
+    assert p.ctx.wkv_device_bytes() > 0.9 * 2 * wl.lanes * (wl.budget + 1) * wl.head_dim * wl.elem_bytes
+    p.prefill(n_prefill, chunk=32)
+    p.compare_state()
+    p.decode(decode)
+    p.compare_state()
+    assert p.n_evictions >= len(p.lanes) * (100 + decode)
+    p.close()
+    torch.cuda.empty_cache()
