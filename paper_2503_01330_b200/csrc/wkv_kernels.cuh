@@ -33,6 +33,9 @@
 
 namespace wkv {
 
+#ifndef WKV_RING_BYTES
+#define WKV_RING_BYTES 65536          // shared-memory ring per CTA (K and V tiles, all stages)
+#endif
 constexpr int kTileSlots = 32;        // cache entries per pipeline stage
 constexpr int kConsumerWarps = 4;     // each owns 8 rows of a tile
 constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
@@ -200,7 +203,9 @@ struct Cfg {
   static constexpr int EPL = D / 16;                        // channels per thread of a 16-thread row group
   static constexpr int kRowBytes = D * (int)sizeof(T);
   static constexpr int kTileBytes = kTileSlots * kRowBytes; // one of K or V
-  static constexpr int kStages = (kTileBytes * 2 * 4 <= 64 * 1024) ? 4 : (kTileBytes * 2 * 3 <= 96 * 1024 ? 3 : 2);
+  static constexpr int kLanesPerRow = G <= 2 ? 8 : 16;      // threads that share one cache row in the scan
+  static constexpr int kFit = WKV_RING_BYTES / (2 * kTileBytes);
+  static constexpr int kStages = kFit < 2 ? 2 : (kFit > 8 ? 8 : kFit);
   static constexpr int kRingBytes = kStages * 2 * kTileBytes;
   // after the ring: per-warp partials [warps][G][D+2], new k/v rows, barriers, epilogue scalars
   static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
@@ -214,7 +219,6 @@ struct Cfg {
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams P) {
   using C = Cfg<T, D, G>;
-  constexpr int EPL = C::EPL;
   constexpr int kStages = C::kStages;
   const float kLog2e = 1.4426950408889634f;
 
@@ -299,82 +303,122 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams 
       }
     }
   } else {
-    // ---------------- consumers: 4 warps x (2 rows per pass, 16 threads per row) ----------------
-    const int half = lane_id >> 4, l16 = lane_id & 15;
-    float qf[G][EPL];
+    // ---------------- consumers: 4 warps, each owns 8 rows of every tile ----------------
+    // A row (one cache entry) is shared by LPR threads.  Thread l of the group owns the partial sums
+    // {l, l+LPR, ...} of the reproducible dot, each a block of D/16 contiguous channels, so butterfly rounds
+    // with off >= LPR are additions inside the thread and only log2(LPR) shuffles remain.
+    constexpr int LPR = C::kLanesPerRow;           // 8 or 16 threads per row
+    constexpr int NP = 16 / LPR;                   // partial sums per thread
+    constexpr int CH = D / 16;                     // channels per partial sum
+    constexpr int RPP = 32 / LPR;                  // rows per warp pass
+    constexpr int PASSES = 8 / RPP;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
+    float qf[G][NP][CH];
 #pragma unroll
-    for (int g = 0; g < G; ++g) load_chunk<EPL>(q_in + g * D + l16 * EPL, qf[g]);
-    float m_run[G], l_run[G], o_acc[G][EPL];
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+      for (int j = 0; j < NP; ++j) load_chunk<CH>(q_in + g * D + (l + LPR * j) * CH, qf[g][j]);
+    float m_run[G], l_run[G], o_acc[G][NP][CH];
 #pragma unroll
     for (int g = 0; g < G; ++g) {
       m_run[g] = -INFINITY;
       l_run[g] = 0.f;
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) o_acc[g][e] = 0.f;
+      for (int j = 0; j < NP; ++j)
+#pragma unroll
+        for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
     }
     float* logit_base = P.logits + (long long)lane_local * G * P.cap;
 
     for (int i = 0; i < n_my_tiles; ++i) {
       const int s = i % kStages;
       mbar_wait(&full_bar[s], (i / kStages) & 1, P.status);
-      const T* tK = reinterpret_cast<const T*>(ring + (size_t)s * 2 * C::kTileBytes);
-      const T* tV = reinterpret_cast<const T*>(ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      T* tK = reinterpret_cast<T*>(ring + (size_t)s * 2 * C::kTileBytes);
+      T* tV = reinterpret_cast<T*>(ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
       const int slot0 = (tile_begin + i) * kTileSlots;
-
-      float sv[G][4];
-      bool valid[4];
-#pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const int row = warp * 8 + it * 2 + half;
-        const int slot = slot0 + row;
-        valid[it] = slot < L;
-        const T* krow = (slot == new_slot) ? new_k : tK + row * D;
-        float kf[EPL];
-        load_chunk<EPL>(krow + l16 * EPL, kf);
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          float acc = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) acc = __fmaf_rn(qf[g][e], kf[e], acc);
-#pragma unroll
-          for (int off = 8; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-          const float sc = __fmul_rn(P.scale, acc);
-          sv[g][it] = valid[it] ? sc : -INFINITY;
+      {
+        // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
+        // row in the tile with the token's k and v before anybody reads it.
+        const int ns_row = new_slot - slot0;
+        if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
+          uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
+          uint32_t* dv = reinterpret_cast<uint32_t*>(tV + ns_row * D);
+          const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
+          const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
+          for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; dv[w] = sv_[w]; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
+          __syncwarp();
         }
       }
-      // park the logits: thread (half, l16 = it) owns row warp*8 + it*2 + half
+
+      float sv[G][PASSES];
+      bool valid[PASSES];
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int row = warp * 8 + ps * RPP + rg;
+        valid[ps] = slot0 + row < L;
+        float kf[NP][CH];
+#pragma unroll
+        for (int j = 0; j < NP; ++j) load_chunk<CH>(tK + row * D + (l + LPR * j) * CH, kf[j]);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          float pp[NP];
+#pragma unroll
+          for (int j = 0; j < NP; ++j) {
+            float acc = 0.f;
+#pragma unroll
+            for (int e = 0; e < CH; ++e) acc = __fmaf_rn(qf[g][j][e], kf[j][e], acc);
+            pp[j] = acc;
+          }
+          float acc = pp[0];
+          if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
+#pragma unroll
+          for (int off = LPR / 2; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+          const float sc = __fmul_rn(P.scale, acc);
+          sv[g][ps] = valid[ps] ? sc : -INFINITY;
+        }
+      }
+      // park the logits: thread l (< PASSES) of row group rg owns row warp*8 + l*RPP + rg
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float mine = l16 == 0 ? sv[g][0] : l16 == 1 ? sv[g][1] : l16 == 2 ? sv[g][2] : sv[g][3];
-        const int slot = slot0 + warp * 8 + l16 * 2 + half;
-        if (l16 < 4 && slot < L) logit_base[(long long)g * P.cap + slot] = mine;
+        float mine = sv[g][0];
+#pragma unroll
+        for (int ps = 1; ps < PASSES; ++ps) mine = l == ps ? sv[g][ps] : mine;
+        const int slot = slot0 + warp * 8 + l * RPP + rg;
+        if (l < PASSES && slot < L) logit_base[(long long)g * P.cap + slot] = mine;
       }
       // online softmax update, one rescale per tile
 #pragma unroll
       for (int g = 0; g < G; ++g) {
-        const float mt = fmaxf(fmaxf(sv[g][0], sv[g][1]), fmaxf(sv[g][2], sv[g][3]));
+        float mt = sv[g][0];
+#pragma unroll
+        for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[g][ps]);
         const float m_new = fmaxf(m_run[g], mt);
         const float m_use = m_new == -INFINITY ? 0.f : m_new;
         const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
         m_run[g] = m_new;
         l_run[g] *= corr;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) o_acc[g][e] *= corr;
+        for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int it = 0; it < 4; ++it) sv[g][it] = fast_exp2((sv[g][it] - m_use) * kLog2e);   // now probabilities
+          for (int e = 0; e < CH; ++e) o_acc[g][j][e] *= corr;
+#pragma unroll
+        for (int ps = 0; ps < PASSES; ++ps) sv[g][ps] = fast_exp2((sv[g][ps] - m_use) * kLog2e);   // now probabilities
       }
 #pragma unroll
-      for (int it = 0; it < 4; ++it) {
-        const int row = warp * 8 + it * 2 + half;
-        const T* vrow = (slot0 + row == new_slot) ? new_v : tV + row * D;
-        float vf[EPL];
-        load_chunk<EPL>(vrow + l16 * EPL, vf);
-        if (valid[it]) {
+      for (int ps = 0; ps < PASSES; ++ps) {
+        const int row = warp * 8 + ps * RPP + rg;
+        float vf[NP][CH];
+#pragma unroll
+        for (int j = 0; j < NP; ++j) load_chunk<CH>(tV + row * D + (l + LPR * j) * CH, vf[j]);
+        if (valid[ps]) {
 #pragma unroll
           for (int g = 0; g < G; ++g) {
-            l_run[g] += sv[g][it];
+            l_run[g] += sv[g][ps];
 #pragma unroll
-            for (int e = 0; e < EPL; ++e) o_acc[g][e] = fmaf(sv[g][it], vf[e], o_acc[g][e]);
+            for (int j = 0; j < NP; ++j)
+#pragma unroll
+              for (int e = 0; e < CH; ++e) o_acc[g][j][e] = fmaf(sv[g][ps], vf[j][e], o_acc[g][j][e]);
           }
         }
       }
@@ -382,23 +426,34 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams 
       if (lane_id == 0) mbar_arrive(&empty_bar[s]);
     }
 
-    // fold the two row groups of the warp, then leave the warp's partial in shared memory
+    // fold the row groups of the warp, then leave the warp's partial in shared memory
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], 16);
-      const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], 16);
-      const float m_new = fmaxf(m_run[g], m_o);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
-      const float l_new = l_run[g] * c_me + l_o * c_o;
-      float* wp = warp_part + (warp * G + g) * (D + 2);
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][e], 16);
-        const float o_new = o_acc[g][e] * c_me + o_o * c_o;
-        if (half == 0) wp[2 + l16 * EPL + e] = o_new;
+      for (int off = 16; off >= LPR; off >>= 1) {
+        const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
+        const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
+        const float m_new = fmaxf(m_run[g], m_o);
+        const float m_use = m_new == -INFINITY ? 0.f : m_new;
+        const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
+        l_run[g] = l_run[g] * c_me + l_o * c_o;
+        m_run[g] = m_new;
+#pragma unroll
+        for (int j = 0; j < NP; ++j)
+#pragma unroll
+          for (int e = 0; e < CH; ++e) {
+            const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
+            o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
+          }
       }
-      if (lane_id == 0) { wp[0] = m_new; wp[1] = l_new; }
+      float* wp = warp_part + (warp * G + g) * (D + 2);
+      if (rg == 0) {
+#pragma unroll
+        for (int j = 0; j < NP; ++j)
+#pragma unroll
+          for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
+      }
+      if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
     }
   }
   __syncthreads();
@@ -422,15 +477,16 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams 
     my_part[g * (D + 2) + 2 + c] = o;
     if (c == 0) { my_part[g * (D + 2)] = mx; my_part[g * (D + 2) + 1] = l; }
   }
-  __threadfence();
   __syncthreads();
   if (tid == 0) {
+    // release: the barrier ordered every thread's partials and logits before this fence (cumulativity)
+    __threadfence();
     const uint32_t prev = atomicAdd(&P.ticket[lane_local], 1u);
+    __threadfence();   // acquire side for the CTA that turns out to be the last
     ep_int[0] = (prev == (uint32_t)P.n_splits - 1) ? 1 : 0;
   }
   __syncthreads();
   if (!ep_int[0]) return;
-  __threadfence();
 
   // =====================================================================================
   // Epilogue, run by the last CTA of the lane.
