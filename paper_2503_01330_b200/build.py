@@ -23,7 +23,8 @@ def _stale() -> bool:
 def build_library(force: bool = False, verbose: bool = False) -> str:
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB + ".tmp"] + SOURCES
+        extra = os.environ.get("WKV_NVCC_EXTRA", "").split()      # build-time tuning macros, e.g. -DWKV_RING_BYTES=49152
+        cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB + ".tmp"] + SOURCES
         subprocess.run(cmd, check=True, cwd=CSRC)
         os.replace(LIB + ".tmp", LIB)
     return LIB

@@ -18,6 +18,8 @@ struct wkv_ctx {
   int cap = 0;            // slots per lane
   int group = 1;
   int n_splits = 1;
+  int chunk_cap = 0;      // cluster kernel: logits per CTA and query head
+  bool use_cluster = false;
   float scale = 0.f;
   size_t elem = 2;
   cudaStream_t stream = nullptr;
@@ -104,52 +106,79 @@ const char* check_config(const wkv_config* c) {
   return nullptr;
 }
 
+// Splits per lane when the caller leaves the choice to the library: a power of two (so the lane's CTAs can form a
+// thread-block cluster), enough CTAs to fill 148 SMs several times over, at least ~4 tiles of work per CTA.
 int auto_splits(const wkv_config& c) {
   const int lanes = c.batch * c.n_kv_heads;
   const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
-  int s = (3552 + lanes - 1) / lanes;                 // about eight waves of 148 SMs x 3 CTAs
-  const int max_by_work = (tiles + 3) / 4;            // at least ~4 tiles per CTA
-  if (s > max_by_work) s = max_by_work;
-  if (s > wkv::kMaxSplits) s = wkv::kMaxSplits;
-  if (s < 1) s = 1;
+  int s = 1;
+  while (s < 16 && lanes * s < 1776 && tiles / (2 * s) >= 4) s *= 2;
   return s;
 }
 
+bool is_cluster_size(int s) { return s == 1 || s == 2 || s == 4 || s == 8 || s == 16; }
+
+constexpr int kMaxDynSmem = 200 * 1024;
+
+// cluster = true: the n_splits CTAs of a lane are launched as one thread-block cluster (kernel B).
 template <typename T, int D, int G>
-cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, cudaStream_t stream) {
+cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, bool cluster, cudaStream_t stream) {
   using C = wkv::Cfg<T, D, G>;
-  static bool attr_done[64] = {};
+  static int attr_done[64][2] = {};            // largest dynamic shared memory size configured per device and kernel
   int dev = 0;
-  cudaGetDevice(&dev);
-  if (dev >= 0 && dev < 64 && !attr_done[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(wkv::decode_step_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         C::kSmemBytes);
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const int smem = C::kFixedBytes + (cluster ? G * P.chunk_cap * 4 : 0);
+  if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
+  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::decode_step_kernel<T, D, G>;
+  if (dev >= 0 && dev < 64 && attr_done[dev][cluster] < smem) {
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    attr_done[dev] = true;
+    if (cluster) {
+      e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+      if (e != cudaSuccess) return e;
+    }
+    attr_done[dev][cluster] = smem;
   }
-  wkv::decode_step_kernel<T, D, G><<<n_ctas, wkv::kThreads, C::kSmemBytes, stream>>>(P);
-  return cudaGetLastError();
+  if (!cluster) {
+    wkv::decode_step_kernel<T, D, G><<<n_ctas, wkv::kThreads, smem, stream>>>(P);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3((unsigned)n_ctas);
+  lc.blockDim = dim3(wkv::kThreads);
+  lc.dynamicSmemBytes = (size_t)smem;
+  lc.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = (unsigned)P.n_splits;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  lc.attrs = at;
+  lc.numAttrs = 1;
+  return cudaLaunchKernelEx(&lc, wkv::decode_step_cluster_kernel<T, D, G>, P);
 }
 
 template <typename T, int D>
-cudaError_t launch_by_group(int G, const wkv::StepParams& P, int n_ctas, cudaStream_t s) {
+cudaError_t launch_by_group(int G, const wkv::StepParams& P, int n_ctas, bool cluster, cudaStream_t s) {
   switch (G) {
-    case 1: return launch_step<T, D, 1>(P, n_ctas, s);
-    case 2: return launch_step<T, D, 2>(P, n_ctas, s);
-    case 4: return launch_step<T, D, 4>(P, n_ctas, s);
-    case 8: return launch_step<T, D, 8>(P, n_ctas, s);
+    case 1: return launch_step<T, D, 1>(P, n_ctas, cluster, s);
+    case 2: return launch_step<T, D, 2>(P, n_ctas, cluster, s);
+    case 4: return launch_step<T, D, 4>(P, n_ctas, cluster, s);
+    case 8: return launch_step<T, D, 8>(P, n_ctas, cluster, s);
   }
   return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P) {
+// cluster = false forces kernel A (global scratch), which the static-scratch entry point needs.
+cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P, bool cluster) {
   const int n_ctas = c->lanes_per_layer * c->n_splits;
   if (c->cfg.dtype == WKV_BF16) {
-    return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n_ctas, c->stream)
-                                  : launch_by_group<__nv_bfloat16, 64>(c->group, P, n_ctas, c->stream);
+    return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n_ctas, cluster, c->stream)
+                                  : launch_by_group<__nv_bfloat16, 64>(c->group, P, n_ctas, cluster, c->stream);
   }
-  return c->cfg.head_dim == 128 ? launch_by_group<float, 128>(c->group, P, n_ctas, c->stream)
-                                : launch_by_group<float, 64>(c->group, P, n_ctas, c->stream);
+  return c->cfg.head_dim == 128 ? launch_by_group<float, 128>(c->group, P, n_ctas, cluster, c->stream)
+                                : launch_by_group<float, 64>(c->group, P, n_ctas, cluster, c->stream);
 }
 
 wkv::StepParams base_params(const wkv_ctx* c, int layer) {
@@ -162,6 +191,7 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   P.cap = c->cap;
   P.budget = c->cfg.budget; P.window = c->cfg.window; P.sink = c->cfg.sink;
   P.n_splits = c->n_splits;
+  P.chunk_cap = c->chunk_cap;
   P.merge = c->cfg.merge;
   P.scale = c->scale;
   return P;
@@ -220,6 +250,12 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   c->lanes_total = (long long)cfg->n_layers * c->lanes_per_layer;
   c->cap = (cfg->budget + 1 + 3) & ~3;
   c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg);
+  {
+    const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+    c->chunk_cap = ((tiles + c->n_splits - 1) / c->n_splits) * wkv::kTileSlots;   // the largest share of an even deal
+    // kernel B needs a cluster-sized split count and room for the chunk's logits next to the ring
+    c->use_cluster = is_cluster_size(c->n_splits) && c->group * c->chunk_cap * 4 <= 64 * 1024;
+  }
   c->scale = cfg->scale != 0.f ? cfg->scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
   c->elem = cfg->dtype == WKV_BF16 ? 2 : 4;
   c->stream = reinterpret_cast<cudaStream_t>(cfg->stream);
@@ -285,7 +321,7 @@ int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, con
   P.ev_bs = c->cfg.n_kv_heads;
   P.seq_lens = nullptr;
   P.tok_idx = 0;
-  cudaError_t e = launch_any(c, P);
+  cudaError_t e = launch_any(c, P, c->use_cluster);
   c->launches++;
   if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch");
   return WKV_OK;
@@ -322,7 +358,7 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   P.tok_idx = 0;
   // the array keeps whatever the previous call (of any context) left: the arrival counters must start at zero
   WKV_CUDA(c, cudaMemsetAsync(base, 0, ticket_bytes, c->stream));
-  e = launch_any(c, P);
+  e = launch_any(c, P, false);
   c->launches++;
   if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (static scratch)");
   return WKV_OK;
@@ -366,7 +402,7 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
     P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
     P.out = out ? (void*)((char*)out + (size_t)t * Hq * D * c->elem) : c->stage_out;
     P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
-    cudaError_t e = launch_any(c, P);
+    cudaError_t e = launch_any(c, P, c->use_cluster);
     c->launches++;
     if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (prefill)");
   }

@@ -27,6 +27,7 @@
 //   merge : D = abar_j + abar_r; w_j = abar_j/D; w_r = abar_r/D; v = fma(w_j, v_j, w_r*v_r), rounded to T.
 // The attention output o_t is not part of that chain and uses fast exp2 with an online softmax.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -34,7 +35,7 @@
 namespace wkv {
 
 #ifndef WKV_RING_BYTES
-#define WKV_RING_BYTES 65536          // shared-memory ring per CTA (K and V tiles, all stages)
+#define WKV_RING_BYTES 32768          // shared-memory ring per CTA (K and V tiles, all stages)
 #endif
 constexpr int kTileSlots = 32;        // cache entries per pipeline stage
 constexpr int kConsumerWarps = 4;     // each owns 8 rows of a tile
@@ -73,6 +74,7 @@ struct StepParams {
   int cap;               // slots per lane (>= budget+1, multiple of 4)
   int budget, window, sink;
   int n_splits;
+  int chunk_cap;         // cluster kernel: logits one CTA can hold per query head (its tiles * 32)
   int merge;
   float scale;
 };
@@ -118,6 +120,10 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                    smem_u32(dst)),
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
+}
+// Hint: bring [src, src + bytes) into L2.  src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -196,271 +202,323 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long x)
 }
 
 // ------------------------------------------------------------------------------------------------
-// shared memory layout
+// compile-time shape of one instantiation and its shared-memory carve-up
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D, int G>
 struct Cfg {
-  static constexpr int EPL = D / 16;                        // channels per thread of a 16-thread row group
   static constexpr int kRowBytes = D * (int)sizeof(T);
   static constexpr int kTileBytes = kTileSlots * kRowBytes; // one of K or V
   static constexpr int kLanesPerRow = G <= 2 ? 8 : 16;      // threads that share one cache row in the scan
   static constexpr int kFit = WKV_RING_BYTES / (2 * kTileBytes);
   static constexpr int kStages = kFit < 2 ? 2 : (kFit > 8 ? 8 : kFit);
   static constexpr int kRingBytes = kStages * 2 * kTileBytes;
-  // after the ring: per-warp partials [warps][G][D+2], new k/v rows, barriers, epilogue scalars
   static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
-  static constexpr int kSmemBytes = kRingBytes + kWarpPartFloats * 4 + 2 * kRowBytes + 2 * kStages * 8 +
-                                    (G * kMaxSplits + 32 + 64) * 4 + 64 * 8 + 128;
+  static constexpr int kCtaPartFloats = G * (D + 2);
+  // ring | warp partials | CTA partial | new k, v rows | mbarriers | epilogue scalars | (cluster kernel: chunk logits)
+  static constexpr int kFixedBytes = kRingBytes + (kWarpPartFloats + kCtaPartFloats) * 4 + 2 * kRowBytes + 2 * kStages * 8 +
+                                     (G * kMaxSplits + 32 + 64) * 4 + 64 * 8 + 128;
 };
 
-// ------------------------------------------------------------------------------------------------
-// the fused decode step
-// ------------------------------------------------------------------------------------------------
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams P) {
-  using C = Cfg<T, D, G>;
-  constexpr int kStages = C::kStages;
-  const float kLog2e = 1.4426950408889634f;
-
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  unsigned char* ring = smem_raw;                                        // [stage][K tile | V tile]
-  float* warp_part = reinterpret_cast<float*>(ring + C::kRingBytes);    // [warp][G][D+2]
-  T* new_k = reinterpret_cast<T*>(warp_part + C::kWarpPartFloats);      // [D]
-  T* new_v = new_k + D;                                                 // [D]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(new_v + D);          // [kStages]
-  uint64_t* empty_bar = full_bar + kStages;                             // [kStages]
-  float* ep_w = reinterpret_cast<float*>(empty_bar + kStages);          // [G][kMaxSplits] split weights
-  float* ep_M = ep_w + G * kMaxSplits;                                  // [G] global max logit (8 reserved each)
-  float* ep_linv = ep_M + 8;                                            // [G]
-  float* ep_Z = ep_linv + 8;                                            // [G]
-  float* ep_misc = ep_Z + 8;                                            // [8] w_j, w_r
-  int* ep_int = reinterpret_cast<int*>(ep_misc + 8);                    // [64] flags, j, r
-  unsigned long long* ep_u64 = reinterpret_cast<unsigned long long*>(ep_int + 64);  // [64] reduction scratch
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
-  const int split = blockIdx.x % P.n_splits;
-  const int lane_local = blockIdx.x / P.n_splits;    // (b, kv head) of this layer
-  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
-  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed (ragged prefill)
-    if (split == 0 && tid == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
-    return;
+struct Smem {
+  unsigned char* ring;       // [stage][K tile | V tile]
+  float* warp_part;          // [warp][G][D+2] : m, l, o[D]
+  float* cta_part;           // [G][D+2]
+  T* new_k;                  // [D]
+  T* new_v;                  // [D]
+  uint64_t* full_bar;        // [kStages]
+  uint64_t* empty_bar;       // [kStages]
+  float* ep_w;               // [G][kMaxSplits] split weights of the output combination
+  float* ep_M;               // [8] global max logit per query head
+  float* ep_linv;            // [8]
+  float* ep_Z;               // [8]
+  float* ep_misc;            // [8] w_j, w_r
+  int* ep_int;               // [64] flags, j, r
+  unsigned long long* ep_u64;// [64] reduction scratch; [48..55] Z partial per head, [56] pick key of this CTA
+  float* chunk_logits;       // [G][chunk_cap] (cluster kernel only)
+  __device__ __forceinline__ explicit Smem(unsigned char* raw) {
+    using C = Cfg<T, D, G>;
+    ring = raw;
+    warp_part = reinterpret_cast<float*>(ring + C::kRingBytes);
+    cta_part = warp_part + C::kWarpPartFloats;
+    new_k = reinterpret_cast<T*>(cta_part + C::kCtaPartFloats);
+    new_v = new_k + D;
+    full_bar = reinterpret_cast<uint64_t*>(new_v + D);
+    empty_bar = full_bar + C::kStages;
+    ep_w = reinterpret_cast<float*>(empty_bar + C::kStages);
+    ep_M = ep_w + G * kMaxSplits;
+    ep_linv = ep_M + 8;
+    ep_Z = ep_linv + 8;
+    ep_misc = ep_Z + 8;
+    ep_int = reinterpret_cast<int*>(ep_misc + 8);
+    ep_u64 = reinterpret_cast<unsigned long long*>(ep_int + 64);
+    chunk_logits = reinterpret_cast<float*>(ep_u64 + 64);
   }
-  const long long lane = (long long)P.lane0 + lane_local;
-  int* st = P.lane_state + lane * LS_STRIDE;
-  const int len = st[LS_LEN], t = st[LS_T], new_slot = st[LS_FREE];
-  const int L = len + 1;                             // entries attended this step (new token included)
+};
 
-  const T* Kl = reinterpret_cast<const T*>(P.Kc) + lane * (long long)P.cap * D;
-  const T* Vl = reinterpret_cast<const T*>(P.Vc) + lane * (long long)P.cap * D;
-  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
-  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
-  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+// What a CTA knows about its lane and its share of the lane's slots.
+template <typename T>
+struct LaneView {
+  long long lane;            // global lane index
+  int lane_local, b, hk, split;
+  int len, t, new_slot, L;   // L = entries attended this step (new token included)
+  int tile_begin, n_tiles;   // this CTA's tiles
+  int slot_begin, slot_end;  // this CTA's slots [slot_begin, slot_end) clipped to L
+  const T *Kl, *Vl, *q_in, *k_in, *v_in;
+  int* st;
+  bool active;
+};
 
-  const int tiles_total = (L + kTileSlots - 1) / kTileSlots;
-  const int tps = (tiles_total + P.n_splits - 1) / P.n_splits;
-  const int tile_begin = split * tps;
-  const int tile_end = min(tiles_total, tile_begin + tps);
-  const int n_my_tiles = max(0, tile_end - tile_begin);
+template <typename T, int D, int G>
+__device__ __forceinline__ LaneView<T> open_lane(const StepParams& P, const Smem<T, D, G>& sm, int lane_local, int split) {
+  using C = Cfg<T, D, G>;
+  LaneView<T> v;
+  const int tid = threadIdx.x;
+  v.lane_local = lane_local;
+  v.split = split;
+  v.b = lane_local / P.n_kv_heads;
+  v.hk = lane_local % P.n_kv_heads;
+  v.active = !(P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[v.b]);   // sequence already consumed (ragged prefill)
+  if (!v.active) {
+    if (split == 0 && tid == 0 && P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = -1;
+    return v;
+  }
+  v.lane = (long long)P.lane0 + lane_local;
+  v.st = P.lane_state + v.lane * LS_STRIDE;
+  v.len = v.st[LS_LEN];
+  v.t = v.st[LS_T];
+  v.new_slot = v.st[LS_FREE];
+  v.L = v.len + 1;
+  v.Kl = reinterpret_cast<const T*>(P.Kc) + v.lane * (long long)P.cap * D;
+  v.Vl = reinterpret_cast<const T*>(P.Vc) + v.lane * (long long)P.cap * D;
+  v.q_in = reinterpret_cast<const T*>(P.q) + v.b * P.q_bs + (long long)v.hk * G * D;
+  v.k_in = reinterpret_cast<const T*>(P.k) + v.b * P.kv_bs + (long long)v.hk * D;
+  v.v_in = reinterpret_cast<const T*>(P.v) + v.b * P.kv_bs + (long long)v.hk * D;
+  // tiles are dealt out evenly: the first (tiles_total mod n_splits) CTAs take one more
+  const int tiles_total = (v.L + kTileSlots - 1) / kTileSlots;
+  const int base = tiles_total / P.n_splits, extra = tiles_total % P.n_splits;
+  v.tile_begin = split * base + min(split, extra);
+  v.n_tiles = base + (split < extra ? 1 : 0);
+  v.slot_begin = min(v.L, v.tile_begin * kTileSlots);
+  v.slot_end = min(v.L, (v.tile_begin + v.n_tiles) * kTileSlots);
 
+  if (tid == 32 && v.slot_end > v.slot_begin) {
+    // The epilogue reads a and pos of these slots long after the scan: pull their lines into L2 now.
+    const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);   // cap is a multiple of 4 slots
+    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
+    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
+  }
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], kConsumerWarps);
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(&sm.full_bar[s], 1);
+      mbar_init(&sm.empty_bar[s], kConsumerWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // the new token's rows: kept in shared memory for the scan (the cache copy of that slot may still be
-  // in flight) and written to the cache by the CTA whose chunk owns the slot
+  // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in
+  // flight) and written to the cache by the CTA whose chunk owns the slot.
   for (int c = tid; c < D; c += kThreads) {
-    new_k[c] = k_in[c];
-    new_v[c] = v_in[c];
+    sm.new_k[c] = v.k_in[c];
+    sm.new_v[c] = v.v_in[c];
   }
-  {
-    const int nt = new_slot / kTileSlots;
-    if (nt >= tile_begin && nt < tile_end) {
-      T* Kw = const_cast<T*>(Kl) + (long long)new_slot * D;
-      T* Vw = const_cast<T*>(Vl) + (long long)new_slot * D;
-      for (int c = tid; c < D; c += kThreads) {
-        Kw[c] = k_in[c];
-        Vw[c] = v_in[c];
-      }
+  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
+    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
+    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
+    for (int c = tid; c < D; c += kThreads) {
+      Kw[c] = v.k_in[c];
+      Vw[c] = v.v_in[c];
     }
   }
   __syncthreads();
+  return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// the scan: logits, online-softmax partial of o, logits parked at logit_dst[g*logit_stride + slot - logit_off]
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+__device__ __forceinline__ void scan_tiles(const StepParams& P, const Smem<T, D, G>& sm, const LaneView<T>& v,
+                                           float* logit_dst, long long logit_stride, int logit_off) {
+  using C = Cfg<T, D, G>;
+  constexpr int kStages = C::kStages;
+  const float kLog2e = 1.4426950408889634f;
+  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
+  const int L = v.L, new_slot = v.new_slot;
 
   if (warp == kConsumerWarps) {
     // ---------------- producer: one thread keeps the ring full ----------------
     if (lane_id == 0) {
-      for (int i = 0; i < n_my_tiles; ++i) {
+      for (int i = 0; i < v.n_tiles; ++i) {
         const int s = i % kStages;
-        if (i >= kStages) mbar_wait(&empty_bar[s], ((i / kStages) - 1) & 1, P.status);
-        const int slot0 = (tile_begin + i) * kTileSlots;
+        if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
+        const int slot0 = (v.tile_begin + i) * kTileSlots;
         const uint32_t bytes = (uint32_t)min(kTileSlots, L - slot0) * C::kRowBytes;
-        unsigned char* dst = ring + (size_t)s * 2 * C::kTileBytes;
-        mbar_expect_tx(&full_bar[s], 2 * bytes);
-        bulk_g2s(dst, Kl + (long long)slot0 * D, bytes, &full_bar[s]);
-        bulk_g2s(dst + C::kTileBytes, Vl + (long long)slot0 * D, bytes, &full_bar[s]);
+        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
+        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
+        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
       }
     }
-  } else {
-    // ---------------- consumers: 4 warps, each owns 8 rows of every tile ----------------
-    // A row (one cache entry) is shared by LPR threads.  Thread l of the group owns the partial sums
-    // {l, l+LPR, ...} of the reproducible dot, each a block of D/16 contiguous channels, so butterfly rounds
-    // with off >= LPR are additions inside the thread and only log2(LPR) shuffles remain.
-    constexpr int LPR = C::kLanesPerRow;           // 8 or 16 threads per row
-    constexpr int NP = 16 / LPR;                   // partial sums per thread
-    constexpr int CH = D / 16;                     // channels per partial sum
-    constexpr int RPP = 32 / LPR;                  // rows per warp pass
-    constexpr int PASSES = 8 / RPP;
-    const int rg = lane_id / LPR, l = lane_id % LPR;
-    float qf[G][NP][CH];
+    return;
+  }
+  // ---------------- consumers: 4 warps, each owns 8 rows of every tile ----------------
+  // A row (one cache entry) is shared by LPR threads.  Thread l of the group owns the partial sums
+  // {l, l+LPR, ...} of the reproducible dot, each a block of D/16 contiguous channels, so butterfly rounds
+  // with off >= LPR are additions inside the thread and only log2(LPR) shuffles remain.
+  constexpr int LPR = C::kLanesPerRow;           // 8 or 16 threads per row
+  constexpr int NP = 16 / LPR;                   // partial sums per thread
+  constexpr int CH = D / 16;                     // channels per partial sum
+  constexpr int RPP = 32 / LPR;                  // rows per warp pass
+  constexpr int PASSES = 8 / RPP;
+  const int rg = lane_id / LPR, l = lane_id % LPR;
+  float qf[G][NP][CH];
 #pragma unroll
-    for (int g = 0; g < G; ++g)
+  for (int g = 0; g < G; ++g)
 #pragma unroll
-      for (int j = 0; j < NP; ++j) load_chunk<CH>(q_in + g * D + (l + LPR * j) * CH, qf[g][j]);
-    float m_run[G], l_run[G], o_acc[G][NP][CH];
+    for (int j = 0; j < NP; ++j) load_chunk<CH>(v.q_in + g * D + (l + LPR * j) * CH, qf[g][j]);
+  float m_run[G], l_run[G], o_acc[G][NP][CH];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    m_run[g] = -INFINITY;
+    l_run[g] = 0.f;
+#pragma unroll
+    for (int j = 0; j < NP; ++j)
+#pragma unroll
+      for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
+  }
+
+  for (int i = 0; i < v.n_tiles; ++i) {
+    const int s = i % kStages;
+    mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
+    T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
+    T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+    const int slot0 = (v.tile_begin + i) * kTileSlots;
+    {
+      // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
+      // row in the tile with the token's k and v before anybody reads it.
+      const int ns_row = new_slot - slot0;
+      if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
+        uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
+        uint32_t* dv = reinterpret_cast<uint32_t*>(tV + ns_row * D);
+        const uint32_t* sk = reinterpret_cast<const uint32_t*>(sm.new_k);
+        const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(sm.new_v);
+        for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; dv[w] = sv_[w]; }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
+        __syncwarp();
+      }
+    }
+
+    float sv[G][PASSES];
+    bool valid[PASSES];
+#pragma unroll
+    for (int ps = 0; ps < PASSES; ++ps) {
+      const int row = warp * 8 + ps * RPP + rg;
+      valid[ps] = slot0 + row < L;
+      float kf[NP][CH];
+#pragma unroll
+      for (int j = 0; j < NP; ++j) load_chunk<CH>(tK + row * D + (l + LPR * j) * CH, kf[j]);
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float pp[NP];
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+          float acc = 0.f;
+#pragma unroll
+          for (int e = 0; e < CH; ++e) acc = __fmaf_rn(qf[g][j][e], kf[j][e], acc);
+          pp[j] = acc;
+        }
+        float acc = pp[0];
+        if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
+#pragma unroll
+        for (int off = LPR / 2; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+        const float sc = __fmul_rn(P.scale, acc);
+        sv[g][ps] = valid[ps] ? sc : -INFINITY;
+      }
+    }
+    // park the logits: thread l (< PASSES) of row group rg owns row warp*8 + l*RPP + rg
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      m_run[g] = -INFINITY;
-      l_run[g] = 0.f;
+      float mine = sv[g][0];
+#pragma unroll
+      for (int ps = 1; ps < PASSES; ++ps) mine = l == ps ? sv[g][ps] : mine;
+      const int slot = slot0 + warp * 8 + l * RPP + rg;
+      if (l < PASSES && slot < L) logit_dst[(long long)g * logit_stride + (slot - logit_off)] = mine;
+    }
+    // online softmax update, one rescale per tile
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float mt = sv[g][0];
+#pragma unroll
+      for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[g][ps]);
+      const float m_new = fmaxf(m_run[g], mt);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
+      m_run[g] = m_new;
+      l_run[g] *= corr;
 #pragma unroll
       for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
+        for (int e = 0; e < CH; ++e) o_acc[g][j][e] *= corr;
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps) sv[g][ps] = fast_exp2((sv[g][ps] - m_use) * kLog2e);   // now probabilities
     }
-    float* logit_base = P.logits + (long long)lane_local * G * P.cap;
-
-    for (int i = 0; i < n_my_tiles; ++i) {
-      const int s = i % kStages;
-      mbar_wait(&full_bar[s], (i / kStages) & 1, P.status);
-      T* tK = reinterpret_cast<T*>(ring + (size_t)s * 2 * C::kTileBytes);
-      T* tV = reinterpret_cast<T*>(ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
-      const int slot0 = (tile_begin + i) * kTileSlots;
-      {
-        // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
-        // row in the tile with the token's k and v before anybody reads it.
-        const int ns_row = new_slot - slot0;
-        if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
-          uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
-          uint32_t* dv = reinterpret_cast<uint32_t*>(tV + ns_row * D);
-          const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
-          const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
-          for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; dv[w] = sv_[w]; }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
-          __syncwarp();
-        }
-      }
-
-      float sv[G][PASSES];
-      bool valid[PASSES];
 #pragma unroll
-      for (int ps = 0; ps < PASSES; ++ps) {
-        const int row = warp * 8 + ps * RPP + rg;
-        valid[ps] = slot0 + row < L;
-        float kf[NP][CH];
+    for (int ps = 0; ps < PASSES; ++ps) {
+      const int row = warp * 8 + ps * RPP + rg;
+      float vf[NP][CH];
 #pragma unroll
-        for (int j = 0; j < NP; ++j) load_chunk<CH>(tK + row * D + (l + LPR * j) * CH, kf[j]);
+      for (int j = 0; j < NP; ++j) load_chunk<CH>(tV + row * D + (l + LPR * j) * CH, vf[j]);
+      if (valid[ps]) {
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          float pp[NP];
+          l_run[g] += sv[g][ps];
 #pragma unroll
-          for (int j = 0; j < NP; ++j) {
-            float acc = 0.f;
+          for (int j = 0; j < NP; ++j)
 #pragma unroll
-            for (int e = 0; e < CH; ++e) acc = __fmaf_rn(qf[g][j][e], kf[j][e], acc);
-            pp[j] = acc;
-          }
-          float acc = pp[0];
-          if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
-#pragma unroll
-          for (int off = LPR / 2; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-          const float sc = __fmul_rn(P.scale, acc);
-          sv[g][ps] = valid[ps] ? sc : -INFINITY;
+            for (int e = 0; e < CH; ++e) o_acc[g][j][e] = fmaf(sv[g][ps], vf[j][e], o_acc[g][j][e]);
         }
       }
-      // park the logits: thread l (< PASSES) of row group rg owns row warp*8 + l*RPP + rg
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float mine = sv[g][0];
-#pragma unroll
-        for (int ps = 1; ps < PASSES; ++ps) mine = l == ps ? sv[g][ps] : mine;
-        const int slot = slot0 + warp * 8 + l * RPP + rg;
-        if (l < PASSES && slot < L) logit_base[(long long)g * P.cap + slot] = mine;
-      }
-      // online softmax update, one rescale per tile
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float mt = sv[g][0];
-#pragma unroll
-        for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[g][ps]);
-        const float m_new = fmaxf(m_run[g], mt);
-        const float m_use = m_new == -INFINITY ? 0.f : m_new;
-        const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
-        m_run[g] = m_new;
-        l_run[g] *= corr;
-#pragma unroll
-        for (int j = 0; j < NP; ++j)
-#pragma unroll
-          for (int e = 0; e < CH; ++e) o_acc[g][j][e] *= corr;
-#pragma unroll
-        for (int ps = 0; ps < PASSES; ++ps) sv[g][ps] = fast_exp2((sv[g][ps] - m_use) * kLog2e);   // now probabilities
-      }
-#pragma unroll
-      for (int ps = 0; ps < PASSES; ++ps) {
-        const int row = warp * 8 + ps * RPP + rg;
-        float vf[NP][CH];
-#pragma unroll
-        for (int j = 0; j < NP; ++j) load_chunk<CH>(tV + row * D + (l + LPR * j) * CH, vf[j]);
-        if (valid[ps]) {
-#pragma unroll
-          for (int g = 0; g < G; ++g) {
-            l_run[g] += sv[g][ps];
-#pragma unroll
-            for (int j = 0; j < NP; ++j)
-#pragma unroll
-              for (int e = 0; e < CH; ++e) o_acc[g][j][e] = fmaf(sv[g][ps], vf[j][e], o_acc[g][j][e]);
-          }
-        }
-      }
-      __syncwarp();
-      if (lane_id == 0) mbar_arrive(&empty_bar[s]);
     }
-
-    // fold the row groups of the warp, then leave the warp's partial in shared memory
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-#pragma unroll
-      for (int off = 16; off >= LPR; off >>= 1) {
-        const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
-        const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
-        const float m_new = fmaxf(m_run[g], m_o);
-        const float m_use = m_new == -INFINITY ? 0.f : m_new;
-        const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
-        l_run[g] = l_run[g] * c_me + l_o * c_o;
-        m_run[g] = m_new;
-#pragma unroll
-        for (int j = 0; j < NP; ++j)
-#pragma unroll
-          for (int e = 0; e < CH; ++e) {
-            const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
-            o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
-          }
-      }
-      float* wp = warp_part + (warp * G + g) * (D + 2);
-      if (rg == 0) {
-#pragma unroll
-        for (int j = 0; j < NP; ++j)
-#pragma unroll
-          for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
-      }
-      if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
-    }
+    __syncwarp();
+    if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
   }
-  __syncthreads();
 
-  // ---------------- CTA partial -> global scratch ----------------
-  float* my_part = P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2);
-  for (int idx = tid; idx < G * D; idx += kThreads) {
+  // fold the row groups of the warp, then leave the warp's partial in shared memory
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+#pragma unroll
+    for (int off = 16; off >= LPR; off >>= 1) {
+      const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
+      const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
+      const float m_new = fmaxf(m_run[g], m_o);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
+      l_run[g] = l_run[g] * c_me + l_o * c_o;
+      m_run[g] = m_new;
+#pragma unroll
+      for (int j = 0; j < NP; ++j)
+#pragma unroll
+        for (int e = 0; e < CH; ++e) {
+          const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
+          o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
+        }
+    }
+    float* wp = sm.warp_part + (warp * G + g) * (D + 2);
+    if (rg == 0) {
+#pragma unroll
+      for (int j = 0; j < NP; ++j)
+#pragma unroll
+        for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
+    }
+    if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
+  }
+}
+
+// The four warp partials -> one (m, l, o[D]) per query head at dst (shared or global).  Call after __syncthreads().
+template <int D, int G>
+__device__ __forceinline__ void combine_warps(const float* warp_part, float* dst) {
+  const float kLog2e = 1.4426950408889634f;
+  for (int idx = threadIdx.x; idx < G * D; idx += kThreads) {
     const int g = idx / D, c = idx % D;
     float mx = -INFINITY;
 #pragma unroll
@@ -474,23 +532,234 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams 
       o += wp[2 + c] * cw;
       l += wp[1] * cw;
     }
-    my_part[g * (D + 2) + 2 + c] = o;
-    if (c == 0) { my_part[g * (D + 2)] = mx; my_part[g * (D + 2) + 1] = l; }
+    dst[g * (D + 2) + 2 + c] = o;
+    if (c == 0) { dst[g * (D + 2)] = mx; dst[g * (D + 2) + 1] = l; }
   }
+}
+
+// ------------------------------------------------------------------------------------------------
+// epilogue pieces (reproducible arithmetic)
+// ------------------------------------------------------------------------------------------------
+// e_i = exp(s_i - M_g), written back in place of the logit, and this thread's share of sum_i trunc(e_i * 2^40).
+// Element i of the range lives at lg[g*stride + i]; kL2 selects loads that bypass L1 (logits written by other SMs).
+template <int G, bool kL2>
+__device__ __forceinline__ void exp_and_zsum(float* lg, long long stride, int n, const float* M, unsigned long long (&zl)[G]) {
+  constexpr int U = 4;                          // loads of U elements are issued before any of them is used
+#pragma unroll
+  for (int g = 0; g < G; ++g) zl[g] = 0ull;
+  for (int i0 = threadIdx.x; i0 < n; i0 += kThreads * U) {
+    float sx[G][U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kThreads;
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        const float* p = lg + (long long)g * stride + i;
+        sx[g][u] = i < n ? (kL2 ? __ldcg(p) : *p) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kThreads;
+      if (i < n) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float e = repro_exp(__fsub_rn(sx[g][u], M[g]));
+          lg[(long long)g * stride + i] = e;    // re-read by the same thread in fold_scores
+          zl[g] += __float2ull_rz(__fmul_rn(e, 1099511627776.0f));
+        }
+      }
+    }
+  }
+}
+
+// Block-wide sums of G 64-bit integers; result[g] valid in every thread after the call.  scratch: 8*G + ... entries.
+template <int G>
+__device__ __forceinline__ void block_sum_u64(unsigned long long (&x)[G], unsigned long long* scratch) {
+  const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const unsigned long long w = warp_sum_u64(x[g]);
+    if (lane_id == 0) scratch[g * 5 + warp] = w;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    unsigned long long z = 0ull;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) z += scratch[g * 5 + w];
+    x[g] = z;
+  }
+  __syncthreads();
+}
+
+// A_t over a range of slots, a = [a,0] + A_t, abar = a/n and the range's pick key (Algorithm 1).
+// e values at lg[g*stride + i] for slot slot0 + i.  Returns the thread's best (key, slot).
+template <typename T, int G>
+__device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<T>& v, const float* lg, long long stride,
+                                            int slot0, int n, const float* Z, bool compress, unsigned long long& best,
+                                            int& best_slot) {
+  float* a_l = P.a + v.lane * P.cap;
+  int32_t* pos_l = P.pos + v.lane * P.cap;
+  const int t = v.t;
+  constexpr int U = 4;                          // a, pos and e of U slots are loaded before any of them is used
+  for (int i0 = threadIdx.x; i0 < n; i0 += kThreads * U) {
+    float a_old[U], ev[G][U];
+    int pos_v[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kThreads;
+      const int slot = slot0 + i;
+      const bool ok = i < n, is_new = slot == v.new_slot;
+      a_old[u] = (ok && !is_new) ? a_l[slot] : 0.f;
+      pos_v[u] = (ok && !is_new) ? pos_l[slot] : t;
+#pragma unroll
+      for (int g = 0; g < G; ++g) ev[g][u] = ok ? lg[(long long)g * stride + i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int i = i0 + u * kThreads;
+      if (i >= n) continue;
+      const int slot = slot0 + i;
+      float pg[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        pg[g] = __fdiv_rn(ev[g][u], Z[g]);
+        if (P.probs)
+          P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + slot] = pg[g];
+      }
+      float pbar = pg[0];
+#pragma unroll
+      for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pg[g]);
+      if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
+      const float a_new = __fadd_rn(a_old[u], pbar);
+      const int pos_i = pos_v[u];
+      a_l[slot] = a_new;
+      if (slot == v.new_slot) pos_l[slot] = t;
+      if (compress && pos_i >= P.sink && pos_i <= t - P.window) {
+        const float abar = __fdiv_rn(a_new, __int2float_rn(t - pos_i + 1));
+        const unsigned long long key = ((unsigned long long)__float_as_uint(abar) << 32) | (uint32_t)pos_i;
+        if (key < best) { best = key; best_slot = slot; }
+      }
+    }
+  }
+}
+
+// Block-wide minimum of the pick key; returns it in every thread and leaves the owning slot in *slot_out (shared).
+__device__ __forceinline__ unsigned long long block_min_key(unsigned long long best, int best_slot, unsigned long long* scratch,
+                                                            int* slot_out) {
+  const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+  const unsigned long long wmin = warp_min_u64(best);
+  if (lane_id == 0) scratch[warp] = wmin;
+  if (threadIdx.x == 0) *slot_out = -1;
+  __syncthreads();
+  unsigned long long bmin = scratch[0];
+#pragma unroll
+  for (int w = 1; w < kThreads / 32; ++w) bmin = scratch[w] < bmin ? scratch[w] : bmin;
+  if (best == bmin && best_slot >= 0) *slot_out = best_slot;       // positions are unique: one owner
+  __syncthreads();
+  return bmin;
+}
+
+// Link the new entry as the chain's tail, unlink the victim j (Algorithm 1: remove K[j], a[j], n[j]; the right
+// neighbour keeps its own key, a and n), merge V[j] into V[next[j]], update the lane state.  One CTA per lane runs it.
+template <typename T, int D, int G>
+__device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const Smem<T, D, G>& sm, bool compress,
+                                            unsigned long long bmin, int j_slot) {
+  const int tid = threadIdx.x;
+  const int t = v.t, new_slot = v.new_slot, L = v.L;
+  float* a_l = P.a + v.lane * P.cap;
+  int32_t* pos_l = P.pos + v.lane * P.cap;
+  int32_t* next_l = P.next + v.lane * P.cap;
+  int32_t* prev_l = P.prev + v.lane * P.cap;
+  if (tid == 0) {
+    int head = v.st[LS_HEAD], tail = v.st[LS_TAIL];
+    next_l[new_slot] = -1;
+    prev_l[new_slot] = tail;
+    if (tail >= 0) next_l[tail] = new_slot; else head = new_slot;
+    tail = new_slot;
+    int ev_pos = -1, new_len = L, new_free = L;          // while growing, slots fill in arrival order
+    sm.ep_int[2] = -1;
+    if (compress) {
+      const int j = j_slot;
+      const int r = j >= 0 ? next_l[j] : -1;
+      if (j < 0 || r < 0 || r >= P.cap) {
+        atomicOr(P.status, kStatusBadLink);              // cannot happen with budget >= sink + window
+      } else {
+        const float abar_j = __uint_as_float((uint32_t)(bmin >> 32));
+        const int pos_r = r == new_slot ? t : __ldcg(pos_l + r);
+        const float abar_r = __fdiv_rn(__ldcg(a_l + r), __int2float_rn(t - pos_r + 1));
+        const float Dn = __fadd_rn(abar_j, abar_r);
+        float wj = 0.5f, wr = 0.5f;
+        if (Dn != 0.f) { wj = __fdiv_rn(abar_j, Dn); wr = __fdiv_rn(abar_r, Dn); }
+        sm.ep_misc[0] = wj;
+        sm.ep_misc[1] = wr;
+        sm.ep_int[2] = j;
+        sm.ep_int[3] = r;
+        ev_pos = (int)(uint32_t)(bmin & 0xffffffffull);
+        const int pv = prev_l[j];
+        if (pv >= 0) next_l[pv] = r; else head = r;
+        prev_l[r] = pv;
+        pos_l[j] = -1;
+        new_len = P.budget;
+        new_free = j;
+      }
+    }
+    v.st[LS_LEN] = new_len;
+    v.st[LS_T] = t + 1;
+    v.st[LS_HEAD] = head;
+    v.st[LS_TAIL] = tail;
+    v.st[LS_FREE] = new_free;
+    if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = ev_pos;
+  }
+  __syncthreads();
+  // V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r), stored in T
+  if (compress && P.merge && sm.ep_int[2] >= 0) {
+    const int j = sm.ep_int[2], r = sm.ep_int[3];
+    const float wj = sm.ep_misc[0], wr = sm.ep_misc[1];
+    T* Vw = const_cast<T*>(v.Vl);
+    for (int c = tid; c < D; c += kThreads) {
+      // the row of this step's token may have been written to the cache by another CTA: take it from shared memory
+      const float vj = to_f32(j == new_slot ? sm.new_v[c] : __ldcg(Vw + (long long)j * D + c));
+      const float vr = to_f32(r == new_slot ? sm.new_v[c] : __ldcg(Vw + (long long)r * D + c));
+      Vw[(long long)r * D + c] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel A: any split count.  Partials and logits go through global scratch; the CTA that arrives last for a
+// lane (atomic ticket -- nobody waits) runs the whole epilogue.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams P) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const Smem<T, D, G> sm(smem_raw);
+  const float kLog2e = 1.4426950408889634f;
+  const int tid = threadIdx.x;
+  const int split = blockIdx.x % P.n_splits;
+  const int lane_local = blockIdx.x / P.n_splits;
+  const LaneView<T> v = open_lane<T, D, G>(P, sm, lane_local, split);
+  if (!v.active) return;
+  const int L = v.L;
+  float* lg = P.logits + (long long)lane_local * G * P.cap;
+
+  scan_tiles<T, D, G>(P, sm, v, lg, P.cap, 0);
+  __syncthreads();
+  combine_warps<D, G>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
   __syncthreads();
   if (tid == 0) {
     // release: the barrier ordered every thread's partials and logits before this fence (cumulativity)
     __threadfence();
     const uint32_t prev = atomicAdd(&P.ticket[lane_local], 1u);
     __threadfence();   // acquire side for the CTA that turns out to be the last
-    ep_int[0] = (prev == (uint32_t)P.n_splits - 1) ? 1 : 0;
+    sm.ep_int[0] = (prev == (uint32_t)P.n_splits - 1) ? 1 : 0;
+    if (sm.ep_int[0]) P.ticket[lane_local] = 0u;          // ready for the next launch
   }
   __syncthreads();
-  if (!ep_int[0]) return;
+  if (!sm.ep_int[0]) return;
 
-  // =====================================================================================
-  // Epilogue, run by the last CTA of the lane.
-  // =====================================================================================
+  // ---- epilogue, run by the last CTA of the lane ----
   // (1) split weights and the global max / normaliser of every query head
   if (tid < G) {
     const int g = tid;
@@ -500,157 +769,152 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams 
     float lsum = 0.f;
     for (int s = 0; s < P.n_splits; ++s) {
       const float w = fast_exp2((__ldcg(pg + (long long)s * G * (D + 2)) - M) * kLog2e);
-      ep_w[g * kMaxSplits + s] = w;
+      sm.ep_w[g * kMaxSplits + s] = w;
       lsum += w * __ldcg(pg + (long long)s * G * (D + 2) + 1);
     }
-    ep_M[g] = M;                       // max of the reproducible logits: exact, order-free
-    ep_linv[g] = 1.f / lsum;
+    sm.ep_M[g] = M;                    // max of the reproducible logits: exact, order-free
+    sm.ep_linv[g] = 1.f / lsum;
   }
   __syncthreads();
-  // (2) o_t = A_t^T V_t  (Background section), V as it was before this step's merge
+  // (2) o_t = A_t^T V_t (Background section), V as it was before this step's merge
   {
-    T* out = reinterpret_cast<T*>(P.out) + b * P.out_bs + (long long)hk * G * D;
+    T* out = reinterpret_cast<T*>(P.out) + v.b * P.out_bs + (long long)v.hk * G * D;
     for (int idx = tid; idx < G * D; idx += kThreads) {
       const int g = idx / D, c = idx % D;
       const float* pg = P.part + (long long)lane_local * P.n_splits * G * (D + 2) + g * (D + 2) + 2 + c;
       float o = 0.f;
-      for (int s = 0; s < P.n_splits; ++s) o += ep_w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
-      out[idx] = from_f32<T>(o * ep_linv[g]);
+      for (int s = 0; s < P.n_splits; ++s) o += sm.ep_w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
+      out[idx] = from_f32<T>(o * sm.ep_linv[g]);
     }
   }
-  // (3) Z_g = sum_i exp(s_i - M_g) as an exact integer sum
-  const float* lg = P.logits + (long long)lane_local * G * P.cap;
+  // (3) Z_g as an exact integer sum
   {
     unsigned long long zl[G];
-#pragma unroll
-    for (int g = 0; g < G; ++g) zl[g] = 0ull;
-    for (int i = tid; i < L; i += kThreads) {
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float e = repro_exp(__fsub_rn(__ldcg(lg + (long long)g * P.cap + i), ep_M[g]));
-        zl[g] += __float2ull_rz(__fmul_rn(e, 1099511627776.0f));
-      }
-    }
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const unsigned long long w = warp_sum_u64(zl[g]);
-      if (lane_id == 0) ep_u64[g * 8 + warp] = w;
-    }
-    __syncthreads();
+    exp_and_zsum<G, true>(lg, P.cap, L, sm.ep_M, zl);
+    block_sum_u64<G>(zl, sm.ep_u64);
     if (tid < G) {
-      unsigned long long z = 0ull;
-      for (int w = 0; w < kThreads / 32; ++w) z += ep_u64[tid * 8 + w];
-      ep_Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        if (g == tid) sm.ep_Z[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
     }
     __syncthreads();
   }
-  // (4) A_t, a = [a,0] + A_t, abar = a/n, candidate key  (Algorithm 1)
-  float* a_l = P.a + lane * P.cap;
-  int32_t* pos_l = P.pos + lane * P.cap;
+  // (4) probabilities, score fold, pick
   const bool compress = L > P.budget;                 // "length of V_t exceeds m"
-  unsigned long long best = ~0ull, bmin = ~0ull;
+  unsigned long long best = ~0ull;
   int best_slot = -1;
-  for (int i = tid; i < L; i += kThreads) {
-    float pbar;
-    {
-      float pg[G];
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float e = repro_exp(__fsub_rn(__ldcg(lg + (long long)g * P.cap + i), ep_M[g]));
-        pg[g] = __fdiv_rn(e, ep_Z[g]);
-        if (P.probs) P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = pg[g];
-      }
-      pbar = pg[0];
-#pragma unroll
-      for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pg[g]);
-      if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
-    }
-    const bool is_new = i == new_slot;
-    const float a_new = __fadd_rn(is_new ? 0.f : a_l[i], pbar);
-    const int pos_i = is_new ? t : pos_l[i];
-    a_l[i] = a_new;
-    if (is_new) pos_l[i] = t;
-    if (compress && pos_i >= P.sink && pos_i <= t - P.window) {
-      const float abar = __fdiv_rn(a_new, __int2float_rn(t - pos_i + 1));
-      const unsigned long long key = ((unsigned long long)__float_as_uint(abar) << 32) | (uint32_t)pos_i;
-      if (key < best) { best = key; best_slot = i; }
-    }
-  }
+  fold_scores<T, G>(P, v, lg, P.cap, 0, L, sm.ep_Z, compress, best, best_slot);
   if (P.probs) {
     for (int i = L + tid; i < P.budget + 1; i += kThreads)
 #pragma unroll
       for (int g = 0; g < G; ++g)
-        P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = 0.f;
+        P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
   }
-  {
-    const unsigned long long wmin = warp_min_u64(best);
-    if (lane_id == 0) ep_u64[32 + warp] = wmin;
-    __syncthreads();                                     // also publishes a_l / pos_l written above to the block
-    bmin = ep_u64[32];
-    for (int w = 1; w < kThreads / 32; ++w) bmin = ep_u64[32 + w] < bmin ? ep_u64[32 + w] : bmin;
-    if (tid == 0) ep_int[1] = -1;
-    __syncthreads();
-    if (compress && best == bmin && best_slot >= 0) ep_int[1] = best_slot;   // positions are unique: one owner
-    __syncthreads();
-  }
-  // (5) link the new entry as the chain's tail; unlink the victim; merge weights
-  int32_t* next_l = P.next + lane * P.cap;
-  int32_t* prev_l = P.prev + lane * P.cap;
-  if (tid == 0) {
-    int head = st[LS_HEAD], tail = st[LS_TAIL];
-    next_l[new_slot] = -1;
-    prev_l[new_slot] = tail;
-    if (tail >= 0) next_l[tail] = new_slot; else head = new_slot;
-    tail = new_slot;
-    int ev_pos = -1, new_len = L, new_free = L;          // while growing, slots fill in arrival order
-    ep_int[2] = -1;
-    if (compress) {
-      const int j = ep_int[1];
-      const int r = next_l[j];
-      if (j < 0 || r < 0 || r >= P.cap) {
-        atomicOr(P.status, kStatusBadLink);              // cannot happen with budget >= sink + window
-      } else {
-        const float abar_j = __uint_as_float((uint32_t)(bmin >> 32));
-        const int pos_r = pos_l[r];
-        const float abar_r = __fdiv_rn(a_l[r], __int2float_rn(t - pos_r + 1));
-        const float Dn = __fadd_rn(abar_j, abar_r);
-        float wj = 0.5f, wr = 0.5f;
-        if (Dn != 0.f) { wj = __fdiv_rn(abar_j, Dn); wr = __fdiv_rn(abar_r, Dn); }
-        ep_misc[0] = wj;
-        ep_misc[1] = wr;
-        ep_int[2] = j;
-        ep_int[3] = r;
-        ev_pos = (int)(uint32_t)(bmin & 0xffffffffull);
-        // Algorithm 1: remove K[j], a[j], n[j]; the neighbour keeps its own key, a and n
-        const int pv = prev_l[j];
-        if (pv >= 0) next_l[pv] = r; else head = r;
-        prev_l[r] = pv;
-        pos_l[j] = -1;
-        new_len = P.budget;
-        new_free = j;
+  const unsigned long long bmin = block_min_key(best, best_slot, sm.ep_u64 + 40, &sm.ep_int[1]);   // also publishes a, pos
+  // (5), (6)
+  finish_lane<T, D, G>(P, v, sm, compress, bmin, sm.ep_int[1]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel B: the n_splits CTAs of a lane form one thread-block cluster (n_splits in {1,2,4,8,16}).  Logits stay in
+// each CTA's shared memory, partials are read through distributed shared memory, and every CTA folds its own
+// slots, so the epilogue runs on all the cluster's threads.  Cluster barriers are hardware barriers among
+// co-scheduled CTAs; every CTA of an active lane reaches every barrier.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const StepParams P) {
+  namespace cg = cooperative_groups;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const Smem<T, D, G> sm(smem_raw);
+  const float kLog2e = 1.4426950408889634f;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x;
+  const int S = P.n_splits;
+  const int split = (int)cluster.block_rank();
+  const int lane_local = blockIdx.x / S;
+  const LaneView<T> v = open_lane<T, D, G>(P, sm, lane_local, split);
+  if (!v.active) return;                                // same decision in every CTA of the cluster
+  const int n_mine = v.slot_end - v.slot_begin;
+
+  scan_tiles<T, D, G>(P, sm, v, sm.chunk_logits, P.chunk_cap, v.slot_begin);
+  __syncthreads();
+  combine_warps<D, G>(sm.warp_part, sm.cta_part);
+  cluster.sync();                                       // #1: every CTA's partial is readable
+
+  // (1) global max per head (every CTA), output weights (rank 0)
+  if (tid < G) {
+    const int g = tid;
+    float M = -INFINITY;
+    for (int s = 0; s < S; ++s) M = fmaxf(M, cluster.map_shared_rank(sm.cta_part, s)[g * (D + 2)]);
+    sm.ep_M[g] = M;
+    if (split == 0) {
+      float lsum = 0.f;
+      for (int s = 0; s < S; ++s) {
+        const float* pp = cluster.map_shared_rank(sm.cta_part, s) + g * (D + 2);
+        const float w = fast_exp2((pp[0] - M) * kLog2e);
+        sm.ep_w[g * kMaxSplits + s] = w;
+        lsum += w * pp[1];
       }
+      sm.ep_linv[g] = 1.f / lsum;
     }
-    st[LS_LEN] = new_len;
-    st[LS_T] = t + 1;
-    st[LS_HEAD] = head;
-    st[LS_TAIL] = tail;
-    st[LS_FREE] = new_free;
-    if (P.evicted) P.evicted[b * P.ev_bs + hk] = ev_pos;
-    P.ticket[lane_local] = 0u;                            // ready for the next launch
   }
   __syncthreads();
-  // (6) V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r)   (Algorithm 1), stored in T
-  if (compress && P.merge && ep_int[2] >= 0) {
-    const int j = ep_int[2], r = ep_int[3];
-    const float wj = ep_misc[0], wr = ep_misc[1];
-    T* Vw = const_cast<T*>(Vl);
-    for (int c = tid; c < D; c += kThreads) {
-      // the row of this step's token may have been written to the cache by another CTA: take it from shared memory
-      const float vj = to_f32(j == new_slot ? new_v[c] : __ldcg(Vw + (long long)j * D + c));
-      const float vr = to_f32(r == new_slot ? new_v[c] : __ldcg(Vw + (long long)r * D + c));
-      Vw[(long long)r * D + c] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
+  // (2) o_t by rank 0
+  if (split == 0) {
+    T* out = reinterpret_cast<T*>(P.out) + v.b * P.out_bs + (long long)v.hk * G * D;
+    for (int idx = tid; idx < G * D; idx += kThreads) {
+      const int g = idx / D, c = idx % D;
+      float o = 0.f;
+      for (int s = 0; s < S; ++s) o += sm.ep_w[g * kMaxSplits + s] * cluster.map_shared_rank(sm.cta_part, s)[g * (D + 2) + 2 + c];
+      out[idx] = from_f32<T>(o * sm.ep_linv[g]);
     }
   }
+  // (3) this CTA's share of Z
+  {
+    unsigned long long zl[G];
+    exp_and_zsum<G, false>(sm.chunk_logits, P.chunk_cap, n_mine, sm.ep_M, zl);
+    block_sum_u64<G>(zl, sm.ep_u64);
+    if (tid == 0) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) sm.ep_u64[48 + g] = zl[g];
+    }
+  }
+  cluster.sync();                                       // #2: Z partials readable (and rank 0 is done with the o partials)
+  if (tid < G) {
+    unsigned long long z = 0ull;
+    for (int s = 0; s < S; ++s) z += cluster.map_shared_rank(sm.ep_u64, s)[48 + tid];
+    sm.ep_Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
+  }
+  __syncthreads();
+  // (4) probabilities, score fold and pick over this CTA's slots
+  const bool compress = v.L > P.budget;
+  unsigned long long best = ~0ull;
+  int best_slot = -1;
+  fold_scores<T, G>(P, v, sm.chunk_logits, P.chunk_cap, v.slot_begin, n_mine, sm.ep_Z, compress, best, best_slot);
+  if (P.probs && split == S - 1) {
+    for (int i = v.L + tid; i < P.budget + 1; i += kThreads)
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
+  }
+  const unsigned long long my_min = block_min_key(best, best_slot, sm.ep_u64 + 40, &sm.ep_int[1]);
+  if (tid == 0) sm.ep_u64[56] = my_min;
+  cluster.sync();                                       // #3: keys readable; a and pos of every slot are written
+  // (5) rank 0 gathers the lane's pick
+  unsigned long long bmin = ~0ull;
+  if (split == 0 && tid == 0) {
+    int j = -1;
+    for (int s = 0; s < S; ++s) {
+      const unsigned long long k = cluster.map_shared_rank(sm.ep_u64, s)[56];
+      if (k < bmin) { bmin = k; j = cluster.map_shared_rank(sm.ep_int, s)[1]; }
+    }
+    sm.ep_int[4] = j;
+    sm.ep_u64[57] = bmin;
+  }
+  cluster.sync();                                       // #4: nobody's shared memory is needed any more
+  if (split != 0) return;
+  bmin = sm.ep_u64[57];
+  finish_lane<T, D, G>(P, v, sm, compress, bmin, sm.ep_int[4]);
 }
 
 // Clears a context: every lane empty, chain heads/tails unset, slot 0 free.
