@@ -161,6 +161,7 @@ def main():
     ap.add_argument("--impl", default="wkv", choices=["wkv", "reference"])
     ap.add_argument("--prefill-tokens", type=int, default=0, help="0 = budget + 64")
     ap.add_argument("--n-splits", type=int, default=0)
+    ap.add_argument("--schedule", type=int, default=0, help="0 = library's choice, 1 = scan + epilogue kernels, 2 = clusters")
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling captures)")
@@ -201,7 +202,7 @@ def main():
     seed = rank_seed(BASE_SEED, rank)
     dt_code = binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16
     ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window, wl.sink,
-                          dt_code, n_splits=args.n_splits, device=dev)
+                          dt_code, n_splits=args.n_splits, device=dev, schedule=args.schedule)
     stream = TokenStream(wl, seed, dev)
     n_prefill = args.prefill_tokens if args.prefill_tokens else wl.budget + 64
     # ragged prompt lengths in the last 32 tokens of the (shortened) prefill: every cache ends up full
@@ -296,7 +297,9 @@ def main():
 
     peak, peak_kind = hbm_peak()
     bytes_launch = algorithmic_bytes_per_launch(wl)
-    launch_ms = elapsed_ms / max(1, launches // 1)
+    # one layer call = the scan kernel plus (two-kernel schedule) the lane-epilogue kernel; their bytes are the
+    # algorithmic bytes of one layer, so the fraction is taken over the whole call, not over the scan alone
+    launch_ms = elapsed_ms / (args.steps * wl.n_layers)
     achieved = bytes_launch / (launch_ms * 1e-3) / 1e9
     traffic = None      # DRAM bytes per launch from an ncu capture; see profiles/
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
@@ -312,8 +315,9 @@ def main():
             "gpu_launches": launches, "clocks": clocks,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_8000_nominal": achieved / 8000.0,
-                         "kernel": "decode_step_kernel", "algorithmic_bytes_per_launch": bytes_launch,
-                         "launch_ms": launch_ms},
+                         "kernel": "scan_kernel (+ lane_epilogue_kernel)" if launches == 2 * args.steps * wl.n_layers
+                         else "decode_step_cluster_kernel",
+                         "algorithmic_bytes_per_launch": bytes_launch, "launch_ms": launch_ms},
             "e2e": {"value": e2e_value, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": n_e2e}}
     if not args.no_cpu_baseline:

@@ -42,6 +42,12 @@ typedef enum {
   WKV_ERR_TIMEOUT = -5  /* a bounded device-side wait gave up (device status word)          */
 } wkv_error;
 
+typedef enum {
+  WKV_SCHEDULE_AUTO = 0,
+  WKV_SCHEDULE_SPLIT = 1,  /* two launches: scan every unit, then one CTA per lane finishes it (any n_splits)    */
+  WKV_SCHEDULE_CLUSTER = 2 /* one launch: a lane's units form a thread-block cluster (n_splits in {1,2,4,8,16})  */
+} wkv_schedule;
+
 /* Device memory provider.  alloc returns a device address aligned to at least 256 bytes, or NULL. */
 typedef void* (*wkv_alloc_fn)(size_t bytes, void* user);
 typedef void (*wkv_release_fn)(void* ptr, void* user);
@@ -60,7 +66,8 @@ typedef struct {
   int32_t dtype;      /* wkv_dtype: storage type of q, k, v, out and the cache                         */
   float scale;        /* softmax scale; 0 selects 1/sqrt(head_dim) (Ideal Merging section)             */
   int32_t merge;      /* 1: WeightedKV; 0: the "Eviction" variant of the Ablation Study (value dropped) */
-  int32_t n_splits;   /* CTAs that share one lane's cache scan; 0 = choose from the shape; max 64      */
+  int32_t n_splits;   /* units a lane's cache scan is cut into; 0 = choose from the shape; max 64         */
+  int32_t schedule;   /* wkv_schedule: how units are mapped to CTAs; 0 = choose from the shape            */
   void* stream;       /* cudaStream_t of the caller; NULL = the legacy default stream                  */
   wkv_alloc_fn alloc; /* NULL = cudaMalloc / cudaFree                                                  */
   wkv_release_fn release;
@@ -85,7 +92,7 @@ int wkv_reset(wkv_ctx* ctx);
 /* Changes the stream later calls are issued on.  The caller orders work across streams. */
 int wkv_set_stream(wkv_ctx* ctx, void* stream);
 
-/* One iteration of Algorithm 1 for every sequence of one layer, one kernel launch, asynchronous.
+/* One iteration of Algorithm 1 for every sequence of one layer (one or two kernel launches), asynchronous.
  *   q    device [batch, n_q_heads, head_dim]   query of the new token
  *   k, v device [batch, n_kv_heads, head_dim]  its key and value, appended to the cache first
  *                                              (Background: K_t = [K_{t-1}, k_t], V_t = [V_{t-1}, v_t])
@@ -105,21 +112,21 @@ int wkv_decode_step(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, c
  * inside a region where allocation is forbidden or would stall (a latency-critical serving loop that
  * promised its allocator a fixed footprint, a process whose memory pool has been handed over entirely to
  * another component, a plug-in that is only allowed to use buffers it is given).  wkv_decode_step already
- * allocates nothing per call, but its scratch (parked logits, per-split partial outputs, arrival counters)
- * was obtained from the memory provider at wkv_create.  This variant runs the same kernel with that
+ * allocates nothing per call, but its scratch (parked logits, per-split partial outputs) was obtained from
+ * the memory provider at wkv_create.  This variant runs the same two kernels (scan, lane epilogue) with that
  * scratch placed in a fixed array of WKV_STATIC_SCRATCH_BYTES bytes that is part of the library image, so a
  * context created through a provider that only hands out caller-owned memory never causes an allocation.
  * Every GPU that loads the library holds the array until the process exits.
  *
  *   Arguments, shapes and results: exactly those of wkv_decode_step, without `probs`.
- *   Limit: batch*n_kv_heads*(4 + group*4*roundup4(budget+1) + n_splits*group*(head_dim+2)*4) bytes (each
+ *   Limit: batch*n_kv_heads*(group*4*roundup4(budget+1) + n_splits*group*(head_dim+2)*4) bytes (each
  *          region rounded up to 256) must fit WKV_STATIC_SCRATCH_BYTES; otherwise WKV_ERR_INVALID is returned,
  *          nothing is launched, and wkv_last_error() names both numbers.
  *   First call on a device: looks up the array's device address (cudaGetSymbolAddress) with that device
  *          current and remembers it.  Make that first call outside any stream capture.
- *   Sharing: all contexts and all calls use the one array, which keeps the previous call's contents.  The
- *          arrival counters are cleared on the stream before each launch; everything else is overwritten
- *          before it is read.  Calls that can overlap on the GPU (different streams, or different contexts
+ *   Sharing: all contexts and all calls use the one array, which keeps the previous call's contents.  Nothing
+ *          in it has to start at zero: every word the second kernel reads has been written by the first
+ *          kernel of the same call.  Calls that can overlap on the GPU (different streams, or different contexts
  *          without ordering between them) race on the array: serialise them.
  *   Calls no cudaMalloc, cudaFree or other allocating routine. */
 #define WKV_STATIC_SCRATCH_BYTES (4u << 20)

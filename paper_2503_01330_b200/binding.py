@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwkv.so")
 
 WKV_F32, WKV_BF16 = 0, 1
+WKV_SCHEDULE_AUTO, WKV_SCHEDULE_SPLIT, WKV_SCHEDULE_CLUSTER = 0, 1, 2
 WKV_OK, WKV_ERR_INVALID, WKV_ERR_ALLOC, WKV_ERR_CUDA, WKV_ERR_STATE, WKV_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)
@@ -23,7 +24,7 @@ RELEASE_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_void_p)
 class wkv_config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("budget", C.c_int32), ("window", C.c_int32), ("sink", C.c_int32),
-                ("dtype", C.c_int32), ("scale", C.c_float), ("merge", C.c_int32), ("n_splits", C.c_int32),
+                ("dtype", C.c_int32), ("scale", C.c_float), ("merge", C.c_int32), ("n_splits", C.c_int32), ("schedule", C.c_int32),
                 ("stream", C.c_void_p), ("alloc", ALLOC_FN), ("release", RELEASE_FN), ("user", C.c_void_p)]
 
 
@@ -87,12 +88,13 @@ def _dp(t):
 
 
 def make_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, budget, window, sink=0, dtype=WKV_BF16, scale=0.0,
-                merge=1, n_splits=0, stream=None):
+                merge=1, n_splits=0, stream=None, schedule=0):
     cfg = wkv_config()
     cfg.n_layers, cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim = n_layers, batch, n_q_heads, n_kv_heads, head_dim
     cfg.budget, cfg.window, cfg.sink, cfg.dtype, cfg.scale, cfg.merge, cfg.n_splits = (budget, window, sink, dtype, scale,
                                                                                      merge, n_splits)
     cfg.stream = stream
+    cfg.schedule = schedule
     return cfg
 
 
@@ -105,7 +107,7 @@ class Context:
     """One wkv_ctx.  Device memory comes from torch's caching allocator through the provider callbacks."""
 
     def __init__(self, n_layers, batch, n_q_heads, n_kv_heads, head_dim, budget, window, sink=0, dtype=WKV_BF16,
-                 scale=0.0, merge=1, n_splits=0, device="cuda:0", torch_alloc=True):
+                 scale=0.0, merge=1, n_splits=0, device="cuda:0", torch_alloc=True, schedule=0):
         self.device = torch.device(device)
         self.dtype = dtype
         self.tdtype = torch.bfloat16 if dtype == WKV_BF16 else torch.float32
@@ -113,7 +115,7 @@ class Context:
         self.budget = budget
         self._bufs = {}
         cfg = make_config(n_layers, batch, n_q_heads, n_kv_heads, head_dim, budget, window, sink, dtype, scale, merge,
-                          n_splits)
+                          n_splits, schedule=schedule)
         err = wkv_config_error(cfg)
         if err is not None:
             raise WkvError(WKV_ERR_INVALID, err)

@@ -20,6 +20,7 @@ struct wkv_ctx {
   int n_splits = 1;
   int chunk_cap = 0;      // cluster kernel: logits per CTA and query head
   bool use_cluster = false;
+  int sm_count = 148;
   float scale = 0.f;
   size_t elem = 2;
   cudaStream_t stream = nullptr;
@@ -33,7 +34,6 @@ struct wkv_ctx {
   int32_t* lane_state = nullptr;
   float* logits = nullptr;
   float* part = nullptr;
-  uint32_t* ticket = nullptr;
   uint32_t* status = nullptr;
   // staging for the host-buffer entry point and for discarded prefill outputs
   void* stage_q = nullptr;
@@ -101,6 +101,7 @@ const char* check_config(const wkv_config* c) {
   if (c->merge != 0 && c->merge != 1) return "merge must be 0 or 1";
   if (c->n_splits < 0 || c->n_splits > wkv::kMaxSplits) return "n_splits must be in [0, 64]";
   if (!(c->scale >= 0.f) || std::isinf(c->scale)) return "scale must be finite and >= 0";
+  if (c->schedule < WKV_SCHEDULE_AUTO || c->schedule > WKV_SCHEDULE_CLUSTER) return "schedule must be 0 (auto), 1 (two kernels) or 2 (clusters)";
   if ((c->alloc == nullptr) != (c->release == nullptr)) return "alloc and release must both be set or both be NULL";
   if ((long long)c->batch * c->n_kv_heads * wkv::kMaxSplits > 0x7fffffffLL) return "batch * n_kv_heads too large";
   return nullptr;
@@ -113,6 +114,12 @@ int auto_splits(const wkv_config& c) {
   const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
   int s = 1;
   while (s < 16 && lanes * s < 1776 && tiles / (2 * s) >= 4) s *= 2;
+  if (c.schedule != WKV_SCHEDULE_CLUSTER && lanes * tiles >= 148 * 64) {
+    // two-kernel schedule: units of about 32 tiles balance the SMs and amortise each CTA's start-up
+    s = (tiles + 31) / 32;
+    if (s > wkv::kMaxSplits) s = wkv::kMaxSplits;
+    if (s < 1) s = 1;
+  }
   return s;
 }
 
@@ -120,18 +127,20 @@ bool is_cluster_size(int s) { return s == 1 || s == 2 || s == 4 || s == 8 || s =
 
 constexpr int kMaxDynSmem = 200 * 1024;
 
-// cluster = true: the n_splits CTAs of a lane are launched as one thread-block cluster (kernel B).
+// cluster = true: one launch, the n_splits CTAs of a lane form a thread-block cluster;
+// otherwise two launches: the scan over all units, then one CTA per lane on the finished scratch.
 template <typename T, int D, int G>
-cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, bool cluster, cudaStream_t stream) {
+cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaStream_t stream) {
   using C = wkv::Cfg<T, D, G>;
   static int attr_done[64][2] = {};            // largest dynamic shared memory size configured per device and kernel
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   const int smem = C::kFixedBytes + (cluster ? G * P.chunk_cap * 4 : 0);
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
-  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::decode_step_kernel<T, D, G>;
-  if (dev >= 0 && dev < 64 && attr_done[dev][cluster] < smem) {
+  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_kernel<T, D, G>;
+  if (attr_done[dev][cluster] < smem) {
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     if (cluster) {
@@ -140,8 +149,12 @@ cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, bool cluster, cuda
     }
     attr_done[dev][cluster] = smem;
   }
+  const int n_ctas = lanes * P.n_splits;
   if (!cluster) {
-    wkv::decode_step_kernel<T, D, G><<<n_ctas, wkv::kThreads, smem, stream>>>(P);
+    wkv::scan_kernel<T, D, G><<<n_ctas, wkv::kThreads, smem, stream>>>(P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    wkv::lane_epilogue_kernel<T, D, G><<<lanes, wkv::kEpilogueThreads, 0, stream>>>(P);
     return cudaGetLastError();
   }
   cudaLaunchConfig_t lc = {};
@@ -160,32 +173,32 @@ cudaError_t launch_step(const wkv::StepParams& P, int n_ctas, bool cluster, cuda
 }
 
 template <typename T, int D>
-cudaError_t launch_by_group(int G, const wkv::StepParams& P, int n_ctas, bool cluster, cudaStream_t s) {
+cudaError_t launch_by_group(int G, const wkv::StepParams& P, int lanes, bool cluster, cudaStream_t s) {
   switch (G) {
-    case 1: return launch_step<T, D, 1>(P, n_ctas, cluster, s);
-    case 2: return launch_step<T, D, 2>(P, n_ctas, cluster, s);
-    case 4: return launch_step<T, D, 4>(P, n_ctas, cluster, s);
-    case 8: return launch_step<T, D, 8>(P, n_ctas, cluster, s);
+    case 1: return launch_step<T, D, 1>(P, lanes, cluster, s);
+    case 2: return launch_step<T, D, 2>(P, lanes, cluster, s);
+    case 4: return launch_step<T, D, 4>(P, lanes, cluster, s);
+    case 8: return launch_step<T, D, 8>(P, lanes, cluster, s);
   }
   return cudaErrorInvalidValue;
 }
 
-// cluster = false forces kernel A (global scratch), which the static-scratch entry point needs.
+// cluster = false forces the two-kernel schedule (global scratch), which the static-scratch entry point needs.
 cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P, bool cluster) {
-  const int n_ctas = c->lanes_per_layer * c->n_splits;
+  const int n = c->lanes_per_layer;
   if (c->cfg.dtype == WKV_BF16) {
-    return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n_ctas, cluster, c->stream)
-                                  : launch_by_group<__nv_bfloat16, 64>(c->group, P, n_ctas, cluster, c->stream);
+    return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n, cluster, c->stream)
+                                  : launch_by_group<__nv_bfloat16, 64>(c->group, P, n, cluster, c->stream);
   }
-  return c->cfg.head_dim == 128 ? launch_by_group<float, 128>(c->group, P, n_ctas, cluster, c->stream)
-                                : launch_by_group<float, 64>(c->group, P, n_ctas, cluster, c->stream);
+  return c->cfg.head_dim == 128 ? launch_by_group<float, 128>(c->group, P, n, cluster, c->stream)
+                                : launch_by_group<float, 64>(c->group, P, n, cluster, c->stream);
 }
 
 wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   wkv::StepParams P;
   std::memset(&P, 0, sizeof(P));
   P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
-  P.lane_state = c->lane_state; P.logits = c->logits; P.part = c->part; P.ticket = c->ticket; P.status = c->status;
+  P.lane_state = c->lane_state; P.logits = c->logits; P.part = c->part; P.status = c->status;
   P.lane0 = layer * c->lanes_per_layer;
   P.n_kv_heads = c->cfg.n_kv_heads;
   P.cap = c->cap;
@@ -199,7 +212,7 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
 
 int run_reset(wkv_ctx* c) {
   wkv::reset_kernel<<<592, 256, 0, c->stream>>>(c->lane_state, c->pos, c->a, c->next, c->prev, c->lanes_total, c->cap,
-                                                c->ticket, c->lanes_per_layer, c->status);
+                                                c->status);
   c->launches++;
   WKV_CUDA(c, cudaGetLastError());
   return WKV_OK;
@@ -244,6 +257,7 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   c->cfg = *cfg;
   if (!c->cfg.alloc) { c->cfg.alloc = default_alloc; c->cfg.release = default_release; c->cfg.user = nullptr; }
   cudaError_t e = cudaGetDevice(&c->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
   if (e != cudaSuccess) { delete c; return WKV_ERR_CUDA; }
   c->group = cfg->n_q_heads / cfg->n_kv_heads;
   c->lanes_per_layer = cfg->batch * cfg->n_kv_heads;
@@ -254,7 +268,15 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
     c->chunk_cap = ((tiles + c->n_splits - 1) / c->n_splits) * wkv::kTileSlots;   // the largest share of an even deal
     // kernel B needs a cluster-sized split count and room for the chunk's logits next to the ring
-    c->use_cluster = is_cluster_size(c->n_splits) && c->group * c->chunk_cap * 4 <= 64 * 1024;
+    const bool can_cluster = is_cluster_size(c->n_splits) && c->group * c->chunk_cap * 4 <= 64 * 1024;
+    if (cfg->schedule == WKV_SCHEDULE_CLUSTER && !can_cluster) {
+      delete c;
+      return WKV_ERR_INVALID;
+    }
+    // few lanes: latency matters, one launch and a cluster sharing the lane's epilogue; many lanes: scan all units
+    // with short-lived CTAs, then finish the lanes in a second launch
+    c->use_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ||
+                     (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_per_layer * tiles < 148 * 64);
   }
   c->scale = cfg->scale != 0.f ? cfg->scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
   c->elem = cfg->dtype == WKV_BF16 ? 2 : 4;
@@ -273,7 +295,6 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   T(take(c, &c->lane_state, (size_t)c->lanes_total * wkv::LS_STRIDE * 4));
   T(take(c, &c->logits, (size_t)c->lanes_per_layer * G * cap * 4));
   T(take(c, &c->part, (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
-  T(take(c, &c->ticket, (size_t)c->lanes_per_layer * 4));
   T(take(c, &c->status, 256));
   T(take(c, &c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * row));
   T(take(c, &c->stage_k, (size_t)c->lanes_per_layer * row));
@@ -322,8 +343,8 @@ int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, con
   P.seq_lens = nullptr;
   P.tok_idx = 0;
   cudaError_t e = launch_any(c, P, c->use_cluster);
-  c->launches++;
-  if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch");
+  c->launches += c->use_cluster ? 1 : 2;
+  if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch");
   return WKV_OK;
 }
 
@@ -333,11 +354,10 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
   if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
   const size_t D = c->cfg.head_dim, G = c->group, lanes = c->lanes_per_layer;
-  // layout inside the static array: tickets | logits | split partials, each region 256-byte aligned
-  const size_t ticket_bytes = (lanes * 4 + 255) & ~(size_t)255;
+  // layout inside the static array: parked logits | split partials, each region 256-byte aligned
   const size_t logit_bytes = (lanes * G * (size_t)c->cap * 4 + 255) & ~(size_t)255;
   const size_t part_bytes = lanes * (size_t)c->n_splits * G * (D + 2) * 4;
-  const size_t need = ticket_bytes + logit_bytes + part_bytes;
+  const size_t need = logit_bytes + part_bytes;
   if (need > kStaticScratchBytes)
     return fail(c, WKV_ERR_INVALID,
                 "wkv_decode_step_static: this shape needs " + std::to_string(need) + " bytes of scratch, the built-in array holds " +
@@ -346,9 +366,8 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   cudaError_t e = static_scratch_base(&base);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetSymbolAddress(static scratch)");
   wkv::StepParams P = base_params(c, layer);
-  P.ticket = reinterpret_cast<uint32_t*>(base);
-  P.logits = reinterpret_cast<float*>(base + ticket_bytes);
-  P.part = reinterpret_cast<float*>(base + ticket_bytes + logit_bytes);
+  P.logits = reinterpret_cast<float*>(base);
+  P.part = reinterpret_cast<float*>(base + logit_bytes);
   P.q = q; P.k = k; P.v = v; P.out = out; P.evicted = evicted_pos; P.probs = nullptr;
   P.q_bs = (long long)c->cfg.n_q_heads * (long long)D;
   P.kv_bs = (long long)c->cfg.n_kv_heads * (long long)D;
@@ -356,11 +375,11 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   P.ev_bs = c->cfg.n_kv_heads;
   P.seq_lens = nullptr;
   P.tok_idx = 0;
-  // the array keeps whatever the previous call (of any context) left: the arrival counters must start at zero
-  WKV_CUDA(c, cudaMemsetAsync(base, 0, ticket_bytes, c->stream));
+  // The array keeps whatever the previous call (of any context) left.  Nothing in it has to start at zero: the scan
+  // kernel writes every logit and every partial of an active lane before the epilogue kernel reads them.
   e = launch_any(c, P, false);
-  c->launches++;
-  if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (static scratch)");
+  c->launches += 2;
+  if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (static scratch)");
   return WKV_OK;
 }
 
@@ -403,8 +422,8 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
     P.out = out ? (void*)((char*)out + (size_t)t * Hq * D * c->elem) : c->stage_out;
     P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
     cudaError_t e = launch_any(c, P, c->use_cluster);
-    c->launches++;
-    if (e != cudaSuccess) return cuda_fail(c, e, "decode_step_kernel launch (prefill)");
+    c->launches += c->use_cluster ? 1 : 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (prefill)");
   }
   return WKV_OK;
 }

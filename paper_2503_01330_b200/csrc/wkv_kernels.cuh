@@ -1,13 +1,19 @@
 // Device code of the WeightedKV decode step for sm_100a.
 //
 // One launch runs one iteration of the paper's Algorithm 1 for every lane (sequence, kv-head) of a layer.
-// grid = lanes * n_splits CTAs (the splits of a lane are adjacent).  The CTAs of a lane split the lane's slots into contiguous chunks; each CTA
-// streams its K and V rows through a shared-memory ring filled by bulk asynchronous copies (one elected
-// producer thread, mbarrier completion), computes the logits, an online-softmax partial of the attention
-// output, and parks the logits in scratch.  The CTA that finishes last for a lane (atomic ticket: nobody
-// waits for anybody) combines the partials into o_t, turns the logits into the probabilities A_t with the
-// reproducible binary32 arithmetic below, folds them into the accumulated scores, picks the eviction
-// victim, merges its value into the right neighbour, and relinks the slot bookkeeping.
+// A lane's slots are cut into n_splits contiguous chunks ("units").  Whoever processes a unit streams its K and V
+// rows through a shared-memory ring filled by bulk asynchronous copies (one producer thread, mbarrier completion),
+// computes the logits, and keeps an online-softmax partial of the attention output.  When all units of a lane are
+// done, the partials become o_t, the logits become the probabilities A_t (reproducible binary32 arithmetic below),
+// A_t is folded into the accumulated scores, the eviction victim is picked, its value is merged into the right
+// neighbour and the slot bookkeeping is relinked.  Two schedules share that code:
+//
+//   scan_kernel + lane_epilogue_kernel   any split count, two launches.  One short-lived CTA per unit parks logits
+//                               and its partial in global scratch; a second kernel with one CTA per lane finishes
+//                               the lanes.  Keeps HBM busiest when there are many lanes.
+//   decode_step_cluster_kernel           one launch: the n_splits CTAs of a lane form one thread-block cluster (n_splits in {1,2,4,8,16}).
+//                               Logits stay in shared memory, partials are read through distributed shared memory
+//                               and every CTA folds its own slots.  Best when there are few lanes (latency-bound).
 //
 // Slots are not kept in position order.  A lane owns budget+1 slots; each holds one cache entry
 // (K row, V row, accumulated score a, original position pos) and is chained to its position neighbours
@@ -58,7 +64,6 @@ struct StepParams {
   int32_t* lane_state;   // [lanes_total][LS_STRIDE]
   float* logits;         // scratch [lanes_per_layer*G][cap]
   float* part;           // scratch [lanes_per_layer][n_splits][G][D+2] : m, l, o[D]
-  uint32_t* ticket;      // scratch [lanes_per_layer], zero between launches
   uint32_t* status;      // device status word
   const void* q;         // [B][..][Hq][D]   batch stride q_bs elements
   const void* k;         // [B][..][Hkv][D]  batch stride kv_bs elements
@@ -124,6 +129,12 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 // Hint: bring [src, src + bytes) into L2.  src 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+// Barrier among the first NT threads of the CTA (NT = kThreads: the whole CTA).
+template <int NT>
+__device__ __forceinline__ void group_sync() {
+  if constexpr (NT == kThreads) __syncthreads();
+  else asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
 }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -201,6 +212,27 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long x)
   return x;
 }
 
+// Scalars and reduction scratch of a lane's epilogue (shared memory, 8-byte aligned base).
+struct EpScratch {
+  float* w;                  // [G][kMaxSplits] split weights of the output combination
+  float* M;                  // [8] global max logit per query head
+  float* linv;               // [8]
+  float* Z;                  // [8]
+  float* misc;               // [8] w_j, w_r
+  int* i32;                  // [64] flags, j, r
+  unsigned long long* u64;   // [128]: [0..63] sums, [64..71] minima, [80..87] Z partial per head, [88..89] pick key
+  __host__ __device__ static constexpr int bytes(int G) { return (G * kMaxSplits + 32 + 64) * 4 + 128 * 8; }
+  __device__ __forceinline__ void carve(unsigned char* base, int G) {
+    w = reinterpret_cast<float*>(base);
+    M = w + G * kMaxSplits;
+    linv = M + 8;
+    Z = linv + 8;
+    misc = Z + 8;
+    i32 = reinterpret_cast<int*>(misc + 8);
+    u64 = reinterpret_cast<unsigned long long*>(i32 + 64);
+  }
+};
+
 // ------------------------------------------------------------------------------------------------
 // compile-time shape of one instantiation and its shared-memory carve-up
 // ------------------------------------------------------------------------------------------------
@@ -212,187 +244,114 @@ struct Cfg {
   static constexpr int kFit = WKV_RING_BYTES / (2 * kTileBytes);
   static constexpr int kStages = kFit < 2 ? 2 : (kFit > 8 ? 8 : kFit);
   static constexpr int kRingBytes = kStages * 2 * kTileBytes;
+  static constexpr int kAuxBytes = 2 * kRowBytes;           // k row and v row of the new token
   static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
   static constexpr int kCtaPartFloats = G * (D + 2);
-  // ring | warp partials | CTA partial | new k, v rows | mbarriers | epilogue scalars | (cluster kernel: chunk logits)
-  static constexpr int kFixedBytes = kRingBytes + (kWarpPartFloats + kCtaPartFloats) * 4 + 2 * kRowBytes + 2 * kStages * 8 +
-                                     (G * kMaxSplits + 32 + 64) * 4 + 64 * 8 + 128;
+  // ring | new token rows | warp partials | CTA partial | mbarriers | epilogue scalars | (cluster: chunk logits)
+  static constexpr int kFixedBytes = kRingBytes + kAuxBytes + (kWarpPartFloats + kCtaPartFloats) * 4 + 2 * kStages * 8 +
+                                     EpScratch::bytes(G) + 128;
 };
 
 template <typename T, int D, int G>
 struct Smem {
   unsigned char* ring;       // [stage][K tile | V tile]
+  T* aux;                    // [ k: D | v: D ] this step's token
   float* warp_part;          // [warp][G][D+2] : m, l, o[D]
   float* cta_part;           // [G][D+2]
-  T* new_k;                  // [D]
-  T* new_v;                  // [D]
   uint64_t* full_bar;        // [kStages]
   uint64_t* empty_bar;       // [kStages]
-  float* ep_w;               // [G][kMaxSplits] split weights of the output combination
-  float* ep_M;               // [8] global max logit per query head
-  float* ep_linv;            // [8]
-  float* ep_Z;               // [8]
-  float* ep_misc;            // [8] w_j, w_r
-  int* ep_int;               // [64] flags, j, r
-  unsigned long long* ep_u64;// [64] reduction scratch; [48..55] Z partial per head, [56] pick key of this CTA
+  EpScratch ep;              // epilogue scalars and reduction scratch
   float* chunk_logits;       // [G][chunk_cap] (cluster kernel only)
   __device__ __forceinline__ explicit Smem(unsigned char* raw) {
     using C = Cfg<T, D, G>;
     ring = raw;
-    warp_part = reinterpret_cast<float*>(ring + C::kRingBytes);
+    aux = reinterpret_cast<T*>(ring + C::kRingBytes);
+    warp_part = reinterpret_cast<float*>(ring + C::kRingBytes + C::kAuxBytes);
     cta_part = warp_part + C::kWarpPartFloats;
-    new_k = reinterpret_cast<T*>(cta_part + C::kCtaPartFloats);
-    new_v = new_k + D;
-    full_bar = reinterpret_cast<uint64_t*>(new_v + D);
+    full_bar = reinterpret_cast<uint64_t*>(cta_part + C::kCtaPartFloats);
     empty_bar = full_bar + C::kStages;
-    ep_w = reinterpret_cast<float*>(empty_bar + C::kStages);
-    ep_M = ep_w + G * kMaxSplits;
-    ep_linv = ep_M + 8;
-    ep_Z = ep_linv + 8;
-    ep_misc = ep_Z + 8;
-    ep_int = reinterpret_cast<int*>(ep_misc + 8);
-    ep_u64 = reinterpret_cast<unsigned long long*>(ep_int + 64);
-    chunk_logits = reinterpret_cast<float*>(ep_u64 + 64);
+    ep.carve(reinterpret_cast<unsigned char*>(empty_bar + C::kStages), G);
+    chunk_logits = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(empty_bar + C::kStages) + EpScratch::bytes(G));
   }
+  __device__ __forceinline__ T* aux_k(int) const { return aux; }
+  __device__ __forceinline__ T* aux_v(int) const { return aux + D; }
 };
 
-// What a CTA knows about its lane and its share of the lane's slots.
+// What the threads working on a unit know about its lane and its share of the lane's slots.
 template <typename T>
 struct LaneView {
   long long lane;            // global lane index
   int lane_local, b, hk, split;
   int len, t, new_slot, L;   // L = entries attended this step (new token included)
-  int tile_begin, n_tiles;   // this CTA's tiles
-  int slot_begin, slot_end;  // this CTA's slots [slot_begin, slot_end) clipped to L
-  const T *Kl, *Vl, *q_in, *k_in, *v_in;
-  int* st;
-  bool active;
+  int tile_begin, n_tiles;   // this unit's tiles
+  int slot_begin, slot_end;  // this unit's slots [slot_begin, slot_end) clipped to L
+  const T *Kl, *Vl;          // the lane's cache rows
+  const T *new_k, *new_v;    // this step's token (shared memory)
+  int* st;                   // the lane's state words
 };
 
-template <typename T, int D, int G>
-__device__ __forceinline__ LaneView<T> open_lane(const StepParams& P, const Smem<T, D, G>& sm, int lane_local, int split) {
-  using C = Cfg<T, D, G>;
-  LaneView<T> v;
-  const int tid = threadIdx.x;
+// Lane-level part of a view: addresses and the even deal of tiles (the first tiles_total % n_splits units get one more).
+template <typename T, int D>
+__device__ __forceinline__ void fill_view(LaneView<T>& v, const StepParams& P, int lane_local, int split, int len, int t,
+                                          int new_slot) {
   v.lane_local = lane_local;
   v.split = split;
   v.b = lane_local / P.n_kv_heads;
   v.hk = lane_local % P.n_kv_heads;
-  v.active = !(P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[v.b]);   // sequence already consumed (ragged prefill)
-  if (!v.active) {
-    if (split == 0 && tid == 0 && P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = -1;
-    return v;
-  }
   v.lane = (long long)P.lane0 + lane_local;
   v.st = P.lane_state + v.lane * LS_STRIDE;
-  v.len = v.st[LS_LEN];
-  v.t = v.st[LS_T];
-  v.new_slot = v.st[LS_FREE];
-  v.L = v.len + 1;
+  v.len = len;
+  v.t = t;
+  v.new_slot = new_slot;
+  v.L = len + 1;
   v.Kl = reinterpret_cast<const T*>(P.Kc) + v.lane * (long long)P.cap * D;
   v.Vl = reinterpret_cast<const T*>(P.Vc) + v.lane * (long long)P.cap * D;
-  v.q_in = reinterpret_cast<const T*>(P.q) + v.b * P.q_bs + (long long)v.hk * G * D;
-  v.k_in = reinterpret_cast<const T*>(P.k) + v.b * P.kv_bs + (long long)v.hk * D;
-  v.v_in = reinterpret_cast<const T*>(P.v) + v.b * P.kv_bs + (long long)v.hk * D;
-  // tiles are dealt out evenly: the first (tiles_total mod n_splits) CTAs take one more
   const int tiles_total = (v.L + kTileSlots - 1) / kTileSlots;
   const int base = tiles_total / P.n_splits, extra = tiles_total % P.n_splits;
   v.tile_begin = split * base + min(split, extra);
   v.n_tiles = base + (split < extra ? 1 : 0);
   v.slot_begin = min(v.L, v.tile_begin * kTileSlots);
   v.slot_end = min(v.L, (v.tile_begin + v.n_tiles) * kTileSlots);
-
-  if (tid == 32 && v.slot_end > v.slot_begin) {
-    // The epilogue reads a and pos of these slots long after the scan: pull their lines into L2 now.
-    const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);   // cap is a multiple of 4 slots
-    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
-    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
-  }
-  if (tid == 0) {
-    for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(&sm.full_bar[s], 1);
-      mbar_init(&sm.empty_bar[s], kConsumerWarps);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in
-  // flight) and written to the cache by the CTA whose chunk owns the slot.
-  for (int c = tid; c < D; c += kThreads) {
-    sm.new_k[c] = v.k_in[c];
-    sm.new_v[c] = v.v_in[c];
-  }
-  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
-    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
-    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
-    for (int c = tid; c < D; c += kThreads) {
-      Kw[c] = v.k_in[c];
-      Vw[c] = v.v_in[c];
-    }
-  }
-  __syncthreads();
-  return v;
 }
 
 // ------------------------------------------------------------------------------------------------
-// the scan: logits, online-softmax partial of o, logits parked at logit_dst[g*logit_stride + slot - logit_off]
+// the scan: per-thread state of the four consumer warps (each warp owns 8 rows of every tile)
 // ------------------------------------------------------------------------------------------------
+// A row (one cache entry) is shared by LPR threads.  Thread l of the group owns the partial sums {l, l+LPR, ...} of
+// the reproducible dot, each a block of D/16 contiguous channels, so butterfly rounds with off >= LPR are additions
+// inside the thread and only log2(LPR) shuffles remain.
 template <typename T, int D, int G>
-__device__ __forceinline__ void scan_tiles(const StepParams& P, const Smem<T, D, G>& sm, const LaneView<T>& v,
-                                           float* logit_dst, long long logit_stride, int logit_off) {
+struct Scanner {
   using C = Cfg<T, D, G>;
-  constexpr int kStages = C::kStages;
-  const float kLog2e = 1.4426950408889634f;
-  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
-  const int L = v.L, new_slot = v.new_slot;
-
-  if (warp == kConsumerWarps) {
-    // ---------------- producer: one thread keeps the ring full ----------------
-    if (lane_id == 0) {
-      for (int i = 0; i < v.n_tiles; ++i) {
-        const int s = i % kStages;
-        if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
-        const int slot0 = (v.tile_begin + i) * kTileSlots;
-        const uint32_t bytes = (uint32_t)min(kTileSlots, L - slot0) * C::kRowBytes;
-        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
-        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
-        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
-        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
-      }
-    }
-    return;
-  }
-  // ---------------- consumers: 4 warps, each owns 8 rows of every tile ----------------
-  // A row (one cache entry) is shared by LPR threads.  Thread l of the group owns the partial sums
-  // {l, l+LPR, ...} of the reproducible dot, each a block of D/16 contiguous channels, so butterfly rounds
-  // with off >= LPR are additions inside the thread and only log2(LPR) shuffles remain.
-  constexpr int LPR = C::kLanesPerRow;           // 8 or 16 threads per row
-  constexpr int NP = 16 / LPR;                   // partial sums per thread
-  constexpr int CH = D / 16;                     // channels per partial sum
-  constexpr int RPP = 32 / LPR;                  // rows per warp pass
-  constexpr int PASSES = 8 / RPP;
-  const int rg = lane_id / LPR, l = lane_id % LPR;
+  static constexpr int LPR = C::kLanesPerRow;    // 8 or 16 threads per row
+  static constexpr int NP = 16 / LPR;            // partial sums per thread
+  static constexpr int CH = D / 16;              // channels per partial sum
+  static constexpr int RPP = 32 / LPR;           // rows per warp pass
+  static constexpr int PASSES = 8 / RPP;
   float qf[G][NP][CH];
-#pragma unroll
-  for (int g = 0; g < G; ++g)
-#pragma unroll
-    for (int j = 0; j < NP; ++j) load_chunk<CH>(v.q_in + g * D + (l + LPR * j) * CH, qf[g][j]);
   float m_run[G], l_run[G], o_acc[G][NP][CH];
+
+  __device__ __forceinline__ void begin(const T* q) {      // q: [G][D], 16-byte aligned (global or shared)
+    const int l = (threadIdx.x & 31) % LPR;
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
-    m_run[g] = -INFINITY;
-    l_run[g] = 0.f;
+    for (int g = 0; g < G; ++g) {
 #pragma unroll
-    for (int j = 0; j < NP; ++j)
+      for (int j = 0; j < NP; ++j) load_chunk<CH>(q + g * D + (l + LPR * j) * CH, qf[g][j]);
+      m_run[g] = -INFINITY;
+      l_run[g] = 0.f;
 #pragma unroll
-      for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
+      for (int j = 0; j < NP; ++j)
+#pragma unroll
+        for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
+    }
   }
 
-  for (int i = 0; i < v.n_tiles; ++i) {
-    const int s = i % kStages;
-    mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
-    T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
-    T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
-    const int slot0 = (v.tile_begin + i) * kTileSlots;
+  // One tile of up to 32 rows starting at slot0; logits parked at logit_dst[g*logit_stride + slot - logit_off].
+  __device__ __forceinline__ void tile(T* tK, T* tV, int slot0, int L, int new_slot, const T* new_k, const T* new_v,
+                                       float scale, float* logit_dst, long long logit_stride, int logit_off) {
+    const float kLog2e = 1.4426950408889634f;
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
     {
       // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
       // row in the tile with the token's k and v before anybody reads it.
@@ -400,14 +359,13 @@ __device__ __forceinline__ void scan_tiles(const StepParams& P, const Smem<T, D,
       if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
         uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
         uint32_t* dv = reinterpret_cast<uint32_t*>(tV + ns_row * D);
-        const uint32_t* sk = reinterpret_cast<const uint32_t*>(sm.new_k);
-        const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(sm.new_v);
+        const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
+        const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
         for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; dv[w] = sv_[w]; }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
         __syncwarp();
       }
     }
-
     float sv[G][PASSES];
     bool valid[PASSES];
 #pragma unroll
@@ -431,7 +389,7 @@ __device__ __forceinline__ void scan_tiles(const StepParams& P, const Smem<T, D,
         if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
 #pragma unroll
         for (int off = LPR / 2; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-        const float sc = __fmul_rn(P.scale, acc);
+        const float sc = __fmul_rn(scale, acc);
         sv[g][ps] = valid[ps] ? sc : -INFINITY;
       }
     }
@@ -479,46 +437,49 @@ __device__ __forceinline__ void scan_tiles(const StepParams& P, const Smem<T, D,
         }
       }
     }
-    __syncwarp();
-    if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
   }
 
-  // fold the row groups of the warp, then leave the warp's partial in shared memory
+  // Fold the warp's row groups and leave the warp's partial (m, l, o[D]) per query head in shared memory.
+  __device__ __forceinline__ void end(float* warp_part) {
+    const float kLog2e = 1.4426950408889634f;
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
 #pragma unroll
-  for (int g = 0; g < G; ++g) {
+    for (int g = 0; g < G; ++g) {
 #pragma unroll
-    for (int off = 16; off >= LPR; off >>= 1) {
-      const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
-      const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
-      const float m_new = fmaxf(m_run[g], m_o);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
-      l_run[g] = l_run[g] * c_me + l_o * c_o;
-      m_run[g] = m_new;
+      for (int off = 16; off >= LPR; off >>= 1) {
+        const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
+        const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
+        const float m_new = fmaxf(m_run[g], m_o);
+        const float m_use = m_new == -INFINITY ? 0.f : m_new;
+        const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
+        l_run[g] = l_run[g] * c_me + l_o * c_o;
+        m_run[g] = m_new;
 #pragma unroll
-      for (int j = 0; j < NP; ++j)
+        for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CH; ++e) {
-          const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
-          o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
-        }
+          for (int e = 0; e < CH; ++e) {
+            const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
+            o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
+          }
+      }
+      float* wp = warp_part + (warp * G + g) * (D + 2);
+      if (rg == 0) {
+#pragma unroll
+        for (int j = 0; j < NP; ++j)
+#pragma unroll
+          for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
+      }
+      if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
     }
-    float* wp = sm.warp_part + (warp * G + g) * (D + 2);
-    if (rg == 0) {
-#pragma unroll
-      for (int j = 0; j < NP; ++j)
-#pragma unroll
-        for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
-    }
-    if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
   }
-}
+};
 
-// The four warp partials -> one (m, l, o[D]) per query head at dst (shared or global).  Call after __syncthreads().
-template <int D, int G>
+// The four warp partials -> one (m, l, o[D]) per query head at dst (shared or global).  Call after the group's barrier.
+template <int D, int G, int NT>
 __device__ __forceinline__ void combine_warps(const float* warp_part, float* dst) {
   const float kLog2e = 1.4426950408889634f;
-  for (int idx = threadIdx.x; idx < G * D; idx += kThreads) {
+  for (int idx = threadIdx.x; idx < G * D; idx += NT) {
     const int g = idx / D, c = idx % D;
     float mx = -INFINITY;
 #pragma unroll
@@ -538,20 +499,20 @@ __device__ __forceinline__ void combine_warps(const float* warp_part, float* dst
 }
 
 // ------------------------------------------------------------------------------------------------
-// epilogue pieces (reproducible arithmetic)
+// epilogue pieces (reproducible arithmetic), run by the first NT threads of a CTA
 // ------------------------------------------------------------------------------------------------
 // e_i = exp(s_i - M_g), written back in place of the logit, and this thread's share of sum_i trunc(e_i * 2^40).
 // Element i of the range lives at lg[g*stride + i]; kL2 selects loads that bypass L1 (logits written by other SMs).
-template <int G, bool kL2>
+template <int G, bool kL2, int NT>
 __device__ __forceinline__ void exp_and_zsum(float* lg, long long stride, int n, const float* M, unsigned long long (&zl)[G]) {
   constexpr int U = 4;                          // loads of U elements are issued before any of them is used
 #pragma unroll
   for (int g = 0; g < G; ++g) zl[g] = 0ull;
-  for (int i0 = threadIdx.x; i0 < n; i0 += kThreads * U) {
+  for (int i0 = threadIdx.x; i0 < n; i0 += NT * U) {
     float sx[G][U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * kThreads;
+      const int i = i0 + u * NT;
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         const float* p = lg + (long long)g * stride + i;
@@ -560,7 +521,7 @@ __device__ __forceinline__ void exp_and_zsum(float* lg, long long stride, int n,
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * kThreads;
+      const int i = i0 + u * NT;
       if (i < n) {
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -573,29 +534,29 @@ __device__ __forceinline__ void exp_and_zsum(float* lg, long long stride, int n,
   }
 }
 
-// Block-wide sums of G 64-bit integers; result[g] valid in every thread after the call.  scratch: 8*G + ... entries.
-template <int G>
-__device__ __forceinline__ void block_sum_u64(unsigned long long (&x)[G], unsigned long long* scratch) {
+// Group-wide sums of G 64-bit integers; x[g] holds the total in every thread after the call.  scratch: G*NT/32 entries.
+template <int G, int NT>
+__device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsigned long long* scratch) {
   const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     const unsigned long long w = warp_sum_u64(x[g]);
-    if (lane_id == 0) scratch[g * 5 + warp] = w;
+    if (lane_id == 0) scratch[g * (NT / 32) + warp] = w;
   }
-  __syncthreads();
+  group_sync<NT>();
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     unsigned long long z = 0ull;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) z += scratch[g * 5 + w];
+    for (int w = 0; w < NT / 32; ++w) z += scratch[g * (NT / 32) + w];
     x[g] = z;
   }
-  __syncthreads();
+  group_sync<NT>();
 }
 
 // A_t over a range of slots, a = [a,0] + A_t, abar = a/n and the range's pick key (Algorithm 1).
-// e values at lg[g*stride + i] for slot slot0 + i.  Returns the thread's best (key, slot).
-template <typename T, int G>
+// e values at lg[g*stride + i] for slot slot0 + i.  Updates the thread's best (key, slot).
+template <typename T, int G, int NT>
 __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<T>& v, const float* lg, long long stride,
                                             int slot0, int n, const float* Z, bool compress, unsigned long long& best,
                                             int& best_slot) {
@@ -603,12 +564,12 @@ __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<
   int32_t* pos_l = P.pos + v.lane * P.cap;
   const int t = v.t;
   constexpr int U = 4;                          // a, pos and e of U slots are loaded before any of them is used
-  for (int i0 = threadIdx.x; i0 < n; i0 += kThreads * U) {
+  for (int i0 = threadIdx.x; i0 < n; i0 += NT * U) {
     float a_old[U], ev[G][U];
     int pos_v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * kThreads;
+      const int i = i0 + u * NT;
       const int slot = slot0 + i;
       const bool ok = i < n, is_new = slot == v.new_slot;
       a_old[u] = (ok && !is_new) ? a_l[slot] : 0.f;
@@ -618,7 +579,7 @@ __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const int i = i0 + u * kThreads;
+      const int i = i0 + u * NT;
       if (i >= n) continue;
       const int slot = slot0 + i;
       float pg[G];
@@ -645,26 +606,27 @@ __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<
   }
 }
 
-// Block-wide minimum of the pick key; returns it in every thread and leaves the owning slot in *slot_out (shared).
-__device__ __forceinline__ unsigned long long block_min_key(unsigned long long best, int best_slot, unsigned long long* scratch,
+// Group-wide minimum of the pick key; returns it in every thread and leaves the owning slot in *slot_out (shared).
+template <int NT>
+__device__ __forceinline__ unsigned long long group_min_key(unsigned long long best, int best_slot, unsigned long long* scratch,
                                                             int* slot_out) {
   const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
   const unsigned long long wmin = warp_min_u64(best);
   if (lane_id == 0) scratch[warp] = wmin;
   if (threadIdx.x == 0) *slot_out = -1;
-  __syncthreads();
+  group_sync<NT>();
   unsigned long long bmin = scratch[0];
 #pragma unroll
-  for (int w = 1; w < kThreads / 32; ++w) bmin = scratch[w] < bmin ? scratch[w] : bmin;
+  for (int w = 1; w < NT / 32; ++w) bmin = scratch[w] < bmin ? scratch[w] : bmin;
   if (best == bmin && best_slot >= 0) *slot_out = best_slot;       // positions are unique: one owner
-  __syncthreads();
+  group_sync<NT>();
   return bmin;
 }
 
 // Link the new entry as the chain's tail, unlink the victim j (Algorithm 1: remove K[j], a[j], n[j]; the right
-// neighbour keeps its own key, a and n), merge V[j] into V[next[j]], update the lane state.  One CTA per lane runs it.
-template <typename T, int D, int G>
-__device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const Smem<T, D, G>& sm, bool compress,
+// neighbour keeps its own key, a and n), merge V[j] into V[next[j]], update the lane state.  One group per lane runs it.
+template <typename T, int D, int G, int NT>
+__device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const EpScratch& ep, bool compress,
                                             unsigned long long bmin, int j_slot) {
   const int tid = threadIdx.x;
   const int t = v.t, new_slot = v.new_slot, L = v.L;
@@ -679,7 +641,7 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     if (tail >= 0) next_l[tail] = new_slot; else head = new_slot;
     tail = new_slot;
     int ev_pos = -1, new_len = L, new_free = L;          // while growing, slots fill in arrival order
-    sm.ep_int[2] = -1;
+    ep.i32[2] = -1;
     if (compress) {
       const int j = j_slot;
       const int r = j >= 0 ? next_l[j] : -1;
@@ -692,10 +654,10 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
         const float Dn = __fadd_rn(abar_j, abar_r);
         float wj = 0.5f, wr = 0.5f;
         if (Dn != 0.f) { wj = __fdiv_rn(abar_j, Dn); wr = __fdiv_rn(abar_r, Dn); }
-        sm.ep_misc[0] = wj;
-        sm.ep_misc[1] = wr;
-        sm.ep_int[2] = j;
-        sm.ep_int[3] = r;
+        ep.misc[0] = wj;
+        ep.misc[1] = wr;
+        ep.i32[2] = j;
+        ep.i32[3] = r;
         ev_pos = (int)(uint32_t)(bmin & 0xffffffffull);
         const int pv = prev_l[j];
         if (pv >= 0) next_l[pv] = r; else head = r;
@@ -712,133 +674,281 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     v.st[LS_FREE] = new_free;
     if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = ev_pos;
   }
-  __syncthreads();
+  group_sync<NT>();
   // V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r), stored in T
-  if (compress && P.merge && sm.ep_int[2] >= 0) {
-    const int j = sm.ep_int[2], r = sm.ep_int[3];
-    const float wj = sm.ep_misc[0], wr = sm.ep_misc[1];
+  if (compress && P.merge && ep.i32[2] >= 0) {
+    const int j = ep.i32[2], r = ep.i32[3];
+    const float wj = ep.misc[0], wr = ep.misc[1];
     T* Vw = const_cast<T*>(v.Vl);
-    for (int c = tid; c < D; c += kThreads) {
-      // the row of this step's token may have been written to the cache by another CTA: take it from shared memory
-      const float vj = to_f32(j == new_slot ? sm.new_v[c] : __ldcg(Vw + (long long)j * D + c));
-      const float vr = to_f32(r == new_slot ? sm.new_v[c] : __ldcg(Vw + (long long)r * D + c));
+    for (int c = tid; c < D; c += NT) {
+      // the row of this step's token may have been written to the cache by other threads: take it from shared memory
+      const float vj = to_f32(j == new_slot ? v.new_v[c] : __ldcg(Vw + (long long)j * D + c));
+      const float vr = to_f32(r == new_slot ? v.new_v[c] : __ldcg(Vw + (long long)r * D + c));
       Vw[(long long)r * D + c] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
     }
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// Kernel A: any split count.  Partials and logits go through global scratch; the CTA that arrives last for a
-// lane (atomic ticket -- nobody waits) runs the whole epilogue.
-// ------------------------------------------------------------------------------------------------
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads) decode_step_kernel(const StepParams P) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  const Smem<T, D, G> sm(smem_raw);
+// The whole epilogue of a lane from global scratch (all partials and logits of the lane are visible to the caller).
+template <typename T, int D, int G, int NT>
+__device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
   const float kLog2e = 1.4426950408889634f;
   const int tid = threadIdx.x;
-  const int split = blockIdx.x % P.n_splits;
-  const int lane_local = blockIdx.x / P.n_splits;
-  const LaneView<T> v = open_lane<T, D, G>(P, sm, lane_local, split);
-  if (!v.active) return;
   const int L = v.L;
-  float* lg = P.logits + (long long)lane_local * G * P.cap;
-
-  scan_tiles<T, D, G>(P, sm, v, lg, P.cap, 0);
-  __syncthreads();
-  combine_warps<D, G>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
-  __syncthreads();
-  if (tid == 0) {
-    // release: the barrier ordered every thread's partials and logits before this fence (cumulativity)
-    __threadfence();
-    const uint32_t prev = atomicAdd(&P.ticket[lane_local], 1u);
-    __threadfence();   // acquire side for the CTA that turns out to be the last
-    sm.ep_int[0] = (prev == (uint32_t)P.n_splits - 1) ? 1 : 0;
-    if (sm.ep_int[0]) P.ticket[lane_local] = 0u;          // ready for the next launch
-  }
-  __syncthreads();
-  if (!sm.ep_int[0]) return;
-
-  // ---- epilogue, run by the last CTA of the lane ----
+  float* lg = P.logits + (long long)v.lane_local * G * P.cap;
+  const float* part = P.part + (long long)v.lane_local * P.n_splits * G * (D + 2);
   // (1) split weights and the global max / normaliser of every query head
   if (tid < G) {
     const int g = tid;
-    const float* pg = P.part + (long long)lane_local * P.n_splits * G * (D + 2) + g * (D + 2);
+    const float* pg = part + g * (D + 2);
     float M = -INFINITY;
     for (int s = 0; s < P.n_splits; ++s) M = fmaxf(M, __ldcg(pg + (long long)s * G * (D + 2)));
     float lsum = 0.f;
     for (int s = 0; s < P.n_splits; ++s) {
       const float w = fast_exp2((__ldcg(pg + (long long)s * G * (D + 2)) - M) * kLog2e);
-      sm.ep_w[g * kMaxSplits + s] = w;
+      ep.w[g * kMaxSplits + s] = w;
       lsum += w * __ldcg(pg + (long long)s * G * (D + 2) + 1);
     }
-    sm.ep_M[g] = M;                    // max of the reproducible logits: exact, order-free
-    sm.ep_linv[g] = 1.f / lsum;
+    ep.M[g] = M;                    // max of the reproducible logits: exact, order-free
+    ep.linv[g] = 1.f / lsum;
   }
-  __syncthreads();
+  group_sync<NT>();
   // (2) o_t = A_t^T V_t (Background section), V as it was before this step's merge
   {
     T* out = reinterpret_cast<T*>(P.out) + v.b * P.out_bs + (long long)v.hk * G * D;
-    for (int idx = tid; idx < G * D; idx += kThreads) {
+    for (int idx = tid; idx < G * D; idx += NT) {
       const int g = idx / D, c = idx % D;
-      const float* pg = P.part + (long long)lane_local * P.n_splits * G * (D + 2) + g * (D + 2) + 2 + c;
+      const float* pg = part + g * (D + 2) + 2 + c;
       float o = 0.f;
-      for (int s = 0; s < P.n_splits; ++s) o += sm.ep_w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
-      out[idx] = from_f32<T>(o * sm.ep_linv[g]);
+      for (int s = 0; s < P.n_splits; ++s) o += ep.w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
+      out[idx] = from_f32<T>(o * ep.linv[g]);
     }
   }
   // (3) Z_g as an exact integer sum
   {
     unsigned long long zl[G];
-    exp_and_zsum<G, true>(lg, P.cap, L, sm.ep_M, zl);
-    block_sum_u64<G>(zl, sm.ep_u64);
+    exp_and_zsum<G, true, NT>(lg, P.cap, L, ep.M, zl);
+    group_sum_u64<G, NT>(zl, ep.u64);
     if (tid < G) {
 #pragma unroll
       for (int g = 0; g < G; ++g)
-        if (g == tid) sm.ep_Z[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
+        if (g == tid) ep.Z[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
     }
-    __syncthreads();
+    group_sync<NT>();
   }
   // (4) probabilities, score fold, pick
   const bool compress = L > P.budget;                 // "length of V_t exceeds m"
   unsigned long long best = ~0ull;
   int best_slot = -1;
-  fold_scores<T, G>(P, v, lg, P.cap, 0, L, sm.ep_Z, compress, best, best_slot);
+  fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, ep.Z, compress, best, best_slot);
   if (P.probs) {
-    for (int i = L + tid; i < P.budget + 1; i += kThreads)
+    for (int i = L + tid; i < P.budget + 1; i += NT)
 #pragma unroll
       for (int g = 0; g < G; ++g)
         P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
   }
-  const unsigned long long bmin = block_min_key(best, best_slot, sm.ep_u64 + 40, &sm.ep_int[1]);   // also publishes a, pos
+  const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, &ep.i32[1]);   // also publishes a, pos
   // (5), (6)
-  finish_lane<T, D, G>(P, v, sm, compress, bmin, sm.ep_int[1]);
+  finish_lane<T, D, G, NT>(P, v, ep, compress, bmin, ep.i32[1]);
 }
 
 // ------------------------------------------------------------------------------------------------
-// Kernel B: the n_splits CTAs of a lane form one thread-block cluster (n_splits in {1,2,4,8,16}).  Logits stay in
-// each CTA's shared memory, partials are read through distributed shared memory, and every CTA folds its own
-// slots, so the epilogue runs on all the cluster's threads.  Cluster barriers are hardware barriers among
+// Kernels A1 + A2: any split count, two launches.  A1 scans: one CTA per unit, logits and partials to global
+// scratch, nothing else -- its CTAs are short-lived and all alike, which keeps HBM busy.  A2 runs one CTA per lane
+// on the finished scratch: o_t, probabilities, score fold, pick, merge, relink.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
+  using C = Cfg<T, D, G>;
+  constexpr int kStages = C::kStages;
+  constexpr int NT = kThreads;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const Smem<T, D, G> sm(smem_raw);
+  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
+  const int split = blockIdx.x % P.n_splits;
+  const int lane_local = blockIdx.x / P.n_splits;
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) return;      // sequence already consumed (ragged prefill)
+  LaneView<T> v;
+  {
+    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+    fill_view<T, D>(v, P, lane_local, split, st[LS_LEN], st[LS_T], st[LS_FREE]);
+  }
+  v.new_k = sm.aux_k(0);
+  v.new_v = sm.aux_v(0);
+  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
+  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+  if (tid == 32 && v.slot_end > v.slot_begin) {
+    // The epilogue kernel reads a and pos of these slots: pull their lines into L2 now.
+    const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);   // cap is a multiple of 4 slots
+    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
+    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.full_bar[s], 1);
+      mbar_init(&sm.empty_bar[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in flight)
+  // and written to the cache by the CTA whose chunk owns the slot.
+  for (int c = tid; c < D; c += NT) {
+    sm.aux_k(0)[c] = k_in[c];
+    sm.aux_v(0)[c] = v_in[c];
+  }
+  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
+    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
+    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
+    for (int c = tid; c < D; c += NT) { Kw[c] = k_in[c]; Vw[c] = v_in[c]; }
+  }
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    if (lane_id == 0) {                                   // producer: keeps the ring full
+      for (int i = 0; i < v.n_tiles; ++i) {
+        const int s = i % kStages;
+        if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
+        const int slot0 = (v.tile_begin + i) * kTileSlots;
+        const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
+        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
+        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
+        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+      }
+    }
+  } else {
+    Scanner<T, D, G> sc;
+    sc.begin(q_in);
+    float* lg = P.logits + (long long)lane_local * G * P.cap;
+    for (int i = 0; i < v.n_tiles; ++i) {
+      const int s = i % kStages;
+      mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
+      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
+      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, lg, P.cap, 0);
+      __syncwarp();
+      if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
+    }
+    sc.end(sm.warp_part);
+  }
+  __syncthreads();
+  combine_warps<D, G, NT>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
+}
+
+constexpr int kEpilogueThreads = 256;
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kEpilogueThreads) lane_epilogue_kernel(const StepParams P) {
+  __shared__ __align__(16) unsigned char ep_raw[EpScratch::bytes(G)];
+  EpScratch ep;
+  ep.carve(ep_raw, G);
+  const int lane_local = blockIdx.x;
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed (ragged prefill)
+    if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
+    return;
+  }
+  LaneView<T> v;
+  const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+  fill_view<T, D>(v, P, lane_local, 0, st[LS_LEN], st[LS_T], st[LS_FREE]);
+  v.new_k = v.Kl + (long long)v.new_slot * D;            // the scan kernel has stored this step's token in the cache
+  v.new_v = v.Vl + (long long)v.new_slot * D;
+  lane_epilogue_from_scratch<T, D, G, kEpilogueThreads>(P, v, ep);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Kernel B: the n_splits CTAs of a lane form one thread-block cluster.  Cluster barriers are hardware barriers among
 // co-scheduled CTAs; every CTA of an active lane reaches every barrier.
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const StepParams P) {
   namespace cg = cooperative_groups;
+  using C = Cfg<T, D, G>;
+  constexpr int kStages = C::kStages;
+  constexpr int NT = kThreads;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const Smem<T, D, G> sm(smem_raw);
   const float kLog2e = 1.4426950408889634f;
   cg::cluster_group cluster = cg::this_cluster();
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
   const int S = P.n_splits;
   const int split = (int)cluster.block_rank();
   const int lane_local = blockIdx.x / S;
-  const LaneView<T> v = open_lane<T, D, G>(P, sm, lane_local, split);
-  if (!v.active) return;                                // same decision in every CTA of the cluster
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed: same decision in every CTA
+    if (split == 0 && tid == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
+    return;
+  }
+  LaneView<T> v;
+  {
+    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+    fill_view<T, D>(v, P, lane_local, split, st[LS_LEN], st[LS_T], st[LS_FREE]);
+  }
+  v.new_k = sm.aux_k(0);
+  v.new_v = sm.aux_v(0);
+  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
+  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
   const int n_mine = v.slot_end - v.slot_begin;
 
-  scan_tiles<T, D, G>(P, sm, v, sm.chunk_logits, P.chunk_cap, v.slot_begin);
+  if (tid == 32 && n_mine > 0) {
+    // The epilogue reads a and pos of these slots long after the scan: pull their lines into L2 now.
+    const uint32_t bytes = (uint32_t)((n_mine * 4 + 15) & ~15);          // cap is a multiple of 4 slots
+    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
+    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.full_bar[s], 1);
+      mbar_init(&sm.empty_bar[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in flight)
+  // and written to the cache by the CTA whose chunk owns the slot.
+  for (int c = tid; c < D; c += NT) {
+    sm.aux_k(0)[c] = k_in[c];
+    sm.aux_v(0)[c] = v_in[c];
+  }
+  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
+    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
+    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
+    for (int c = tid; c < D; c += NT) { Kw[c] = k_in[c]; Vw[c] = v_in[c]; }
+  }
   __syncthreads();
-  combine_warps<D, G>(sm.warp_part, sm.cta_part);
+
+  if (warp == kConsumerWarps) {
+    if (lane_id == 0) {                                   // producer: keeps the ring full
+      for (int i = 0; i < v.n_tiles; ++i) {
+        const int s = i % kStages;
+        if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
+        const int slot0 = (v.tile_begin + i) * kTileSlots;
+        const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
+        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
+        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
+        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+      }
+    }
+  } else {
+    Scanner<T, D, G> sc;
+    sc.begin(q_in);
+    for (int i = 0; i < v.n_tiles; ++i) {
+      const int s = i % kStages;
+      mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
+      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
+      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, sm.chunk_logits,
+              P.chunk_cap, v.slot_begin);
+      __syncwarp();
+      if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
+    }
+    sc.end(sm.warp_part);
+  }
+  __syncthreads();
+  combine_warps<D, G, NT>(sm.warp_part, sm.cta_part);
   cluster.sync();                                       // #1: every CTA's partial is readable
 
   // (1) global max per head (every CTA), output weights (rank 0)
@@ -846,80 +956,79 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
     const int g = tid;
     float M = -INFINITY;
     for (int s = 0; s < S; ++s) M = fmaxf(M, cluster.map_shared_rank(sm.cta_part, s)[g * (D + 2)]);
-    sm.ep_M[g] = M;
+    sm.ep.M[g] = M;
     if (split == 0) {
       float lsum = 0.f;
       for (int s = 0; s < S; ++s) {
         const float* pp = cluster.map_shared_rank(sm.cta_part, s) + g * (D + 2);
         const float w = fast_exp2((pp[0] - M) * kLog2e);
-        sm.ep_w[g * kMaxSplits + s] = w;
+        sm.ep.w[g * kMaxSplits + s] = w;
         lsum += w * pp[1];
       }
-      sm.ep_linv[g] = 1.f / lsum;
+      sm.ep.linv[g] = 1.f / lsum;
     }
   }
   __syncthreads();
   // (2) o_t by rank 0
   if (split == 0) {
     T* out = reinterpret_cast<T*>(P.out) + v.b * P.out_bs + (long long)v.hk * G * D;
-    for (int idx = tid; idx < G * D; idx += kThreads) {
+    for (int idx = tid; idx < G * D; idx += NT) {
       const int g = idx / D, c = idx % D;
       float o = 0.f;
-      for (int s = 0; s < S; ++s) o += sm.ep_w[g * kMaxSplits + s] * cluster.map_shared_rank(sm.cta_part, s)[g * (D + 2) + 2 + c];
-      out[idx] = from_f32<T>(o * sm.ep_linv[g]);
+      for (int s = 0; s < S; ++s) o += sm.ep.w[g * kMaxSplits + s] * cluster.map_shared_rank(sm.cta_part, s)[g * (D + 2) + 2 + c];
+      out[idx] = from_f32<T>(o * sm.ep.linv[g]);
     }
   }
   // (3) this CTA's share of Z
   {
     unsigned long long zl[G];
-    exp_and_zsum<G, false>(sm.chunk_logits, P.chunk_cap, n_mine, sm.ep_M, zl);
-    block_sum_u64<G>(zl, sm.ep_u64);
+    exp_and_zsum<G, false, NT>(sm.chunk_logits, P.chunk_cap, n_mine, sm.ep.M, zl);
+    group_sum_u64<G, NT>(zl, sm.ep.u64);
     if (tid == 0) {
 #pragma unroll
-      for (int g = 0; g < G; ++g) sm.ep_u64[48 + g] = zl[g];
+      for (int g = 0; g < G; ++g) sm.ep.u64[80 + g] = zl[g];
     }
   }
   cluster.sync();                                       // #2: Z partials readable (and rank 0 is done with the o partials)
   if (tid < G) {
     unsigned long long z = 0ull;
-    for (int s = 0; s < S; ++s) z += cluster.map_shared_rank(sm.ep_u64, s)[48 + tid];
-    sm.ep_Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
+    for (int s = 0; s < S; ++s) z += cluster.map_shared_rank(sm.ep.u64, s)[80 + tid];
+    sm.ep.Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
   }
   __syncthreads();
   // (4) probabilities, score fold and pick over this CTA's slots
   const bool compress = v.L > P.budget;
   unsigned long long best = ~0ull;
   int best_slot = -1;
-  fold_scores<T, G>(P, v, sm.chunk_logits, P.chunk_cap, v.slot_begin, n_mine, sm.ep_Z, compress, best, best_slot);
+  fold_scores<T, G, NT>(P, v, sm.chunk_logits, P.chunk_cap, v.slot_begin, n_mine, sm.ep.Z, compress, best, best_slot);
   if (P.probs && split == S - 1) {
-    for (int i = v.L + tid; i < P.budget + 1; i += kThreads)
+    for (int i = v.L + tid; i < P.budget + 1; i += NT)
 #pragma unroll
       for (int g = 0; g < G; ++g)
         P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
   }
-  const unsigned long long my_min = block_min_key(best, best_slot, sm.ep_u64 + 40, &sm.ep_int[1]);
-  if (tid == 0) sm.ep_u64[56] = my_min;
+  const unsigned long long my_min = group_min_key<NT>(best, best_slot, sm.ep.u64 + 64, &sm.ep.i32[1]);
+  if (tid == 0) sm.ep.u64[88] = my_min;
   cluster.sync();                                       // #3: keys readable; a and pos of every slot are written
   // (5) rank 0 gathers the lane's pick
-  unsigned long long bmin = ~0ull;
   if (split == 0 && tid == 0) {
+    unsigned long long bmin = ~0ull;
     int j = -1;
     for (int s = 0; s < S; ++s) {
-      const unsigned long long k = cluster.map_shared_rank(sm.ep_u64, s)[56];
-      if (k < bmin) { bmin = k; j = cluster.map_shared_rank(sm.ep_int, s)[1]; }
+      const unsigned long long k = cluster.map_shared_rank(sm.ep.u64, s)[88];
+      if (k < bmin) { bmin = k; j = cluster.map_shared_rank(sm.ep.i32, s)[1]; }
     }
-    sm.ep_int[4] = j;
-    sm.ep_u64[57] = bmin;
+    sm.ep.i32[4] = j;
+    sm.ep.u64[89] = bmin;
   }
   cluster.sync();                                       // #4: nobody's shared memory is needed any more
   if (split != 0) return;
-  bmin = sm.ep_u64[57];
-  finish_lane<T, D, G>(P, v, sm, compress, bmin, sm.ep_int[4]);
+  finish_lane<T, D, G, NT>(P, v, sm.ep, compress, sm.ep.u64[89], sm.ep.i32[4]);
 }
 
 // Clears a context: every lane empty, chain heads/tails unset, slot 0 free.
 __global__ void reset_kernel(int32_t* lane_state, int32_t* pos, float* a, int32_t* next, int32_t* prev, long long lanes,
-                             int cap, uint32_t* ticket, int n_ticket, uint32_t* status) {
+                             int cap, uint32_t* status) {
   const long long n = lanes * cap;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     pos[i] = -1;
@@ -932,8 +1041,6 @@ __global__ void reset_kernel(int32_t* lane_state, int32_t* pos, float* a, int32_
     st[LS_LEN] = 0; st[LS_T] = 0; st[LS_HEAD] = -1; st[LS_TAIL] = -1; st[LS_FREE] = 0;
     st[5] = 0; st[6] = 0; st[7] = 0;
   }
-  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_ticket; i += (long long)gridDim.x * blockDim.x)
-    ticket[i] = 0u;
   if (blockIdx.x == 0 && threadIdx.x == 0) *status = 0u;
 }
 

@@ -13,15 +13,16 @@ from parity_util import Parity
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,n_sample,decode", [("llama7b_b8", 12, 16), ("serving_b16", 12, 12), ("gqa_b32", 10, 8)])
-def test_full_shape_sampled_lanes(name, n_sample, decode):
+@pytest.mark.parametrize("name,n_sample,decode,schedule", [("llama7b_b8", 12, 16, 0), ("serving_b16", 12, 12, 0),
+                                                           ("gqa_b32", 10, 8, 0), ("llama7b_b8", 6, 8, 2)])
+def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     wl = WORKLOADS[name]
     n_prefill = wl.budget + 160
     rng = np.random.default_rng(11)
     lens = rng.integers(n_prefill - 60, n_prefill + 1, wl.batch)       # ragged prompt ends, all beyond the budget
     lens[0] = n_prefill
     lens[-1] = n_prefill - 60
-    p = Parity(wl, sample=n_sample, ragged=lens.tolist())
+    p = Parity(wl, sample=n_sample, ragged=lens.tolist(), schedule=schedule)      # 0: the schedule bench.py gets
     assert p.ctx.wkv_device_bytes() > 0.9 * 2 * wl.lanes * (wl.budget + 1) * wl.head_dim * wl.elem_bytes
     p.prefill(n_prefill, chunk=32)
     p.compare_state()

@@ -41,9 +41,12 @@ def test_tiny_config_every_step():
     ("bf16", 128, 2, 2, 8, 8, 0, 0, 40),       # window == budget: a single candidate
     ("bf16", 128, 2, 2, 200, 32, 0, 64, 260),  # maximum split count
 ])
-def test_shapes_every_step(dtype, d, hq, hkv, m, W, S, splits, steps):
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+def test_shapes_every_step(dtype, d, hq, hkv, m, W, S, splits, steps, schedule):
+    if schedule == binding.WKV_SCHEDULE_CLUSTER and splits not in (0, 1, 2, 4, 8, 16):
+        pytest.skip("a cluster needs a power-of-two split count")
     wl = small(batch=3, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=W, S=S, rank=16 if dtype == "bf16" else 0)
-    p = Parity(wl, seed=17 + m, n_splits=splits)
+    p = Parity(wl, seed=17 + m, n_splits=splits, schedule=schedule)
     p.decode(steps)
     p.compare_state()
     assert p.n_evictions == wl.lanes * max(0, steps - m)
@@ -54,8 +57,8 @@ def test_split_count_does_not_change_results():
     """The same stream under 1, 2, 5 and 16 CTAs per lane: identical eviction sequences and bit-identical a."""
     wl = small(batch=2, d=128, dtype="bf16", m=150, W=8, rank=16)
     states = []
-    for splits in (1, 2, 5, 16):
-        p = Parity(wl, seed=5, n_splits=splits)
+    for splits, schedule in ((1, 1), (2, 2), (5, 1), (16, 2), (8, 1), (4, 0)):
+        p = Parity(wl, seed=5, n_splits=splits, schedule=schedule)
         assert p.ctx.wkv_splits() == splits
         p.decode(230)
         states.append([p.ctx.wkv_export_state(*ln) for ln in p.lanes])
@@ -65,10 +68,11 @@ def test_split_count_does_not_change_results():
             assert torch.equal(s0["pos"], s1["pos"]) and torch.equal(s0["a"], s1["a"]) and torch.equal(s0["V"], s1["V"])
 
 
-def test_ragged_prefill_then_decode():
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+def test_ragged_prefill_then_decode(schedule):
     """Per-sequence prompt lengths, one shorter than the budget so that lane is still growing during decode."""
     wl = small(layers=2, batch=4, d=128, dtype="bf16", m=96, W=8, rank=16)
-    p = Parity(wl, seed=9, ragged=[150, 40, 97, 96])
+    p = Parity(wl, seed=9, ragged=[150, 40, 97, 96], schedule=schedule)
     p.prefill(150, chunk=50)
     p.compare_state()
     p.decode(80)
@@ -76,10 +80,11 @@ def test_ragged_prefill_then_decode():
     p.close()
 
 
-def test_probabilities_output():
-    wl = small(batch=1, hq=4, hkv=2, d=64, dtype="f32", m=20, W=2)
-    p = Parity(wl, seed=3, check_probs=True)
-    p.decode(45)
+@pytest.mark.parametrize("schedule,splits", [(binding.WKV_SCHEDULE_SPLIT, 3), (binding.WKV_SCHEDULE_CLUSTER, 2)])
+def test_probabilities_output(schedule, splits):
+    wl = small(batch=1, hq=4, hkv=2, d=64, dtype="f32", m=70, W=2)
+    p = Parity(wl, seed=3, check_probs=True, schedule=schedule, n_splits=splits)
+    p.decode(95)
     p.close()
 
 
@@ -152,11 +157,12 @@ def test_argument_errors_leave_context_usable():
     ctx.close()
 
 
-def test_llama7b_layer_config_all_lanes():
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_AUTO, binding.WKV_SCHEDULE_SPLIT])
+def test_llama7b_layer_config_all_lanes(schedule):
     """One Llama-2-7B-shaped layer (32 heads x 128, bf16, budget 2048, window 64): every lane, every step of a
     prefill that fills the cache and runs 300 compressions, then 64 decode steps."""
     wl = WORKLOADS["llama7b_layer"]
-    p = Parity(wl)
+    p = Parity(wl, schedule=schedule)
     p.prefill(wl.budget + 300, chunk=128)
     p.decode(64)
     mism = p.compare_state()
