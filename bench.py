@@ -267,6 +267,25 @@ def main():
     assert int((ev >= 0).sum()) == ev.numel(), "every lane must compress in the timed region"
     value = aggregate_steps_per_s(world, args.steps, elapsed_ms)
 
+    # ---- additionally: the same steps through wkv_decode_step_layers (all layers' inputs handed over at once, so the
+    # library may overlap one layer's lane epilogues with the next layer's scan) ----
+    n_all = max(1, min(args.steps, 100))
+    for i in range(3):
+        q, k, v = toks[i]
+        ctx.wkv_decode_step_layers(q, k, v, out, ev)
+    torch.cuda.synchronize()
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a0.record()
+    for i in range(n_all):
+        q, k, v = toks[args.warmup + i]
+        ctx.wkv_decode_step_layers(q, k, v, out, ev)
+    a1.record()
+    torch.cuda.synchronize()
+    all_ms = max_over_ranks(a0.elapsed_time(a1), dist, dev)
+    all_layers = {"value": aggregate_steps_per_s(world, n_all, all_ms), "unit": "steps/s", "steps": n_all,
+                  "ms_per_step": all_ms / n_all,
+                  "note": "wkv_decode_step_layers: one call per step with every layer's q, k, v ready beforehand"}
+
     # ---- end to end: host buffers through wkv_decode_step_host, copies inside the timed region ----
     n_e2e = max(1, min(args.e2e_steps, args.steps))
     host = [tuple(x.cpu().pin_memory() for x in toks[args.warmup + i]) for i in range(n_e2e)]
@@ -312,7 +331,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
             "config": workload_config(wl, args, ctx.wkv_splits()),
-            "gpu_launches": launches, "clocks": clocks,
+            "gpu_launches": launches, "clocks": clocks, "all_layers_call": all_layers,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_8000_nominal": achieved / 8000.0,
                          "kernel": "scan_kernel (+ lane_epilogue_kernel)" if launches == 2 * args.steps * wl.n_layers

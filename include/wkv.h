@@ -106,6 +106,15 @@ int wkv_set_stream(wkv_ctx* ctx, void* stream);
 int wkv_decode_step(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
                     int32_t* evicted_pos, float* probs);
 
+/* All layers of one decode step in one call: wkv_decode_step for layer 0, 1, ..., n_layers-1 (Algorithm 1 per lane;
+ * the lanes of different layers are independent).
+ *   q   device [n_layers, batch, n_q_heads, head_dim];  k, v device [n_layers, batch, n_kv_heads, head_dim]
+ *   out device [n_layers, batch, n_q_heads, head_dim];  evicted_pos device [n_layers, batch, n_kv_heads] or NULL
+ * By making this call the caller states that ALL layers' q, k, v are complete on the stream before it; the library
+ * uses that to let each layer's cache scan run while the previous layer's per-lane epilogue is still finishing
+ * (results are identical to n_layers separate calls).  Inputs must not overlap the outputs.  Asynchronous. */
+int wkv_decode_step_layers(wkv_ctx* ctx, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos);
+
 /* No counterpart in the paper: this entry point exists for callers that must not allocate device memory.
  *
  * Some hosts of this library cannot call cudaMalloc at the moment they need a decode step: code running

@@ -29,7 +29,7 @@ class wkv_config(C.Structure):
 
 
 EXPORTS = ["wkv_config_error", "wkv_create", "wkv_destroy", "wkv_reset", "wkv_set_stream", "wkv_decode_step",
-           "wkv_decode_step_static", "wkv_decode_step_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
+           "wkv_decode_step_layers", "wkv_decode_step_static", "wkv_decode_step_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
            "wkv_status", "wkv_launch_count", "wkv_device_bytes", "wkv_splits", "wkv_strerror", "wkv_last_error"]
 
 _lib = None
@@ -51,6 +51,7 @@ def lib():
         L.wkv_reset.argtypes = [vp]
         L.wkv_set_stream.argtypes = [vp, vp]
         L.wkv_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+        L.wkv_decode_step_layers.argtypes = [vp, vp, vp, vp, vp, vp]
         L.wkv_decode_step_static.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.wkv_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.wkv_prefill.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp]
@@ -167,6 +168,9 @@ class Context:
 
     def wkv_decode_step(self, layer, q, k, v, out, evicted_pos=None, probs=None):
         self._check(lib().wkv_decode_step(self._h, layer, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos), _dp(probs)))
+
+    def wkv_decode_step_layers(self, q, k, v, out, evicted_pos=None):
+        self._check(lib().wkv_decode_step_layers(self._h, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos)))
 
     def wkv_decode_step_static(self, layer, q, k, v, out, evicted_pos=None):
         """wkv_decode_step with its scratch in the library's built-in device array: for callers that may not

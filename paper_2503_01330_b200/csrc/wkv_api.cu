@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/wkv.h: configuration checks, device state, launches,
 // export / import of lanes.  All arithmetic of the method lives in wkv_kernels.cuh.
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -32,8 +33,13 @@ struct wkv_ctx {
   int32_t* next = nullptr;
   int32_t* prev = nullptr;
   int32_t* lane_state = nullptr;
-  float* logits = nullptr;
-  float* part = nullptr;
+  float* logits[2] = {nullptr, nullptr};   // two scratch sets: consecutive layer calls may overlap (see prepare_overlap)
+  float* part[2] = {nullptr, nullptr};
+  int parity = 0;
+  // what the previous layer call of this context wrote for the caller, and for which layer
+  int last_layer = -1;
+  const char* last_out[3] = {nullptr, nullptr, nullptr};
+  size_t last_out_bytes[3] = {0, 0, 0};
   uint32_t* status = nullptr;
   // staging for the host-buffer entry point and for discarded prefill outputs
   void* stage_q = nullptr;
@@ -151,11 +157,28 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
   }
   const int n_ctas = lanes * P.n_splits;
   if (!cluster) {
-    wkv::scan_kernel<T, D, G><<<n_ctas, wkv::kThreads, smem, stream>>>(P);
-    e = cudaGetLastError();
+    // Both kernels are launched with programmatic stream serialization: each may be set up while its predecessor
+    // drains and orders itself against it on the device (griddep_wait in the kernels).
+    cudaLaunchAttribute pdl[1];
+    pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    pdl[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t k1 = {};
+    k1.gridDim = dim3((unsigned)n_ctas);
+    k1.blockDim = dim3(wkv::kThreads);
+    k1.dynamicSmemBytes = (size_t)smem;
+    k1.stream = stream;
+    k1.attrs = pdl;
+    k1.numAttrs = 1;
+    e = cudaLaunchKernelEx(&k1, wkv::scan_kernel<T, D, G>, P);
     if (e != cudaSuccess) return e;
-    wkv::lane_epilogue_kernel<T, D, G><<<lanes, wkv::kEpilogueThreads, 0, stream>>>(P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t k2 = {};
+    k2.gridDim = dim3((unsigned)lanes);
+    k2.blockDim = dim3(wkv::kEpilogueThreads);
+    k2.dynamicSmemBytes = 0;
+    k2.stream = stream;
+    k2.attrs = pdl;
+    k2.numAttrs = 1;
+    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G>, P);
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)n_ctas);
@@ -198,7 +221,7 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   wkv::StepParams P;
   std::memset(&P, 0, sizeof(P));
   P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
-  P.lane_state = c->lane_state; P.logits = c->logits; P.part = c->part; P.status = c->status;
+  P.lane_state = c->lane_state; P.logits = c->logits[0]; P.part = c->part[0]; P.status = c->status;
   P.lane0 = layer * c->lanes_per_layer;
   P.n_kv_heads = c->cfg.n_kv_heads;
   P.cap = c->cap;
@@ -208,6 +231,44 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   P.merge = c->cfg.merge;
   P.scale = c->scale;
   return P;
+}
+
+bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
+  if (!a || !b || !na || !nb) return false;
+  const char* x = (const char*)a;
+  const char* y = (const char*)b;
+  return x < y + nb && y < x + na;
+}
+
+// The context whose kernels were the last ones this library launched (see prepare_overlap).
+std::atomic<const wkv_ctx*> g_last_launcher{nullptr};
+
+// Two-kernel schedule: choose the scratch set of this layer call and decide whether its scan may start while the
+// previous call's lane epilogue is still running.  Only a caller that vouches for its inputs (inputs_ready: q, k, v of
+// this call were complete before the previous layer call was issued -- wkv_decode_step_layers) can get that overlap,
+// and then only if the previous call of this context was for another layer, no other context launched in between,
+// and this call's inputs do not alias what the previous call wrote for the caller.  A scan behind a foreign kernel
+// always waits for it first: nothing is known about when that kernel's results become visible.
+void prepare_overlap(wkv_ctx* c, wkv::StepParams& P, int layer, size_t q_bytes, size_t kv_bytes, bool inputs_ready) {
+  c->parity ^= 1;
+  P.logits = c->logits[c->parity];
+  P.part = c->part[c->parity];
+  bool wait = !inputs_ready || c->last_layer < 0 || c->last_layer == layer || g_last_launcher.load() != c;
+  for (int i = 0; i < 3 && !wait; ++i) {
+    wait = ranges_overlap(P.q, q_bytes, c->last_out[i], c->last_out_bytes[i]) ||
+           ranges_overlap(P.k, kv_bytes, c->last_out[i], c->last_out_bytes[i]) ||
+           ranges_overlap(P.v, kv_bytes, c->last_out[i], c->last_out_bytes[i]);
+  }
+  P.wait_at_start = wait ? 1 : 0;
+  c->last_layer = layer;
+  g_last_launcher.store(c);
+}
+
+void note_outputs(wkv_ctx* c, const void* out, size_t out_bytes, const void* ev, size_t ev_bytes, const void* probs,
+                  size_t probs_bytes) {
+  c->last_out[0] = (const char*)out;   c->last_out_bytes[0] = out_bytes;
+  c->last_out[1] = (const char*)ev;    c->last_out_bytes[1] = ev_bytes;
+  c->last_out[2] = (const char*)probs; c->last_out_bytes[2] = probs_bytes;
 }
 
 int run_reset(wkv_ctx* c) {
@@ -293,8 +354,10 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   T(take(c, &c->next, (size_t)c->lanes_total * cap * 4));
   T(take(c, &c->prev, (size_t)c->lanes_total * cap * 4));
   T(take(c, &c->lane_state, (size_t)c->lanes_total * wkv::LS_STRIDE * 4));
-  T(take(c, &c->logits, (size_t)c->lanes_per_layer * G * cap * 4));
-  T(take(c, &c->part, (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
+  for (int i = 0; i < 2; ++i) {
+    T(take(c, &c->logits[i], (size_t)c->lanes_per_layer * G * cap * 4));
+    T(take(c, &c->part[i], (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
+  }
   T(take(c, &c->status, 256));
   T(take(c, &c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * row));
   T(take(c, &c->stage_k, (size_t)c->lanes_per_layer * row));
@@ -319,17 +382,19 @@ void wkv_destroy(wkv_ctx* c) {
 
 int wkv_reset(wkv_ctx* c) {
   if (!c) return WKV_ERR_INVALID;
+  c->last_layer = -1;
   return run_reset(c);
 }
 
 int wkv_set_stream(wkv_ctx* c, void* stream) {
   if (!c) return WKV_ERR_INVALID;
+  c->last_layer = -1;                  // nothing is known about what runs on the new stream
   c->stream = reinterpret_cast<cudaStream_t>(stream);
   return WKV_OK;
 }
 
-int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
-                    int32_t* evicted_pos, float* probs) {
+static int decode_step_impl(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                            int32_t* evicted_pos, float* probs, bool inputs_ready) {
   if (!c) return WKV_ERR_INVALID;
   if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
   if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
@@ -342,9 +407,43 @@ int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, con
   P.ev_bs = c->cfg.n_kv_heads;
   P.seq_lens = nullptr;
   P.tok_idx = 0;
+  const size_t row = (size_t)D * c->elem;
+  const size_t q_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * row, kv_bytes = (size_t)c->lanes_per_layer * row;
+  if (!c->use_cluster) prepare_overlap(c, P, layer, q_bytes, kv_bytes, inputs_ready);
   cudaError_t e = launch_any(c, P, c->use_cluster);
   c->launches += c->use_cluster ? 1 : 2;
   if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch");
+  note_outputs(c, out, q_bytes, evicted_pos, (size_t)c->lanes_per_layer * 4, probs,
+               (size_t)c->cfg.batch * c->cfg.n_q_heads * (c->cfg.budget + 1) * 4);
+  return WKV_OK;
+}
+
+int wkv_decode_step(wkv_ctx* c, int32_t layer, const void* q, const void* k, const void* v, void* out,
+                    int32_t* evicted_pos, float* probs) {
+  return decode_step_impl(c, layer, q, k, v, out, evicted_pos, probs, false);
+}
+
+int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
+  const size_t row = (size_t)c->cfg.head_dim * c->elem;
+  const size_t q_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * row, kv_bytes = (size_t)c->lanes_per_layer * row;
+  const size_t nl = (size_t)c->cfg.n_layers;
+  // the whole output range belongs to this call: a later layer's inputs must not alias an earlier layer's outputs
+  if (ranges_overlap(q, q_bytes * nl, out, q_bytes * nl) || ranges_overlap(k, kv_bytes * nl, out, q_bytes * nl) ||
+      ranges_overlap(v, kv_bytes * nl, out, q_bytes * nl) ||
+      ranges_overlap(q, q_bytes * nl, evicted_pos, (size_t)c->lanes_per_layer * 4 * nl) ||
+      ranges_overlap(k, kv_bytes * nl, evicted_pos, (size_t)c->lanes_per_layer * 4 * nl) ||
+      ranges_overlap(v, kv_bytes * nl, evicted_pos, (size_t)c->lanes_per_layer * 4 * nl))
+    return fail(c, WKV_ERR_INVALID, "wkv_decode_step_layers: inputs and outputs must not overlap");
+  c->last_layer = -1;                   // the first layer's scan orders itself behind whatever ran before this call
+  for (int layer = 0; layer < c->cfg.n_layers; ++layer) {
+    int rc = decode_step_impl(c, layer, (const char*)q + layer * q_bytes, (const char*)k + layer * kv_bytes,
+                              (const char*)v + layer * kv_bytes, (char*)out + layer * q_bytes,
+                              evicted_pos ? evicted_pos + (size_t)layer * c->lanes_per_layer : nullptr, nullptr, true);
+    if (rc != WKV_OK) return rc;
+  }
+  c->last_layer = -1;
   return WKV_OK;
 }
 
@@ -377,6 +476,9 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   P.tok_idx = 0;
   // The array keeps whatever the previous call (of any context) left.  Nothing in it has to start at zero: the scan
   // kernel writes every logit and every partial of an active lane before the epilogue kernel reads them.
+  P.wait_at_start = 1;                 // one array for everybody: never start before the previous kernel has finished
+  c->last_layer = -1;
+  g_last_launcher.store(nullptr);
   e = launch_any(c, P, false);
   c->launches += 2;
   if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (static scratch)");
@@ -392,7 +494,7 @@ int wkv_decode_step_host(wkv_ctx* c, int32_t layer, const void* q, const void* k
   WKV_CUDA(c, cudaMemcpyAsync(c->stage_q, q, qb, cudaMemcpyHostToDevice, c->stream));
   WKV_CUDA(c, cudaMemcpyAsync(c->stage_k, k, kb, cudaMemcpyHostToDevice, c->stream));
   WKV_CUDA(c, cudaMemcpyAsync(c->stage_v, v, kb, cudaMemcpyHostToDevice, c->stream));
-  int rc = wkv_decode_step(c, layer, c->stage_q, c->stage_k, c->stage_v, c->stage_out, c->stage_ev, nullptr);
+  int rc = decode_step_impl(c, layer, c->stage_q, c->stage_k, c->stage_v, c->stage_out, c->stage_ev, nullptr, false);
   if (rc != WKV_OK) return rc;
   WKV_CUDA(c, cudaMemcpyAsync(out, c->stage_out, qb, cudaMemcpyDeviceToHost, c->stream));
   if (evicted_pos)
@@ -421,10 +523,12 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
     P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
     P.out = out ? (void*)((char*)out + (size_t)t * Hq * D * c->elem) : c->stage_out;
     P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
+    if (!c->use_cluster) prepare_overlap(c, P, layer, 0, 0, false);     // token after token on one layer: no overlap
     cudaError_t e = launch_any(c, P, c->use_cluster);
     c->launches += c->use_cluster ? 1 : 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (prefill)");
   }
+  note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
   return WKV_OK;
 }
 

@@ -81,6 +81,7 @@ struct StepParams {
   int n_splits;
   int chunk_cap;         // cluster kernel: logits one CTA can hold per query head (its tiles * 32)
   int merge;
+  int wait_at_start;     // scan kernel: 1 = wait for the preceding kernel before touching anything (see scan_kernel)
   float scale;
 };
 
@@ -130,6 +131,12 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void l2_prefetch(const void* src, uint32_t bytes) {
   asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
+// Programmatic dependent launch.  griddep_wait: block until the kernel this one was launched behind has completed and
+// its writes are visible (returns at once when the launch carried no such dependency).  griddep_launch: allow the
+// next kernel in the stream to begin once every CTA of this grid has called it or exited.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Barrier among the first NT threads of the CTA (NT = kThreads: the whole CTA).
 template <int NT>
 __device__ __forceinline__ void group_sync() {
@@ -288,6 +295,7 @@ struct LaneView {
   const T *Kl, *Vl;          // the lane's cache rows
   const T *new_k, *new_v;    // this step's token (shared memory)
   int* st;                   // the lane's state words
+  int head, tail;            // chain ends before this step (only the code that finishes the lane reads them)
 };
 
 // Lane-level part of a view: addresses and the even deal of tiles (the first tiles_total % n_splits units get one more).
@@ -303,6 +311,8 @@ __device__ __forceinline__ void fill_view(LaneView<T>& v, const StepParams& P, i
   v.len = len;
   v.t = t;
   v.new_slot = new_slot;
+  v.head = -1;
+  v.tail = -1;
   v.L = len + 1;
   v.Kl = reinterpret_cast<const T*>(P.Kc) + v.lane * (long long)P.cap * D;
   v.Vl = reinterpret_cast<const T*>(P.Vc) + v.lane * (long long)P.cap * D;
@@ -628,14 +638,21 @@ __device__ __forceinline__ unsigned long long group_min_key(unsigned long long b
 template <typename T, int D, int G, int NT>
 __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const EpScratch& ep, bool compress,
                                             unsigned long long bmin, int j_slot) {
+  static_assert(NT >= D, "one thread per channel of the merged row");
   const int tid = threadIdx.x;
   const int t = v.t, new_slot = v.new_slot, L = v.L;
   float* a_l = P.a + v.lane * P.cap;
   int32_t* pos_l = P.pos + v.lane * P.cap;
   int32_t* next_l = P.next + v.lane * P.cap;
   int32_t* prev_l = P.prev + v.lane * P.cap;
+  T* Vw = const_cast<T*>(v.Vl);
+  // the victim's value row does not depend on the chain walk below: fetch it meanwhile
+  // (the row of this step's token may have been written to the cache by other threads: v.new_v is the safe copy)
+  float vj = 0.f;
+  const bool merging = compress && P.merge && j_slot >= 0;
+  if (merging && tid < D) vj = to_f32(j_slot == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)j_slot * D + tid));
   if (tid == 0) {
-    int head = v.st[LS_HEAD], tail = v.st[LS_TAIL];
+    int head = v.head, tail = v.tail;
     next_l[new_slot] = -1;
     prev_l[new_slot] = tail;
     if (tail >= 0) next_l[tail] = new_slot; else head = new_slot;
@@ -648,6 +665,7 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
       if (j < 0 || r < 0 || r >= P.cap) {
         atomicOr(P.status, kStatusBadLink);              // cannot happen with budget >= sink + window
       } else {
+        const int pv = prev_l[j];
         const float abar_j = __uint_as_float((uint32_t)(bmin >> 32));
         const int pos_r = r == new_slot ? t : __ldcg(pos_l + r);
         const float abar_r = __fdiv_rn(__ldcg(a_l + r), __int2float_rn(t - pos_r + 1));
@@ -659,7 +677,6 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
         ep.i32[2] = j;
         ep.i32[3] = r;
         ev_pos = (int)(uint32_t)(bmin & 0xffffffffull);
-        const int pv = prev_l[j];
         if (pv >= 0) next_l[pv] = r; else head = r;
         prev_l[r] = pv;
         pos_l[j] = -1;
@@ -676,16 +693,11 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
   }
   group_sync<NT>();
   // V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r), stored in T
-  if (compress && P.merge && ep.i32[2] >= 0) {
-    const int j = ep.i32[2], r = ep.i32[3];
+  if (merging && ep.i32[2] >= 0 && tid < D) {
+    const int r = ep.i32[3];
     const float wj = ep.misc[0], wr = ep.misc[1];
-    T* Vw = const_cast<T*>(v.Vl);
-    for (int c = tid; c < D; c += NT) {
-      // the row of this step's token may have been written to the cache by other threads: take it from shared memory
-      const float vj = to_f32(j == new_slot ? v.new_v[c] : __ldcg(Vw + (long long)j * D + c));
-      const float vr = to_f32(r == new_slot ? v.new_v[c] : __ldcg(Vw + (long long)r * D + c));
-      Vw[(long long)r * D + c] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
-    }
+    const float vr = to_f32(r == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r * D + tid));
+    Vw[(long long)r * D + tid] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
   }
 }
 
@@ -768,7 +780,17 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
   const int split = blockIdx.x % P.n_splits;
   const int lane_local = blockIdx.x / P.n_splits;
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
-  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) return;      // sequence already consumed (ragged prefill)
+  // Ordering against the kernel launched just before this one.  Normally the scan waits for it right here.  When the
+  // caller has handed over all layers of a step at once (wkv_decode_step_layers) and the host saw no conflict, that
+  // kernel is the lane epilogue of the previous layer, which works on other lanes and on the other scratch set: the
+  // scan then runs alongside it and waits only at its very end, so that the completion of this grid still implies the
+  // completion of everything before it and later kernels need not reason about more than one predecessor.
+  if (P.wait_at_start) griddep_wait();
+  griddep_launch();
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {            // sequence already consumed (ragged prefill)
+    if (!P.wait_at_start) griddep_wait();
+    return;
+  }
   LaneView<T> v;
   {
     const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
@@ -835,6 +857,7 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
   }
   __syncthreads();
   combine_warps<D, G, NT>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
+  if (!P.wait_at_start) griddep_wait();
 }
 
 constexpr int kEpilogueThreads = 256;
@@ -846,15 +869,24 @@ __global__ void __launch_bounds__(kEpilogueThreads) lane_epilogue_kernel(const S
   ep.carve(ep_raw, G);
   const int lane_local = blockIdx.x;
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
-  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed (ragged prefill)
+  const bool active = !(P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]);   // else: sequence already consumed
+  // The lane's state words were last written by an earlier lane epilogue of the same layer, which is complete (the
+  // scan in front of this kernel did not finish before everything older had finished): read them before waiting.
+  LaneView<T> v;
+  const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+  if (active) {
+    fill_view<T, D>(v, P, lane_local, 0, st[LS_LEN], st[LS_T], st[LS_FREE]);
+    v.head = st[LS_HEAD];
+    v.tail = st[LS_TAIL];
+    v.new_k = v.Kl + (long long)v.new_slot * D;          // the scan kernel has stored this step's token in the cache
+    v.new_v = v.Vl + (long long)v.new_slot * D;
+  }
+  griddep_wait();                                        // the scan is complete: logits and partials are visible
+  griddep_launch();                                      // the next kernel in the stream may be set up alongside
+  if (!active) {
     if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
     return;
   }
-  LaneView<T> v;
-  const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
-  fill_view<T, D>(v, P, lane_local, 0, st[LS_LEN], st[LS_T], st[LS_FREE]);
-  v.new_k = v.Kl + (long long)v.new_slot * D;            // the scan kernel has stored this step's token in the cache
-  v.new_v = v.Vl + (long long)v.new_slot * D;
   lane_epilogue_from_scratch<T, D, G, kEpilogueThreads>(P, v, ep);
 }
 
@@ -892,6 +924,7 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
   const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
   const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
   const int n_mine = v.slot_end - v.slot_begin;
+  if (split == 0) { v.head = v.st[LS_HEAD]; v.tail = v.st[LS_TAIL]; }
 
   if (tid == 32 && n_mine > 0) {
     // The epilogue reads a and pos of these slots long after the scan: pull their lines into L2 now.

@@ -108,7 +108,7 @@ class Parity:
             self.t += tc
 
     # ---- decode through wkv_decode_step --------------------------------------------------------------
-    def decode(self, n_steps, host_entry=False):
+    def decode(self, n_steps, host_entry=False, layers_entry=False):
         wl = self.wl
         for s in range(n_steps):
             q, k, v = self.stream.token(self.t)
@@ -120,6 +120,8 @@ class Parity:
                     self.ctx.wkv_decode_step_host(layer, qh[layer], kh[layer], vh[layer], oh[layer], eh[layer])
                 self.out.copy_(oh)
                 self.ev.copy_(eh)
+            elif layers_entry:
+                self.ctx.wkv_decode_step_layers(q, k, v, self.out, self.ev)
             else:
                 for layer in range(wl.n_layers):
                     self.ctx.wkv_decode_step(layer, q[layer], k[layer], v[layer], self.out[layer], self.ev[layer],

@@ -27,6 +27,7 @@ def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     p.prefill(n_prefill, chunk=32)
     p.compare_state()
     p.decode(decode)
+    p.decode(4, layers_entry=True)
     p.compare_state()
     assert p.n_evictions >= len(p.lanes) * (100 + decode)
     p.close()

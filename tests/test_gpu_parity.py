@@ -105,6 +105,18 @@ def test_host_buffer_entry_point():
     p.close()
 
 
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+def test_all_layers_entry_point(schedule):
+    """wkv_decode_step_layers lets consecutive layers overlap on the GPU; results must not change."""
+    wl = small(layers=6, batch=3, d=128, dtype="bf16", m=120, W=8, rank=16)
+    p = Parity(wl, seed=12, schedule=schedule, n_splits=2)
+    p.decode(100, layers_entry=True)
+    p.decode(20)
+    p.decode(60, layers_entry=True)
+    p.compare_state()
+    p.close()
+
+
 def test_export_import_roundtrip_and_continue():
     wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=24, W=3)
     p = Parity(wl, seed=8)
