@@ -253,13 +253,16 @@ void prepare_overlap(wkv_ctx* c, wkv::StepParams& P, int layer, size_t q_bytes, 
   c->parity ^= 1;
   P.logits = c->logits[c->parity];
   P.part = c->part[c->parity];
-  bool wait = !inputs_ready || c->last_layer < 0 || c->last_layer == layer || g_last_launcher.load() != c;
-  for (int i = 0; i < 3 && !wait; ++i) {
-    wait = ranges_overlap(P.q, q_bytes, c->last_out[i], c->last_out_bytes[i]) ||
-           ranges_overlap(P.k, kv_bytes, c->last_out[i], c->last_out_bytes[i]) ||
-           ranges_overlap(P.v, kv_bytes, c->last_out[i], c->last_out_bytes[i]);
+  // 2: the previous kernel may touch this layer's lanes or is unknown; 1: it cannot, but it may be what produces this
+  // call's inputs; 0: the caller vouches for the inputs and they do not alias the previous call's outputs.
+  int level = (c->last_layer < 0 || c->last_layer == layer || g_last_launcher.load() != c) ? 2 : (inputs_ready ? 0 : 1);
+  for (int i = 0; i < 3 && level == 0; ++i) {
+    if (ranges_overlap(P.q, q_bytes, c->last_out[i], c->last_out_bytes[i]) ||
+        ranges_overlap(P.k, kv_bytes, c->last_out[i], c->last_out_bytes[i]) ||
+        ranges_overlap(P.v, kv_bytes, c->last_out[i], c->last_out_bytes[i]))
+      level = 1;
   }
-  P.wait_at_start = wait ? 1 : 0;
+  P.wait_at_start = level;
   c->last_layer = layer;
   g_last_launcher.store(c);
 }
@@ -476,7 +479,7 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   P.tok_idx = 0;
   // The array keeps whatever the previous call (of any context) left.  Nothing in it has to start at zero: the scan
   // kernel writes every logit and every partial of an active lane before the epilogue kernel reads them.
-  P.wait_at_start = 1;                 // one array for everybody: never start before the previous kernel has finished
+  P.wait_at_start = 2;                 // one array for everybody: never start before the previous kernel has finished
   c->last_layer = -1;
   g_last_launcher.store(nullptr);
   e = launch_any(c, P, false);

@@ -81,7 +81,7 @@ struct StepParams {
   int n_splits;
   int chunk_cap;         // cluster kernel: logits one CTA can hold per query head (its tiles * 32)
   int merge;
-  int wait_at_start;     // scan kernel: 1 = wait for the preceding kernel before touching anything (see scan_kernel)
+  int wait_at_start;     // scan kernel: how it orders itself against the preceding kernel, 0 / 1 / 2 (see scan_kernel)
   float scale;
 };
 
@@ -780,15 +780,19 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
   const int split = blockIdx.x % P.n_splits;
   const int lane_local = blockIdx.x / P.n_splits;
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
-  // Ordering against the kernel launched just before this one.  Normally the scan waits for it right here.  When the
-  // caller has handed over all layers of a step at once (wkv_decode_step_layers) and the host saw no conflict, that
-  // kernel is the lane epilogue of the previous layer, which works on other lanes and on the other scratch set: the
-  // scan then runs alongside it and waits only at its very end, so that the completion of this grid still implies the
-  // completion of everything before it and later kernels need not reason about more than one predecessor.
-  if (P.wait_at_start) griddep_wait();
+  // Ordering against the kernel launched just before this one (P.wait_at_start, chosen by the host):
+  //   2  wait right here: the predecessor may touch this layer's lanes (same layer twice in a row, reset, ...).
+  //   1  the predecessor works on other memory, but the caller's q, k, v may come from it: set up, read the lane's
+  //      state and put the first K/V tiles in flight, then wait before the first read of a caller input.
+  //   0  the caller has handed over all layers of a step at once (wkv_decode_step_layers): the predecessor is the lane
+  //      epilogue of the previous layer (other lanes, other scratch set); scan alongside it and wait only at the very
+  //      end, so that the completion of this grid still implies the completion of everything before it and later
+  //      kernels need not reason about more than one predecessor.
+  if (P.wait_at_start == 2) griddep_wait();
   griddep_launch();
+  if (P.wait_at_start == 1 && P.seq_lens != nullptr) griddep_wait();     // seq_lens is a caller input
   if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {            // sequence already consumed (ragged prefill)
-    if (!P.wait_at_start) griddep_wait();
+    if (P.wait_at_start != 2) griddep_wait();
     return;
   }
   LaneView<T> v;
@@ -807,13 +811,25 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
     l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
     l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
   }
-  if (tid == 0) {
+  // The producer thread sets the ring up and fills every stage once; none of that reads a caller input.
+  auto issue_tile = [&](int i) {
+    const int s = i % kStages;
+    const int slot0 = (v.tile_begin + i) * kTileSlots;
+    const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
+    unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
+    mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
+    bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+    bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+  };
+  if (tid == kConsumerWarps * 32) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.full_bar[s], 1);
       mbar_init(&sm.empty_bar[s], kConsumerWarps);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int i = 0; i < min(v.n_tiles, kStages); ++i) issue_tile(i);
   }
+  if (P.wait_at_start == 1) griddep_wait();
   // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in flight)
   // and written to the cache by the CTA whose chunk owns the slot.
   for (int c = tid; c < D; c += NT) {
@@ -829,15 +845,9 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
 
   if (warp == kConsumerWarps) {
     if (lane_id == 0) {                                   // producer: keeps the ring full
-      for (int i = 0; i < v.n_tiles; ++i) {
-        const int s = i % kStages;
-        if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
-        const int slot0 = (v.tile_begin + i) * kTileSlots;
-        const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
-        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
-        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
-        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
-        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+      for (int i = kStages; i < v.n_tiles; ++i) {
+        mbar_wait(&sm.empty_bar[i % kStages], ((i / kStages) - 1) & 1, P.status);
+        issue_tile(i);
       }
     }
   } else {
