@@ -32,6 +32,15 @@ from paper_2503_01330_b200.synth import BASE_SEED, WORKLOADS, TokenStream, seque
 
 METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
+# workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
+# profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
+NCU_TRAFFIC = {"serving_b16": (1090744000 + 26963000 + 14383000, "e2e03d96b85b4c92")}
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    path = os.path.join(ROOT, "paper_2503_01330_b200", "csrc", "wkv_kernels.cuh")
+    return hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
 
 
 # ------------------------------------------------------------------------------------------------------
@@ -320,13 +329,11 @@ def main():
     # algorithmic bytes of one layer, so the fraction is taken over the whole call, not over the scan alone
     launch_ms = elapsed_ms / (args.steps * wl.n_layers)
     achieved = bytes_launch / (launch_ms * 1e-3) / 1e9
-    traffic = None      # DRAM bytes per launch from an ncu capture; see profiles/
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        try:
-            traffic = json.load(open(tpath)).get(wl.name)
-        except Exception:
-            traffic = None
+    # DRAM bytes per layer call from the ncu capture summarised under profiles/ (scan + lane epilogue kernels); only
+    # reported while the kernel source is the one that was profiled
+    traffic = None
+    if NCU_TRAFFIC.get(wl.name) and NCU_TRAFFIC[wl.name][1] == kernel_source_hash() and not args.layers:
+        traffic = NCU_TRAFFIC[wl.name][0]
     line = {"metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
