@@ -37,9 +37,10 @@
 //
 // Pinned binary32 rules (mode 1); every operation is IEEE-754 binary32 round-to-nearest-even,
 // no flush-to-zero, no contraction except where fma is written:
-//   P1 dot : 16 partial sums; partial r covers channels [r*d/16, (r+1)*d/16) left to right as
-//            acc = fma(q_c, k_c, acc) from +0.  Then four butterfly rounds p_r <- p_r + p_{r xor off},
-//            off = 8,4,2,1.  s = scale32 * p_0, scale32 = (float) scale.
+//   P1 dot : 16 partial sums; partial r covers channels [r*d/16, (r+1)*d/16): its even channels and its odd
+//            channels are each accumulated left to right as acc = fma(q_c, k_c, acc) from +0 and the two
+//            chains are added.  Then four butterfly rounds p_r <- p_r + p_{r xor off}, off = 8,4,2,1.
+//            s = scale32 * p_0, scale32 = (float) scale.
 //   P2 max : M = max_i s_i;  x_i = s_i - M.
 //   P3 exp : e = 0 if x < -87; else n = rint(x*LOG2E); f = fma(n,-LN2_HI,x); f = fma(n,-LN2_LO,f);
 //            degree-7 Horner in fma with c_k = (float)(1/k!); e = poly * 2^n (exact).
@@ -92,9 +93,12 @@ float pinned_dot(const float* q, const float* k, int d, float scale32) {
   float p[16];
   const int w = d / 16;
   for (int r = 0; r < 16; ++r) {
-    float acc = 0.0f;
-    for (int c = r * w; c < (r + 1) * w; ++c) acc = std::fmaf(q[c], k[c], acc);
-    p[r] = acc;
+    float even = 0.0f, odd = 0.0f;
+    for (int c = r * w; c < (r + 1) * w; ++c) {
+      if ((c - r * w) % 2 == 0) even = std::fmaf(q[c], k[c], even);
+      else odd = std::fmaf(q[c], k[c], odd);
+    }
+    p[r] = even + odd;
   }
   for (int off = 8; off >= 1; off >>= 1) {
     float nxt[16];

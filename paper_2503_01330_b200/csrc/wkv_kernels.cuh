@@ -23,8 +23,9 @@
 // Reproducible binary32 score path (decides the eviction index, therefore specified operation by operation;
 // all operations IEEE round-to-nearest-even, explicit intrinsics so the compiler neither contracts nor
 // reassociates):
-//   dot   : 16 partial sums over contiguous channel blocks of head_dim/16, fma chain from +0, then a
-//           butterfly p_r + p_{r^off}, off = 8,4,2,1; logit = scale * p.
+//   dot   : 16 partial sums over contiguous channel blocks of head_dim/16; inside a block the even channels and the
+//           odd channels each form an fma chain from +0 (one packed fp32x2 fma per channel pair) and the two chains
+//           are added; then a butterfly p_r + p_{r^off}, off = 8,4,2,1; logit = scale * p.
 //   exp   : 0 below -87; n = rint(x*LOG2E); Cody-Waite reduction with LN2_HI/LN2_LO; degree-7 Taylor
 //           polynomial in Horner form with fma; exact scaling by 2^n.
 //   sum   : Z = float(sum_i trunc(e_i * 2^40)) * 2^-40 -- an integer sum, hence order-free.
@@ -183,6 +184,54 @@ template <typename T> __device__ __forceinline__ T from_f32(float x);
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
+// Packed pairs of binary32 values in one 64-bit register.  fma2 / mul2 are two independent IEEE round-to-nearest
+// operations per instruction (no flush-to-zero), so each half is bit-identical to the scalar fma / multiply.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ float lo_of(f32x2 v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float hi_of(f32x2 v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// NPAIR (even, odd) channel pairs of a row chunk, widened to fp32.  16-byte aligned except the 8-byte bf16 x 4 case.
+template <int NPAIR>
+__device__ __forceinline__ void load_pairs(const float* p, f32x2 (&x)[NPAIR]) {
+#pragma unroll
+  for (int i = 0; i < NPAIR; i += 2) {
+    const float4 t = *reinterpret_cast<const float4*>(p + 2 * i);
+    x[i] = pack2(t.x, t.y);
+    x[i + 1] = pack2(t.z, t.w);
+  }
+}
+template <int NPAIR>
+__device__ __forceinline__ void load_pairs(const __nv_bfloat16* p, f32x2 (&x)[NPAIR]) {
+  if constexpr (NPAIR == 2) {
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    x[0] = pack2(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u));
+    x[1] = pack2(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+  } else {
+#pragma unroll
+    for (int i = 0; i < NPAIR; i += 4) {
+      const uint4 t = *reinterpret_cast<const uint4*>(p + 2 * i);
+      x[i + 0] = pack2(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u));
+      x[i + 1] = pack2(__uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+      x[i + 2] = pack2(__uint_as_float(t.z << 16), __uint_as_float(t.z & 0xffff0000u));
+      x[i + 3] = pack2(__uint_as_float(t.w << 16), __uint_as_float(t.w & 0xffff0000u));
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // reproducible exp (see the header comment)
 // ------------------------------------------------------------------------------------------------
@@ -336,23 +385,25 @@ struct Scanner {
   static constexpr int LPR = C::kLanesPerRow;    // 8 or 16 threads per row
   static constexpr int NP = 16 / LPR;            // partial sums per thread
   static constexpr int CH = D / 16;              // channels per partial sum
+  static constexpr int CP = CH / 2;              // ... as (even, odd) channel pairs: the arithmetic is packed fp32x2
   static constexpr int RPP = 32 / LPR;           // rows per warp pass
   static constexpr int PASSES = 8 / RPP;
-  float qf[G][NP][CH];
-  float m_run[G], l_run[G], o_acc[G][NP][CH];
+  f32x2 qf[G][NP][CP];
+  float m_run[G], l_run[G];
+  f32x2 o_acc[G][NP][CP];
 
   __device__ __forceinline__ void begin(const T* q) {      // q: [G][D], 16-byte aligned (global or shared)
     const int l = (threadIdx.x & 31) % LPR;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
 #pragma unroll
-      for (int j = 0; j < NP; ++j) load_chunk<CH>(q + g * D + (l + LPR * j) * CH, qf[g][j]);
+      for (int j = 0; j < NP; ++j) load_pairs<CP>(q + g * D + (l + LPR * j) * CH, qf[g][j]);
       m_run[g] = -INFINITY;
       l_run[g] = 0.f;
 #pragma unroll
       for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CH; ++e) o_acc[g][j][e] = 0.f;
+        for (int e = 0; e < CP; ++e) o_acc[g][j][e] = 0ull;
     }
   }
 
@@ -382,18 +433,18 @@ struct Scanner {
     for (int ps = 0; ps < PASSES; ++ps) {
       const int row = warp * 8 + ps * RPP + rg;
       valid[ps] = slot0 + row < L;
-      float kf[NP][CH];
+      f32x2 kf[NP][CP];
 #pragma unroll
-      for (int j = 0; j < NP; ++j) load_chunk<CH>(tK + row * D + (l + LPR * j) * CH, kf[j]);
+      for (int j = 0; j < NP; ++j) load_pairs<CP>(tK + row * D + (l + LPR * j) * CH, kf[j]);
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         float pp[NP];
 #pragma unroll
         for (int j = 0; j < NP; ++j) {
-          float acc = 0.f;
+          f32x2 acc = 0ull;                                            // (even-channel chain, odd-channel chain)
 #pragma unroll
-          for (int e = 0; e < CH; ++e) acc = __fmaf_rn(qf[g][j][e], kf[j][e], acc);
-          pp[j] = acc;
+          for (int e = 0; e < CP; ++e) acc = fma2(qf[g][j][e], kf[j][e], acc);
+          pp[j] = __fadd_rn(lo_of(acc), hi_of(acc));
         }
         float acc = pp[0];
         if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
@@ -421,29 +472,31 @@ struct Scanner {
       const float m_new = fmaxf(m_run[g], mt);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
+      const f32x2 corr2 = pack2(corr, corr);
       m_run[g] = m_new;
       l_run[g] *= corr;
 #pragma unroll
       for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CH; ++e) o_acc[g][j][e] *= corr;
+        for (int e = 0; e < CP; ++e) o_acc[g][j][e] = mul2(o_acc[g][j][e], corr2);
 #pragma unroll
       for (int ps = 0; ps < PASSES; ++ps) sv[g][ps] = fast_exp2((sv[g][ps] - m_use) * kLog2e);   // now probabilities
     }
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
       const int row = warp * 8 + ps * RPP + rg;
-      float vf[NP][CH];
+      f32x2 vf[NP][CP];
 #pragma unroll
-      for (int j = 0; j < NP; ++j) load_chunk<CH>(tV + row * D + (l + LPR * j) * CH, vf[j]);
+      for (int j = 0; j < NP; ++j) load_pairs<CP>(tV + row * D + (l + LPR * j) * CH, vf[j]);
       if (valid[ps]) {
 #pragma unroll
         for (int g = 0; g < G; ++g) {
           l_run[g] += sv[g][ps];
+          const f32x2 p2 = pack2(sv[g][ps], sv[g][ps]);
 #pragma unroll
           for (int j = 0; j < NP; ++j)
 #pragma unroll
-            for (int e = 0; e < CH; ++e) o_acc[g][j][e] = fmaf(sv[g][ps], vf[j][e], o_acc[g][j][e]);
+            for (int e = 0; e < CP; ++e) o_acc[g][j][e] = fma2(p2, vf[j][e], o_acc[g][j][e]);
         }
       }
     }
@@ -465,12 +518,13 @@ struct Scanner {
         const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
         l_run[g] = l_run[g] * c_me + l_o * c_o;
         m_run[g] = m_new;
+        const f32x2 c_me2 = pack2(c_me, c_me), c_o2 = pack2(c_o, c_o);
 #pragma unroll
         for (int j = 0; j < NP; ++j)
 #pragma unroll
-          for (int e = 0; e < CH; ++e) {
-            const float o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
-            o_acc[g][j][e] = o_acc[g][j][e] * c_me + o_o * c_o;
+          for (int e = 0; e < CP; ++e) {
+            const f32x2 o_o = __shfl_xor_sync(0xffffffffu, o_acc[g][j][e], off);
+            o_acc[g][j][e] = fma2(o_acc[g][j][e], c_me2, mul2(o_o, c_o2));
           }
       }
       float* wp = warp_part + (warp * G + g) * (D + 2);
@@ -478,7 +532,10 @@ struct Scanner {
 #pragma unroll
         for (int j = 0; j < NP; ++j)
 #pragma unroll
-          for (int e = 0; e < CH; ++e) wp[2 + (l + LPR * j) * CH + e] = o_acc[g][j][e];
+          for (int e = 0; e < CP; ++e) {
+            wp[2 + (l + LPR * j) * CH + 2 * e] = lo_of(o_acc[g][j][e]);
+            wp[2 + (l + LPR * j) * CH + 2 * e + 1] = hi_of(o_acc[g][j][e]);
+          }
       }
       if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
     }
