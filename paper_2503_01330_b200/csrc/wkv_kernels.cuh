@@ -388,23 +388,35 @@ struct Scanner {
   static constexpr int CP = CH / 2;              // ... as (even, odd) channel pairs: the arithmetic is packed fp32x2
   static constexpr int RPP = 32 / LPR;           // rows per warp pass
   static constexpr int PASSES = 8 / RPP;
+  // With G query heads the butterfly is run as a reduce-scatter: each round with more than one head left halves the
+  // heads a thread carries, so a row's LPR threads end up owning one head each (LH threads per head) and the softmax
+  // bookkeeping is done once per head instead of once per thread.  The additions are those of the plain butterfly.
+  static constexpr int LH = LPR / G;             // threads per (row, head) after the reduce-scatter
+  static_assert(G <= LPR && LH >= 1, "at most one head per thread of a row");
   f32x2 qf[G][NP][CP];
-  float m_run[G], l_run[G];
+  float m_run, l_run;                            // online softmax of this thread's head: head_of(l) = l / LH
   f32x2 o_acc[G][NP][CP];
 
   __device__ __forceinline__ void begin(const T* q) {      // q: [G][D], 16-byte aligned (global or shared)
     const int l = (threadIdx.x & 31) % LPR;
+    m_run = -INFINITY;
+    l_run = 0.f;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
 #pragma unroll
       for (int j = 0; j < NP; ++j) load_pairs<CP>(q + g * D + (l + LPR * j) * CH, qf[g][j]);
-      m_run[g] = -INFINITY;
-      l_run[g] = 0.f;
 #pragma unroll
       for (int j = 0; j < NP; ++j)
 #pragma unroll
         for (int e = 0; e < CP; ++e) o_acc[g][j][e] = 0ull;
     }
+  }
+
+  // value of head g's owner threads, for every thread of the row group
+  __device__ __forceinline__ static float from_head(float mine, int g) {
+    if constexpr (G == 1) return mine;
+    const int lane_id = threadIdx.x & 31;
+    return __shfl_sync(0xffffffffu, mine, (lane_id & ~(LPR - 1)) | (g * LH));
   }
 
   // One tile of up to 32 rows starting at slot0; logits parked at logit_dst[g*logit_stride + slot - logit_off].
@@ -413,6 +425,7 @@ struct Scanner {
     const float kLog2e = 1.4426950408889634f;
     const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
     const int rg = lane_id / LPR, l = lane_id % LPR;
+    const int my_head = l / LH, li = l % LH;
     {
       // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
       // row in the tile with the token's k and v before anybody reads it.
@@ -427,7 +440,7 @@ struct Scanner {
         __syncwarp();
       }
     }
-    float sv[G][PASSES];
+    float sv[PASSES];                                                // logits of my head, one row per pass
     bool valid[PASSES];
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
@@ -436,6 +449,7 @@ struct Scanner {
       f32x2 kf[NP][CP];
 #pragma unroll
       for (int j = 0; j < NP; ++j) load_pairs<CP>(tK + row * D + (l + LPR * j) * CH, kf[j]);
+      float vals[G];
 #pragma unroll
       for (int g = 0; g < G; ++g) {
         float pp[NP];
@@ -446,41 +460,59 @@ struct Scanner {
           for (int e = 0; e < CP; ++e) acc = fma2(qf[g][j][e], kf[j][e], acc);
           pp[j] = __fadd_rn(lo_of(acc), hi_of(acc));
         }
-        float acc = pp[0];
-        if constexpr (NP == 2) acc = __fadd_rn(pp[0], pp[1]);        // butterfly round off = 8
+        vals[g] = pp[0];
+        if constexpr (NP == 2) vals[g] = __fadd_rn(pp[0], pp[1]);      // butterfly round off = 8
+      }
+      // butterfly rounds off = LPR/2 .. 1: p_r + p_{r^off}; while several heads are left, each partner keeps half
 #pragma unroll
-        for (int off = LPR / 2; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-        const float sc = __fmul_rn(scale, acc);
-        sv[g][ps] = valid[ps] ? sc : -INFINITY;
+      for (int off = LPR / 2, n = G; off >= 1; off >>= 1) {
+        if (n > 1) {
+          const bool upper = (l & off) != 0;
+#pragma unroll
+          for (int i = 0; i < n / 2; ++i) {
+            const float keep = upper ? vals[n / 2 + i] : vals[i];
+            const float send = upper ? vals[i] : vals[n / 2 + i];
+            vals[i] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, off));
+          }
+          n >>= 1;
+        } else {
+          vals[0] = __fadd_rn(vals[0], __shfl_xor_sync(0xffffffffu, vals[0], off));
+        }
+      }
+      const float sc = __fmul_rn(scale, vals[0]);
+      sv[ps] = valid[ps] ? sc : -INFINITY;
+    }
+    // park the logits of my head: thread li of the head's LH threads takes the passes ps with ps % LH == li
+#pragma unroll
+    for (int ps = 0; ps < PASSES; ++ps) {
+      const int slot = slot0 + warp * 8 + ps * RPP + rg;
+      if ((ps % LH) == li && slot < L) logit_dst[(long long)my_head * logit_stride + (slot - logit_off)] = sv[ps];
+    }
+    // online softmax update of my head, one rescale per tile
+    float corr;
+    {
+      float mt = sv[0];
+#pragma unroll
+      for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[ps]);
+      const float m_new = fmaxf(m_run, mt);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      corr = fast_exp2((m_run - m_use) * kLog2e);
+      m_run = m_new;
+      l_run *= corr;
+#pragma unroll
+      for (int ps = 0; ps < PASSES; ++ps) {
+        sv[ps] = fast_exp2((sv[ps] - m_use) * kLog2e);                 // now probabilities (0 for rows beyond L)
+        l_run += sv[ps];
       }
     }
-    // park the logits: thread l (< PASSES) of row group rg owns row warp*8 + l*RPP + rg
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-      float mine = sv[g][0];
-#pragma unroll
-      for (int ps = 1; ps < PASSES; ++ps) mine = l == ps ? sv[g][ps] : mine;
-      const int slot = slot0 + warp * 8 + l * RPP + rg;
-      if (l < PASSES && slot < L) logit_dst[(long long)g * logit_stride + (slot - logit_off)] = mine;
-    }
-    // online softmax update, one rescale per tile
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-      float mt = sv[g][0];
-#pragma unroll
-      for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[g][ps]);
-      const float m_new = fmaxf(m_run[g], mt);
-      const float m_use = m_new == -INFINITY ? 0.f : m_new;
-      const float corr = fast_exp2((m_run[g] - m_use) * kLog2e);
-      const f32x2 corr2 = pack2(corr, corr);
-      m_run[g] = m_new;
-      l_run[g] *= corr;
+      const float cg = from_head(corr, g);
+      const f32x2 corr2 = pack2(cg, cg);
 #pragma unroll
       for (int j = 0; j < NP; ++j)
 #pragma unroll
         for (int e = 0; e < CP; ++e) o_acc[g][j][e] = mul2(o_acc[g][j][e], corr2);
-#pragma unroll
-      for (int ps = 0; ps < PASSES; ++ps) sv[g][ps] = fast_exp2((sv[g][ps] - m_use) * kLog2e);   // now probabilities
     }
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
@@ -488,11 +520,13 @@ struct Scanner {
       f32x2 vf[NP][CP];
 #pragma unroll
       for (int j = 0; j < NP; ++j) load_pairs<CP>(tV + row * D + (l + LPR * j) * CH, vf[j]);
-      if (valid[ps]) {
+      float pg[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) pg[g] = from_head(sv[ps], g);
+      if (valid[ps]) {                                                 // rows beyond L hold stale bytes, possibly NaN
 #pragma unroll
         for (int g = 0; g < G; ++g) {
-          l_run[g] += sv[g][ps];
-          const f32x2 p2 = pack2(sv[g][ps], sv[g][ps]);
+          const f32x2 p2 = pack2(pg[g], pg[g]);
 #pragma unroll
           for (int j = 0; j < NP; ++j)
 #pragma unroll
@@ -507,18 +541,20 @@ struct Scanner {
     const float kLog2e = 1.4426950408889634f;
     const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
     const int rg = lane_id / LPR, l = lane_id % LPR;
+    const int my_head = l / LH, li = l % LH;
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
+    for (int off = 16; off >= LPR; off >>= 1) {
+      const float m_o = __shfl_xor_sync(0xffffffffu, m_run, off);     // same head on both sides
+      const float l_o = __shfl_xor_sync(0xffffffffu, l_run, off);
+      const float m_new = fmaxf(m_run, m_o);
+      const float m_use = m_new == -INFINITY ? 0.f : m_new;
+      const float c_me = fast_exp2((m_run - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
+      l_run = l_run * c_me + l_o * c_o;
+      m_run = m_new;
 #pragma unroll
-      for (int off = 16; off >= LPR; off >>= 1) {
-        const float m_o = __shfl_xor_sync(0xffffffffu, m_run[g], off);
-        const float l_o = __shfl_xor_sync(0xffffffffu, l_run[g], off);
-        const float m_new = fmaxf(m_run[g], m_o);
-        const float m_use = m_new == -INFINITY ? 0.f : m_new;
-        const float c_me = fast_exp2((m_run[g] - m_use) * kLog2e), c_o = fast_exp2((m_o - m_use) * kLog2e);
-        l_run[g] = l_run[g] * c_me + l_o * c_o;
-        m_run[g] = m_new;
-        const f32x2 c_me2 = pack2(c_me, c_me), c_o2 = pack2(c_o, c_o);
+      for (int g = 0; g < G; ++g) {
+        const float cm = from_head(c_me, g), co = from_head(c_o, g);
+        const f32x2 c_me2 = pack2(cm, cm), c_o2 = pack2(co, co);
 #pragma unroll
         for (int j = 0; j < NP; ++j)
 #pragma unroll
@@ -527,8 +563,11 @@ struct Scanner {
             o_acc[g][j][e] = fma2(o_acc[g][j][e], c_me2, mul2(o_o, c_o2));
           }
       }
-      float* wp = warp_part + (warp * G + g) * (D + 2);
-      if (rg == 0) {
+    }
+    if (rg == 0) {
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float* wp = warp_part + (warp * G + g) * (D + 2);
 #pragma unroll
         for (int j = 0; j < NP; ++j)
 #pragma unroll
@@ -537,7 +576,11 @@ struct Scanner {
             wp[2 + (l + LPR * j) * CH + 2 * e + 1] = hi_of(o_acc[g][j][e]);
           }
       }
-      if (lane_id == 0) { wp[0] = m_run[g]; wp[1] = l_run[g]; }
+      if (li == 0) {
+        float* wp = warp_part + (warp * G + my_head) * (D + 2);
+        wp[0] = m_run;
+        wp[1] = l_run;
+      }
     }
   }
 };
