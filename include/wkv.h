@@ -111,8 +111,9 @@ int wkv_decode_step(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, c
  *   q   device [n_layers, batch, n_q_heads, head_dim];  k, v device [n_layers, batch, n_kv_heads, head_dim]
  *   out device [n_layers, batch, n_q_heads, head_dim];  evicted_pos device [n_layers, batch, n_kv_heads] or NULL
  * By making this call the caller states that ALL layers' q, k, v are complete on the stream before it; the library
- * uses that to let each layer's cache scan run while the previous layer's per-lane epilogue is still finishing
- * (results are identical to n_layers separate calls).  Inputs must not overlap the outputs.  Asynchronous. */
+ * uses that to run the lanes of all layers in one launch when a layer alone is small, or else to let each layer's
+ * cache scan run while the previous layer's per-lane epilogue is still finishing (results are identical to n_layers
+ * separate calls).  Inputs must not overlap the outputs.  Asynchronous. */
 int wkv_decode_step_layers(wkv_ctx* ctx, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos);
 
 /* No counterpart in the paper: this entry point exists for callers that must not allocate device memory.

@@ -21,6 +21,11 @@ struct wkv_ctx {
   int n_splits = 1;
   int chunk_cap = 0;      // cluster kernel: logits per CTA and query head
   bool use_cluster = false;
+  // all layers of a step in one launch (wkv_decode_step_layers), when the scratch for every lane at once is small
+  bool fused_ok = false, fused_cluster = false;
+  int fused_splits = 1, fused_chunk_cap = 0;
+  float* fused_logits = nullptr;
+  float* fused_part = nullptr;
   int sm_count = 148;
   float scale = 0.f;
   size_t elem = 2;
@@ -115,8 +120,7 @@ const char* check_config(const wkv_config* c) {
 
 // Splits per lane when the caller leaves the choice to the library: a power of two (so the lane's CTAs can form a
 // thread-block cluster), enough CTAs to fill 148 SMs several times over, at least ~4 tiles of work per CTA.
-int auto_splits(const wkv_config& c) {
-  const int lanes = c.batch * c.n_kv_heads;
+int auto_splits(const wkv_config& c, long long lanes) {
   const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
   int s = 1;
   while (s < 16 && lanes * s < 1776 && tiles / (2 * s) >= 4) s *= 2;
@@ -207,8 +211,8 @@ cudaError_t launch_by_group(int G, const wkv::StepParams& P, int lanes, bool clu
 }
 
 // cluster = false forces the two-kernel schedule (global scratch), which the static-scratch entry point needs.
-cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P, bool cluster) {
-  const int n = c->lanes_per_layer;
+cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P, bool cluster, int lanes = 0) {
+  const int n = lanes > 0 ? lanes : c->lanes_per_layer;
   if (c->cfg.dtype == WKV_BF16) {
     return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n, cluster, c->stream)
                                   : launch_by_group<__nv_bfloat16, 64>(c->group, P, n, cluster, c->stream);
@@ -327,7 +331,7 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   c->lanes_per_layer = cfg->batch * cfg->n_kv_heads;
   c->lanes_total = (long long)cfg->n_layers * c->lanes_per_layer;
   c->cap = (cfg->budget + 1 + 3) & ~3;
-  c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg);
+  c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_per_layer);
   {
     const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
     c->chunk_cap = ((tiles + c->n_splits - 1) / c->n_splits) * wkv::kTileSlots;   // the largest share of an even deal
@@ -341,6 +345,18 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     // with short-lived CTAs, then finish the lanes in a second launch
     c->use_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ||
                      (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_per_layer * tiles < 148 * 64);
+  }
+  if (cfg->n_layers > 1 && c->lanes_total * wkv::kMaxSplits < 0x7fffffffLL) {
+    // One launch for all layers: the lanes of all layers are just more lanes.  Worth it when a layer alone cannot
+    // fill the GPU; allowed when the scratch for every lane at once stays small.
+    const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+    c->fused_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_total);
+    c->fused_chunk_cap = ((tiles + c->fused_splits - 1) / c->fused_splits) * wkv::kTileSlots;
+    const bool can_cluster = is_cluster_size(c->fused_splits) && c->group * c->fused_chunk_cap * 4 <= 64 * 1024;
+    c->fused_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ? can_cluster
+                       : (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_total * tiles < 148 * 64);
+    const size_t bytes = (size_t)c->lanes_total * c->group * ((size_t)c->cap * 4 + (size_t)c->fused_splits * (cfg->head_dim + 2) * 4);
+    c->fused_ok = bytes <= ((size_t)64 << 20) && (cfg->schedule != WKV_SCHEDULE_CLUSTER || can_cluster);
   }
   c->scale = cfg->scale != 0.f ? cfg->scale : (float)(1.0 / std::sqrt((double)cfg->head_dim));
   c->elem = cfg->dtype == WKV_BF16 ? 2 : 4;
@@ -360,6 +376,10 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   for (int i = 0; i < 2; ++i) {
     T(take(c, &c->logits[i], (size_t)c->lanes_per_layer * G * cap * 4));
     T(take(c, &c->part[i], (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
+  }
+  if (c->fused_ok) {
+    T(take(c, &c->fused_logits, (size_t)c->lanes_total * G * cap * 4));
+    T(take(c, &c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4));
   }
   T(take(c, &c->status, 256));
   T(take(c, &c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * row));
@@ -440,6 +460,26 @@ int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void*
       ranges_overlap(v, kv_bytes * nl, evicted_pos, (size_t)c->lanes_per_layer * 4 * nl))
     return fail(c, WKV_ERR_INVALID, "wkv_decode_step_layers: inputs and outputs must not overlap");
   c->last_layer = -1;                   // the first layer's scan orders itself behind whatever ran before this call
+  if (c->fused_ok) {
+    // the lanes of all layers in one launch (pair): [n_layers, batch, ...] is [n_layers*batch, ...] to the kernels
+    wkv::StepParams P = base_params(c, 0);
+    P.n_splits = c->fused_splits;
+    P.chunk_cap = c->fused_chunk_cap;
+    P.logits = c->fused_logits;
+    P.part = c->fused_part;
+    P.q = q; P.k = k; P.v = v; P.out = out; P.evicted = evicted_pos; P.probs = nullptr;
+    P.q_bs = (long long)c->cfg.n_q_heads * c->cfg.head_dim;
+    P.kv_bs = (long long)c->cfg.n_kv_heads * c->cfg.head_dim;
+    P.out_bs = P.q_bs;
+    P.ev_bs = c->cfg.n_kv_heads;
+    P.wait_at_start = 2;
+    g_last_launcher.store(c);
+    cudaError_t e = launch_any(c, P, c->fused_cluster, (int)c->lanes_total);
+    c->launches += c->fused_cluster ? 1 : 2;
+    if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (all layers)");
+    note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+    return WKV_OK;
+  }
   for (int layer = 0; layer < c->cfg.n_layers; ++layer) {
     int rc = decode_step_impl(c, layer, (const char*)q + layer * q_bytes, (const char*)k + layer * kv_bytes,
                               (const char*)v + layer * kv_bytes, (char*)out + layer * q_bytes,

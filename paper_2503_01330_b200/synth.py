@@ -66,6 +66,12 @@ WORKLOADS = {
     # serving batch, ragged prefill lengths
     "serving_b16": Workload("serving_b16", 32, 16, 32, 32, 128, "bf16", 4096, 128, 0, 16384, 8192, 512, 16, 0.05,
                             False),
+    # the paper's own cache settings (Experiments section): 4 initial tokens kept, cache 1024 with 508 recent tokens
+    # and cache 256 with 124 recent tokens, Llama-2-7B KV shape, one sequence, 4k context
+    "paper_cache1024": Workload("paper_cache1024", 32, 1, 32, 32, 128, "bf16", 1024, 508, 4, 4096, 4096, 512, 16, 0.05,
+                                False),
+    "paper_cache256": Workload("paper_cache256", 32, 1, 32, 32, 128, "bf16", 256, 124, 4, 4096, 4096, 512, 16, 0.05,
+                               False),
     # grouped-query variant: 32 query heads share 8 kv heads
     "gqa_b32": Workload("gqa_b32", 32, 32, 32, 8, 128, "bf16", 3277, 128, 0, 32768, 32768, 512, 16, 0.05, False),
 }

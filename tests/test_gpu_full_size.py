@@ -32,3 +32,20 @@ def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     assert p.n_evictions >= len(p.lanes) * (100 + decode)
     p.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["paper_cache1024", "paper_cache256"])
+def test_paper_cache_settings(name):
+    """The cache settings of the paper's Experiments section (4 initial tokens kept, 1024 / 508 recent and 256 / 124
+    recent), Llama-2-7B KV shape: streamed prompt, per-layer decode calls and the all-layers call (one launch)."""
+    wl = WORKLOADS[name]
+    p = Parity(wl, sample=16, ragged=[wl.budget + 300])
+    p.prefill(wl.budget + 300, chunk=64)
+    p.compare_state()
+    p.decode(16)
+    p.decode(48, layers_entry=True)
+    p.decode(8)
+    p.compare_state()
+    for ln in p.lanes:                                     # the four initial tokens are never removed
+        assert p.ctx.wkv_export_state(*ln)["pos"][:4].tolist() == [0, 1, 2, 3]
+    p.close()
