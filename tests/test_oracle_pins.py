@@ -517,3 +517,31 @@ def test_pinned_mode_tracks_double_mode(dtype):
         np.testing.assert_allclose(sp["a"], sd["a"], rtol=1e-5, atol=1e-7)
         tol = 2 ** -7 if dtype == BF16 else 1e-5
         np.testing.assert_allclose(sp["V"], sd["V"], rtol=tol, atol=tol)
+
+
+# ---------------------------------------------------------------------------------------------
+# the Ideal Merging section: the closed form really leaves the output unchanged; its two-term cut is convex
+# ---------------------------------------------------------------------------------------------
+def test_ideal_merge_identity_and_convex_approximation():
+    from oracle.diagnostics import attention_output, ideal_merged_value, instant_convex_merge
+    rng = np.random.default_rng(42)
+    for t, d in ((3, 8), (17, 16), (200, 64)):
+        q = rng.standard_normal(d)
+        K = rng.standard_normal((t, d))
+        V = rng.standard_normal((t, d))
+        scale = 1 / math.sqrt(d)
+        full = attention_output(q, K, V, scale)
+        v_ideal = ideal_merged_value(q, K, V, scale)
+        merged = attention_output(q, K[1:], np.vstack([v_ideal, V[2:]]), scale)      # k1 dropped, k2 kept
+        np.testing.assert_allclose(merged, full, rtol=1e-11, atol=1e-12)
+        v_cvx, w = instant_convex_merge(q, K, V, scale)
+        assert (w >= 0).all() and abs(w.sum() - 1) < 1e-15
+        assert (v_cvx <= np.maximum(V[0], V[1]) + 1e-15).all() and (v_cvx >= np.minimum(V[0], V[1]) - 1e-15).all()
+        # dropping the v3.. terms and renormalising the remaining two coefficients gives exactly the convex form
+        s = scale * (K @ q)
+        c1, c2 = math.exp(s[0] - s[1]), 1.0
+        np.testing.assert_allclose(v_cvx, (c1 * V[0] + c2 * V[1]) / (c1 + c2), rtol=1e-12)
+    # with a single further token of negligible weight the ideal value is the convex one (here: the plain mean)
+    q = np.zeros(4); K = np.zeros((3, 4)); K[2, 0] = -200.0; q[0] = 1.0
+    V = rng.standard_normal((3, 4))
+    np.testing.assert_allclose(ideal_merged_value(q, K, V, 1.0), 0.5 * (V[0] + V[1]), atol=1e-12)
