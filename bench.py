@@ -300,16 +300,14 @@ def main():
     host = [tuple(x.cpu().pin_memory() for x in toks[args.warmup + i]) for i in range(n_e2e)]
     out_h = torch.empty(out.shape, dtype=out.dtype).pin_memory()
     ev_h = torch.empty(ev.shape, dtype=ev.dtype).pin_memory()
-    for layer in range(wl.n_layers):                                   # warm the path once
-        ctx.wkv_decode_step_host(layer, host[0][0][layer], host[0][1][layer], host[0][2][layer], out_h[layer], ev_h[layer])
+    ctx.wkv_decode_step_layers_host(host[0][0], host[0][1], host[0][2], out_h, ev_h)       # warm the path once
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h0.record()
     for q, k, v in host:
-        for layer in range(wl.n_layers):
-            ctx.wkv_decode_step_host(layer, q[layer], k[layer], v[layer], out_h[layer], ev_h[layer])
+        ctx.wkv_decode_step_layers_host(q, k, v, out_h, ev_h)    # copies in, all layers, copies out, stream wait
     h1.record()
     torch.cuda.synchronize()
     e2e_ms = h0.elapsed_time(h1)
@@ -345,7 +343,7 @@ def main():
                          else "decode_step_cluster_kernel",
                          "algorithmic_bytes_per_launch": bytes_launch, "launch_ms": launch_ms},
             "e2e": {"value": e2e_value, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "steps": n_e2e}}
+                    "steps": n_e2e, "call": "wkv_decode_step_layers_host: one call per step from pinned host buffers"}}
     if not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         n_lanes, n_steps = cores, 8

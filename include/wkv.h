@@ -148,6 +148,11 @@ int wkv_decode_step_static(wkv_ctx* ctx, int32_t layer, const void* q, const voi
 int wkv_decode_step_host(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
                          int32_t* evicted_pos);
 
+/* wkv_decode_step_layers from HOST buffers (shapes as there, all layers of one step): three copies in, the step, two
+ * copies out, then waits for the stream. */
+int wkv_decode_step_layers_host(wkv_ctx* ctx, const void* q, const void* k, const void* v, void* out,
+                                int32_t* evicted_pos);
+
 /* Consumes a prompt exactly as Algorithm 1 does: token by token, compressing as soon as a lane exceeds
  * the budget (the algorithm has no separate prompt phase).  One kernel launch per token, asynchronous.
  *   Q    device [batch, T_max, n_q_heads, head_dim], K, V device [batch, T_max, n_kv_heads, head_dim]
@@ -178,6 +183,13 @@ int wkv_import_state(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, in
 /* Reads and clears the device status word (waits for the stream): WKV_OK, or WKV_ERR_TIMEOUT if a bounded
  * wait inside a kernel gave up since the last call. */
 int wkv_status(wkv_ctx* ctx);
+
+/* Self-test of the error path for device-side waits.  Every wait inside the kernels (on a shared-memory barrier fed
+ * by a bulk copy) is bounded: after a fixed number of polls the waiting thread sets a bit in the device status word
+ * and carries on, so a kernel always terminates.  This call launches a one-thread kernel that waits on a barrier
+ * nothing will complete (20000 polls, a few milliseconds); afterwards wkv_status returns WKV_ERR_TIMEOUT once and the
+ * context is as usable as before.  Nothing faults or hangs.  Asynchronous. */
+int wkv_selftest_wait_timeout(wkv_ctx* ctx);
 
 /* Number of kernels this context has launched so far, and bytes it obtained from the provider. */
 int64_t wkv_launch_count(const wkv_ctx* ctx);

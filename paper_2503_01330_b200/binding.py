@@ -29,8 +29,8 @@ class wkv_config(C.Structure):
 
 
 EXPORTS = ["wkv_config_error", "wkv_create", "wkv_destroy", "wkv_reset", "wkv_set_stream", "wkv_decode_step",
-           "wkv_decode_step_layers", "wkv_decode_step_static", "wkv_decode_step_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
-           "wkv_status", "wkv_launch_count", "wkv_device_bytes", "wkv_splits", "wkv_strerror", "wkv_last_error"]
+           "wkv_decode_step_layers", "wkv_decode_step_static", "wkv_decode_step_host", "wkv_decode_step_layers_host", "wkv_prefill", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
+           "wkv_status", "wkv_selftest_wait_timeout", "wkv_launch_count", "wkv_device_bytes", "wkv_splits", "wkv_strerror", "wkv_last_error"]
 
 _lib = None
 
@@ -54,11 +54,13 @@ def lib():
         L.wkv_decode_step_layers.argtypes = [vp, vp, vp, vp, vp, vp]
         L.wkv_decode_step_static.argtypes = [vp, i32, vp, vp, vp, vp, vp]
         L.wkv_decode_step_host.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+        L.wkv_decode_step_layers_host.argtypes = [vp, vp, vp, vp, vp, vp]
         L.wkv_prefill.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp]
         L.wkv_export_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.wkv_export_slots.argtypes = [vp, i32, i32, i32, vp]
         L.wkv_import_state.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.wkv_status.argtypes = [vp]
+        L.wkv_selftest_wait_timeout.argtypes = [vp]
         L.wkv_launch_count.restype = C.c_int64
         L.wkv_launch_count.argtypes = [vp]
         L.wkv_device_bytes.restype = C.c_int64
@@ -180,6 +182,9 @@ class Context:
     def wkv_decode_step_host(self, layer, q, k, v, out, evicted_pos=None):
         self._check(lib().wkv_decode_step_host(self._h, layer, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos)))
 
+    def wkv_decode_step_layers_host(self, q, k, v, out, evicted_pos=None):
+        self._check(lib().wkv_decode_step_layers_host(self._h, _dp(q), _dp(k), _dp(v), _dp(out), _dp(evicted_pos)))
+
     def wkv_prefill(self, layer, Q, K, V, seq_lens=None, out=None, evicted_pos=None):
         T_max = Q.shape[1]
         self._check(lib().wkv_prefill(self._h, layer, _dp(Q), _dp(K), _dp(V), _dp(seq_lens), T_max, _dp(out),
@@ -213,6 +218,9 @@ class Context:
 
     def wkv_status(self):
         return lib().wkv_status(self._h)
+
+    def wkv_selftest_wait_timeout(self):
+        self._check(lib().wkv_selftest_wait_timeout(self._h))
 
     def wkv_launch_count(self):
         return int(lib().wkv_launch_count(self._h))

@@ -382,11 +382,12 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     T(take(c, &c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4));
   }
   T(take(c, &c->status, 256));
-  T(take(c, &c->stage_q, (size_t)cfg->batch * cfg->n_q_heads * row));
-  T(take(c, &c->stage_k, (size_t)c->lanes_per_layer * row));
-  T(take(c, &c->stage_v, (size_t)c->lanes_per_layer * row));
-  T(take(c, &c->stage_out, (size_t)cfg->batch * cfg->n_q_heads * row));
-  T(take(c, &c->stage_ev, (size_t)c->lanes_per_layer * 4));
+  // staging holds one step of all layers (the host entry points copy through it)
+  T(take(c, &c->stage_q, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row));
+  T(take(c, &c->stage_k, (size_t)c->lanes_total * row));
+  T(take(c, &c->stage_v, (size_t)c->lanes_total * row));
+  T(take(c, &c->stage_out, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row));
+  T(take(c, &c->stage_ev, (size_t)c->lanes_total * 4));
   if (rc == WKV_OK) rc = run_reset(c);
   if (rc != WKV_OK) {
     wkv_destroy(c);
@@ -546,6 +547,23 @@ int wkv_decode_step_host(wkv_ctx* c, int32_t layer, const void* q, const void* k
   return WKV_OK;
 }
 
+int wkv_decode_step_layers_host(wkv_ctx* c, const void* q, const void* k, const void* v, void* out, int32_t* evicted_pos) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!q || !k || !v || !out) return fail(c, WKV_ERR_INVALID, "q, k, v and out must not be NULL");
+  const size_t row = (size_t)c->cfg.head_dim * c->elem;
+  const size_t qb = (size_t)c->cfg.n_layers * c->cfg.batch * c->cfg.n_q_heads * row, kb = (size_t)c->lanes_total * row;
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_q, q, qb, cudaMemcpyHostToDevice, c->stream));
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_k, k, kb, cudaMemcpyHostToDevice, c->stream));
+  WKV_CUDA(c, cudaMemcpyAsync(c->stage_v, v, kb, cudaMemcpyHostToDevice, c->stream));
+  int rc = wkv_decode_step_layers(c, c->stage_q, c->stage_k, c->stage_v, c->stage_out, c->stage_ev);
+  if (rc != WKV_OK) return rc;
+  WKV_CUDA(c, cudaMemcpyAsync(out, c->stage_out, qb, cudaMemcpyDeviceToHost, c->stream));
+  if (evicted_pos)
+    WKV_CUDA(c, cudaMemcpyAsync(evicted_pos, c->stage_ev, (size_t)c->lanes_total * 4, cudaMemcpyDeviceToHost, c->stream));
+  WKV_CUDA(c, cudaStreamSynchronize(c->stream));
+  return WKV_OK;
+}
+
 int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                 int32_t T_max, void* out, int32_t* evicted_pos) {
   if (!c) return WKV_ERR_INVALID;
@@ -671,6 +689,15 @@ int wkv_status(wkv_ctx* c) {
     if (w & wkv::kStatusWaitTimeout) return fail(c, WKV_ERR_TIMEOUT, "a bounded wait inside a kernel gave up");
     return fail(c, WKV_ERR_STATE, "a kernel found inconsistent slot links");
   }
+  return WKV_OK;
+}
+
+int wkv_selftest_wait_timeout(wkv_ctx* c) {
+  if (!c) return WKV_ERR_INVALID;
+  wkv::wait_selftest_kernel<<<1, 32, 0, c->stream>>>(c->status, 20000u);
+  c->launches++;
+  c->last_layer = -1;
+  WKV_CUDA(c, cudaGetLastError());
   return WKV_OK;
 }
 

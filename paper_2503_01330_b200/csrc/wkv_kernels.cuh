@@ -111,9 +111,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls, records it in the status word and returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+// Bounded wait: gives up after `limit` polls, records it in the status word and returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status, uint32_t limit = kSpinLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 64) __nanosleep(64);
   }
@@ -1167,6 +1167,17 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
   cluster.sync();                                       // #4: nobody's shared memory is needed any more
   if (split != 0) return;
   finish_lane<T, D, G, NT>(P, v, sm.ep, compress, sm.ep.u64[89], sm.ep.i32[4]);
+}
+
+// Exercises the give-up path of the bounded wait without any fault: one thread waits on an mbarrier that nothing
+// will ever complete, runs out of polls, records that in the status word, and the kernel ends normally.
+__global__ void wait_selftest_kernel(uint32_t* status, uint32_t polls) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_wait(&bar, 0, status, polls);
+  }
 }
 
 // Clears a context: every lane empty, chain heads/tails unset, slot 0 free.

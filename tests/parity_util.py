@@ -116,8 +116,11 @@ class Parity:
                 qh, kh, vh = (x.cpu().pin_memory() for x in (q, k, v))
                 oh = torch.empty_like(self.out, device="cpu").pin_memory()
                 eh = torch.empty_like(self.ev, device="cpu").pin_memory()
-                for layer in range(wl.n_layers):
-                    self.ctx.wkv_decode_step_host(layer, qh[layer], kh[layer], vh[layer], oh[layer], eh[layer])
+                if layers_entry:
+                    self.ctx.wkv_decode_step_layers_host(qh, kh, vh, oh, eh)
+                else:
+                    for layer in range(wl.n_layers):
+                        self.ctx.wkv_decode_step_host(layer, qh[layer], kh[layer], vh[layer], oh[layer], eh[layer])
                 self.out.copy_(oh)
                 self.ev.copy_(eh)
             elif layers_entry:

@@ -101,6 +101,7 @@ def test_host_buffer_entry_point():
     p = Parity(wl, seed=6)
     p.decode(30)
     p.decode(60, host_entry=True)
+    p.decode(20, host_entry=True, layers_entry=True)
     p.compare_state()
     p.close()
 
@@ -150,6 +151,19 @@ def test_large_budget_is_full_attention():
         want = torch.einsum("bht,bhtd->bhd", att, V)
         assert_close(p.out[0].cpu().numpy(), want.cpu().numpy(), "f32", f"full attention step {t}")
         assert (p.ev == -1).all()
+    p.close()
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing completes runs out of polls: the status word says so, once, and decoding goes on."""
+    wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=12, W=2)
+    p = Parity(wl, seed=2)
+    p.decode(20)
+    p.ctx.wkv_selftest_wait_timeout()
+    assert p.ctx.wkv_status() == binding.WKV_ERR_TIMEOUT
+    assert p.ctx.wkv_status() == binding.WKV_OK          # reading clears it
+    p.decode(20)                                         # same context, still in step with the oracle
+    p.compare_state()
     p.close()
 
 
