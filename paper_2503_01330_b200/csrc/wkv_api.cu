@@ -40,6 +40,8 @@ struct wkv_ctx {
   int32_t* lane_state = nullptr;
   float* logits[2] = {nullptr, nullptr};   // two scratch sets: consecutive layer calls may overlap (see prepare_overlap)
   float* part[2] = {nullptr, nullptr};
+  uint32_t* ticket[2] = {nullptr, nullptr};
+  uint32_t* fused_ticket = nullptr;
   int parity = 0;
   // what the previous layer call of this context wrote for the caller, and for which layer
   int last_layer = -1;
@@ -257,6 +259,7 @@ void prepare_overlap(wkv_ctx* c, wkv::StepParams& P, int layer, size_t q_bytes, 
   c->parity ^= 1;
   P.logits = c->logits[c->parity];
   P.part = c->part[c->parity];
+  P.ticket = c->ticket[c->parity];
   // 2: the previous kernel may touch this layer's lanes or is unknown; 1: it cannot, but it may be what produces this
   // call's inputs; 0: the caller vouches for the inputs and they do not alias the previous call's outputs.
   int level = (c->last_layer < 0 || c->last_layer == layer || g_last_launcher.load() != c) ? 2 : (inputs_ready ? 0 : 1);
@@ -279,6 +282,8 @@ void note_outputs(wkv_ctx* c, const void* out, size_t out_bytes, const void* ev,
 }
 
 int run_reset(wkv_ctx* c) {
+  for (int i = 0; i < 2; ++i) WKV_CUDA(c, cudaMemsetAsync(c->ticket[i], 0, (size_t)c->lanes_per_layer * 4, c->stream));
+  if (c->fused_ticket) WKV_CUDA(c, cudaMemsetAsync(c->fused_ticket, 0, (size_t)c->lanes_total * 4, c->stream));
   wkv::reset_kernel<<<592, 256, 0, c->stream>>>(c->lane_state, c->pos, c->a, c->next, c->prev, c->lanes_total, c->cap,
                                                 c->status);
   c->launches++;
@@ -376,10 +381,12 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   for (int i = 0; i < 2; ++i) {
     T(take(c, &c->logits[i], (size_t)c->lanes_per_layer * G * cap * 4));
     T(take(c, &c->part[i], (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
+    T(take(c, &c->ticket[i], (size_t)c->lanes_per_layer * 4));
   }
   if (c->fused_ok) {
     T(take(c, &c->fused_logits, (size_t)c->lanes_total * G * cap * 4));
     T(take(c, &c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4));
+    T(take(c, &c->fused_ticket, (size_t)c->lanes_total * 4));
   }
   T(take(c, &c->status, 256));
   // staging holds one step of all layers (the host entry points copy through it)
@@ -468,6 +475,7 @@ int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void*
     P.chunk_cap = c->fused_chunk_cap;
     P.logits = c->fused_logits;
     P.part = c->fused_part;
+    P.ticket = c->fused_ticket;
     P.q = q; P.k = k; P.v = v; P.out = out; P.evicted = evicted_pos; P.probs = nullptr;
     P.q_bs = (long long)c->cfg.n_q_heads * c->cfg.head_dim;
     P.kv_bs = (long long)c->cfg.n_kv_heads * c->cfg.head_dim;

@@ -65,6 +65,7 @@ struct StepParams {
   int32_t* lane_state;   // [lanes_total][LS_STRIDE]
   float* logits;         // scratch [lanes_per_layer*G][cap]
   float* part;           // scratch [lanes_per_layer][n_splits][G][D+2] : m, l, o[D]
+  uint32_t* ticket;      // scratch [lanes_per_layer] or nullptr: units of the lane whose scan is finished (zero between calls)
   uint32_t* status;      // device status word
   const void* q;         // [B][..][Hq][D]   batch stride q_bs elements
   const void* k;         // [B][..][Hkv][D]  batch stride kv_bs elements
@@ -967,6 +968,14 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
   }
   __syncthreads();
   combine_warps<D, G, NT>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
+  if (P.ticket != nullptr) {
+    // tell the lane's epilogue CTA (already resident in the next kernel, or not yet) that this unit is in scratch
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();                                   // release: the barrier ordered every thread's stores before it
+      atomicAdd(&P.ticket[lane_local], 1u);
+    }
+  }
   if (!P.wait_at_start) griddep_wait();
 }
 
@@ -991,13 +1000,41 @@ __global__ void __launch_bounds__(kEpilogueThreads) lane_epilogue_kernel(const S
     v.new_k = v.Kl + (long long)v.new_slot * D;          // the scan kernel has stored this step's token in the cache
     v.new_v = v.Vl + (long long)v.new_slot * D;
   }
-  griddep_wait();                                        // the scan is complete: logits and partials are visible
-  griddep_launch();                                      // the next kernel in the stream may be set up alongside
-  if (!active) {
-    if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
-    return;
+  // When is the lane's scan in scratch?  Without tickets: when the whole scan kernel has completed.  With tickets: as
+  // soon as the lane's own n_splits units have reported -- this kernel's CTAs become resident only after every CTA of
+  // the scan has started (that is the launch condition), so the units being waited for are running or done and never
+  // depend on this kernel; the wait is bounded all the same.
+  if (P.ticket == nullptr || !active) {
+    griddep_wait();
+    griddep_launch();
+    if (!active) {
+      if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
+      return;
+    }
+  } else {
+    if (threadIdx.x == 0) {
+      volatile uint32_t* tk = P.ticket + lane_local;
+      int ok = 0;
+      for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (*tk >= (uint32_t)P.n_splits) { ok = 1; break; }
+        __nanosleep(100);
+      }
+      if (!ok) atomicOr(P.status, kStatusWaitTimeout);
+      __threadfence();                                   // acquire side of the units' release
+      ep.i32[5] = ok;
+    }
+    __syncthreads();
+    griddep_launch();                                    // the next kernel in the stream may be set up alongside
+    if (!ep.i32[5]) {                                    // gave up: leave the lane untouched, the status word says so
+      griddep_wait();
+      return;
+    }
   }
   lane_epilogue_from_scratch<T, D, G, kEpilogueThreads>(P, v, ep);
+  if (P.ticket != nullptr) {
+    if (threadIdx.x == 0) P.ticket[lane_local] = 0u;     // ready for the next call that uses this scratch set
+    griddep_wait();                                      // keeps "this grid complete => the scan complete" literally true
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
