@@ -346,10 +346,11 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
       delete c;
       return WKV_ERR_INVALID;
     }
-    // few lanes: latency matters, one launch and a cluster sharing the lane's epilogue; many lanes: scan all units
-    // with short-lived CTAs, then finish the lanes in a second launch
+    // a handful of lanes: latency is everything, one launch and a cluster sharing the lane's epilogue (measured:
+    // 10.8 vs 14.2 us per step on 4 lanes x 5 tiles); otherwise scan all units with short-lived CTAs and finish the
+    // lanes in a second launch (17.4 vs 18.4 us on 32 lanes x 65 tiles, and far ahead on large shapes)
     c->use_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ||
-                     (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_per_layer * tiles < 148 * 64);
+                     (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_per_layer * tiles < 148 * 4);
   }
   if (cfg->n_layers > 1 && c->lanes_total * wkv::kMaxSplits < 0x7fffffffLL) {
     // One launch for all layers: the lanes of all layers are just more lanes.  Worth it when a layer alone cannot
@@ -359,7 +360,7 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     c->fused_chunk_cap = ((tiles + c->fused_splits - 1) / c->fused_splits) * wkv::kTileSlots;
     const bool can_cluster = is_cluster_size(c->fused_splits) && c->group * c->fused_chunk_cap * 4 <= 64 * 1024;
     c->fused_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ? can_cluster
-                       : (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_total * tiles < 148 * 64);
+                       : (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_total * tiles < 148 * 4);
     const size_t bytes = (size_t)c->lanes_total * c->group * ((size_t)c->cap * 4 + (size_t)c->fused_splits * (cfg->head_dim + 2) * 4);
     c->fused_ok = bytes <= ((size_t)64 << 20) && (cfg->schedule != WKV_SCHEDULE_CLUSTER || can_cluster);
   }
