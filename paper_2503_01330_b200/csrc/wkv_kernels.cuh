@@ -506,14 +506,17 @@ struct Scanner {
         l_run += sv[ps];
       }
     }
+    // the running maxima settle after a few tiles: rescale the output accumulators only when some head's maximum moved
+    if (__any_sync(0xffffffffu, corr != 1.0f)) {
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      const float cg = from_head(corr, g);
-      const f32x2 corr2 = pack2(cg, cg);
+      for (int g = 0; g < G; ++g) {
+        const float cg = from_head(corr, g);
+        const f32x2 corr2 = pack2(cg, cg);
 #pragma unroll
-      for (int j = 0; j < NP; ++j)
+        for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CP; ++e) o_acc[g][j][e] = mul2(o_acc[g][j][e], corr2);
+          for (int e = 0; e < CP; ++e) o_acc[g][j][e] = mul2(o_acc[g][j][e], corr2);
+      }
     }
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
