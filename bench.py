@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090744000 + 26963000 + 14383000, "e2e03d96b85b4c92")}
+NCU_TRAFFIC = {"serving_b16": (1090291000 + 26968000 + 13558000, "2eaa22dea7b78f4e")}
 
 
 def kernel_source_hash() -> str:
