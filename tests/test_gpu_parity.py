@@ -183,14 +183,33 @@ def test_argument_errors_leave_context_usable():
     ctx.close()
 
 
-@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_AUTO, binding.WKV_SCHEDULE_SPLIT])
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_AUTO, binding.WKV_SCHEDULE_CLUSTER])
 def test_llama7b_layer_config_all_lanes(schedule):
-    """One Llama-2-7B-shaped layer (32 heads x 128, bf16, budget 2048, window 64): every lane, every step of a
-    prefill that fills the cache and runs 300 compressions, then 64 decode steps."""
+    """One Llama-2-7B-shaped layer at its full size (32 heads x 128, bf16, budget 2048, window 64): prefill 4096,
+    1024 decode steps, every lane, every step -- 3072 compressions per lane, about 10^5 bit-exact picks in all."""
     wl = WORKLOADS["llama7b_layer"]
     p = Parity(wl, schedule=schedule)
-    p.prefill(wl.budget + 300, chunk=128)
-    p.decode(64)
-    mism = p.compare_state()
-    assert p.n_evictions == wl.lanes * 364
+    p.prefill(wl.prefill, chunk=128)
+    p.compare_state()
+    p.decode(wl.decode)
+    p.compare_state()
+    assert p.n_evictions == wl.lanes * (wl.prefill + wl.decode - wl.budget)
     p.close()
+
+
+def test_two_contexts_interleaved_on_one_stream():
+    """Calls of two contexts alternate on the same stream; each must stay in step with its own oracle (the library
+    may overlap consecutive launches of ONE context, never across contexts)."""
+    wa = small(layers=3, batch=2, d=128, dtype="bf16", m=60, W=4, rank=16)
+    wb = small(layers=2, batch=3, hq=4, hkv=2, d=64, dtype="f32", m=45, W=3)
+    pa = Parity(wa, seed=31, schedule=binding.WKV_SCHEDULE_SPLIT, n_splits=2)
+    pb = Parity(wb, seed=32, schedule=binding.WKV_SCHEDULE_SPLIT, n_splits=3)
+    for _ in range(12):
+        pa.decode(5, layers_entry=True)
+        pb.decode(4)
+        pa.decode(3)
+        pb.decode(4, layers_entry=True)
+    pa.compare_state()
+    pb.compare_state()
+    pa.close()
+    pb.close()
