@@ -121,6 +121,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
   atomicOr(status, kStatusWaitTimeout);
   return false;
 }
+// A consumer warp hands a ring stage back to the producer.  The fence puts every lane's reads of the stage ahead of
+// lane 0's arrival whatever instruction did the reading: with fragment loads (ldmatrix) in place of plain loads, the
+// reads of a tile's last channels were observed behind the arrival, picking up the tile that the producer put there next.
+__device__ __forceinline__ void release_stage(uint64_t* empty_bar) {
+  __threadfence_block();
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) mbar_arrive(empty_bar);
+}
 // Bulk asynchronous copy global -> this CTA's shared memory, completion counted in bytes on an mbarrier.
 // dst, src 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -964,8 +972,7 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
       T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
       T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
       sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, lg, P.cap, 0);
-      __syncwarp();
-      if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
+      release_stage(&sm.empty_bar[s]);
     }
     sc.end(sm.warp_part);
   }
@@ -1125,8 +1132,7 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
       T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
       sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, sm.chunk_logits,
               P.chunk_cap, v.slot_begin);
-      __syncwarp();
-      if (lane_id == 0) mbar_arrive(&sm.empty_bar[s]);
+      release_stage(&sm.empty_bar[s]);
     }
     sc.end(sm.warp_part);
   }

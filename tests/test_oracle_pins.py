@@ -545,3 +545,28 @@ def test_ideal_merge_identity_and_convex_approximation():
     q = np.zeros(4); K = np.zeros((3, 4)); K[2, 0] = -200.0; q[0] = 1.0
     V = rng.standard_normal((3, 4))
     np.testing.assert_allclose(ideal_merged_value(q, K, V, 1.0), 0.5 * (V[0] + V[1]), atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# the paper's ablation (WeightedKV against plain eviction with the same picks) on synthetic streams: error of the
+# outputs against full attention.  Direction only -- the paper's own numbers are perplexities of a trained model.
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("rho", [0.0, 0.5])
+def test_merging_loses_less_than_eviction_on_synthetic_streams(rho):
+    from oracle.diagnostics import compression_output_error
+    rng = np.random.default_rng(7)
+    T, n, G, d, r = 320, 8, 1, 32, 8
+    basis = rng.standard_normal((n, d, r))
+    K = np.einsum("ndr,tnr->tnd", basis, rng.standard_normal((T, n, r))) / math.sqrt(r) + 0.05 * rng.standard_normal((T, n, d))
+    Q = rng.standard_normal((T, n, G, d))
+    noise = rng.standard_normal((T, n, d))
+    V = np.zeros((T, n, d))
+    V[0] = noise[0]
+    for t in range(1, T):                               # values drift slowly for rho near 1, independent for rho = 0
+        V[t] = rho * V[t - 1] + math.sqrt(1 - rho * rho) * noise[t]
+    Q, K, V = (x.astype(np.float32) for x in (Q, K, V))
+    for m, W in ((64, 8), (128, 16)):
+        e_merge, n1 = compression_output_error(Q, K, V, m, W, merge=1)
+        e_evict, n0 = compression_output_error(Q, K, V, m, W, merge=0)
+        assert n1 == n0 == n * (T - m)                  # same trigger; the ablation changes only what happens to the value
+        assert e_merge < 0.97 * e_evict, (rho, m, e_merge, e_evict)
