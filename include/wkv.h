@@ -162,6 +162,19 @@ int wkv_decode_step_layers_host(wkv_ctx* ctx, const void* q, const void* k, cons
 int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                 int32_t T_max, void* out, int32_t* evicted_pos);
 
+/* The same prompt, same arguments and same results as wkv_prefill, with the uncompressed start of the prompt done as
+ * one dense problem per lane.  Algorithm 1 compresses only once a lane holds more than `budget` entries, so its first
+ * min(T_max, budget) iterations are causal attention (Background section) plus the running sums of the attention
+ * columns; when no lane of the layer has consumed a token since wkv_create / wkv_reset, one kernel computes those
+ * iterations for all lanes of the layer (every logit, probability and accumulated score with the arithmetic of the
+ * streamed step, scores added in the order of the tokens), and the remaining tokens are streamed as in wkv_prefill.
+ * If the layer is not empty the whole prompt is streamed.  K, positions, accumulated scores and removed positions are
+ * bit-identical to wkv_prefill's; outputs and merged values agree within rounding.
+ * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider and
+ * keeps them until wkv_destroy.  Q, K, V, out must be 16-byte aligned.  Asynchronous. */
+int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                     int32_t T_max, void* out, int32_t* evicted_pos);
+
 /* Copies one lane to HOST memory in position order and checks its bookkeeping (links form one chain of
  * `len` entries with strictly increasing positions); waits for the stream.  Any destination may be NULL.
  *   len, tokens : entries held / tokens consumed so far

@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/wkv.h: configuration checks, device state, launches,
 // export / import of lanes.  All arithmetic of the method lives in wkv_kernels.cuh.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -10,6 +11,7 @@
 
 #include "../../include/wkv.h"
 #include "wkv_kernels.cuh"
+#include "wkv_prefill.cuh"
 
 struct wkv_ctx {
   wkv_config cfg;
@@ -54,6 +56,11 @@ struct wkv_ctx {
   void* stage_v = nullptr;
   void* stage_out = nullptr;
   int32_t* stage_ev = nullptr;
+  // bulk prompt phase: scratch for the logits of one block of query rows per lane (taken on first use), and which
+  // layers have consumed no token since creation / the last reset
+  float* bulk_S = nullptr;
+  int bulk_stride = 0;
+  std::vector<char> fresh;
   std::vector<void*> owned;
   long long device_bytes = 0;
   long long launches = 0;
@@ -282,6 +289,7 @@ void note_outputs(wkv_ctx* c, const void* out, size_t out_bytes, const void* ev,
 }
 
 int run_reset(wkv_ctx* c) {
+  c->fresh.assign((size_t)c->cfg.n_layers, 1);
   for (int i = 0; i < 2; ++i) WKV_CUDA(c, cudaMemsetAsync(c->ticket[i], 0, (size_t)c->lanes_per_layer * 4, c->stream));
   if (c->fused_ticket) WKV_CUDA(c, cudaMemsetAsync(c->fused_ticket, 0, (size_t)c->lanes_total * 4, c->stream));
   wkv::reset_kernel<<<592, 256, 0, c->stream>>>(c->lane_state, c->pos, c->a, c->next, c->prev, c->lanes_total, c->cap,
@@ -313,6 +321,24 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
   if (layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || h < 0 || h >= c->cfg.n_kv_heads)
     return fail(c, WKV_ERR_INVALID, "layer / sequence / kv_head out of range");
   return WKV_OK;
+}
+
+template <typename T, int D>
+cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
+  constexpr int smem = wkv::bulk_smem_bytes<D>();
+  auto go = [&](auto kern) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    kern<<<lanes, wkv::kBulkThreads, smem, s>>>(P);
+    return cudaGetLastError();
+  };
+  switch (G) {
+    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1>);
+    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2>);
+    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4>);
+    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8>);
+  }
+  return cudaErrorInvalidValue;
 }
 
 }  // namespace
@@ -441,6 +467,7 @@ static int decode_step_impl(wkv_ctx* c, int32_t layer, const void* q, const void
   P.tok_idx = 0;
   const size_t row = (size_t)D * c->elem;
   const size_t q_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * row, kv_bytes = (size_t)c->lanes_per_layer * row;
+  c->fresh[layer] = 0;
   if (!c->use_cluster) prepare_overlap(c, P, layer, q_bytes, kv_bytes, inputs_ready);
   cudaError_t e = launch_any(c, P, c->use_cluster);
   c->launches += c->use_cluster ? 1 : 2;
@@ -484,6 +511,7 @@ int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void*
     P.ev_bs = c->cfg.n_kv_heads;
     P.wait_at_start = 2;
     g_last_launcher.store(c);
+    c->fresh.assign((size_t)c->cfg.n_layers, 0);
     cudaError_t e = launch_any(c, P, c->fused_cluster, (int)c->lanes_total);
     c->launches += c->fused_cluster ? 1 : 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (all layers)");
@@ -531,6 +559,7 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   // kernel writes every logit and every partial of an active lane before the epilogue kernel reads them.
   P.wait_at_start = 2;                 // one array for everybody: never start before the previous kernel has finished
   c->last_layer = -1;
+  c->fresh[layer] = 0;
   g_last_launcher.store(nullptr);
   e = launch_any(c, P, false);
   c->launches += 2;
@@ -573,12 +602,9 @@ int wkv_decode_step_layers_host(wkv_ctx* c, const void* q, const void* k, const 
   return WKV_OK;
 }
 
-int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
-                int32_t T_max, void* out, int32_t* evicted_pos) {
-  if (!c) return WKV_ERR_INVALID;
-  if (!Q || !K || !V) return fail(c, WKV_ERR_INVALID, "Q, K and V must not be NULL");
-  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
-  if (T_max < 0) return fail(c, WKV_ERR_INVALID, "T_max must be >= 0");
+// Tokens [t_begin, T_max) of a prompt, one step of Algorithm 1 per token.
+static int stream_tokens(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                         int32_t t_begin, int32_t T_max, void* out, int32_t* evicted_pos) {
   const long long D = c->cfg.head_dim, Hq = c->cfg.n_q_heads, Hk = c->cfg.n_kv_heads;
   wkv::StepParams P = base_params(c, layer);
   P.seq_lens = seq_lens;
@@ -586,7 +612,8 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
   P.kv_bs = (long long)T_max * Hk * D;
   P.out_bs = out ? P.q_bs : Hq * D;
   P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
-  for (int t = 0; t < T_max; ++t) {
+  if (t_begin < T_max) c->fresh[layer] = 0;
+  for (int t = t_begin; t < T_max; ++t) {
     P.tok_idx = t;
     P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
     P.k = (const char*)K + (size_t)t * Hk * D * c->elem;
@@ -600,6 +627,65 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
   }
   note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
   return WKV_OK;
+}
+
+static int check_prefill_args(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, int32_t T_max) {
+  if (!c) return WKV_ERR_INVALID;
+  if (!Q || !K || !V) return fail(c, WKV_ERR_INVALID, "Q, K and V must not be NULL");
+  if (layer < 0 || layer >= c->cfg.n_layers) return fail(c, WKV_ERR_INVALID, "layer out of range");
+  if (T_max < 0) return fail(c, WKV_ERR_INVALID, "T_max must be >= 0");
+  return WKV_OK;
+}
+
+int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                int32_t T_max, void* out, int32_t* evicted_pos) {
+  const int rc = check_prefill_args(c, layer, Q, K, V, T_max);
+  if (rc != WKV_OK) return rc;
+  return stream_tokens(c, layer, Q, K, V, seq_lens, 0, T_max, out, evicted_pos);
+}
+
+int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                     int32_t T_max, void* out, int32_t* evicted_pos) {
+  int rc = check_prefill_args(c, layer, Q, K, V, T_max);
+  if (rc != WKV_OK) return rc;
+  int32_t n0 = 0;
+  if (c->fresh[layer] && T_max > 0) {
+    // Every lane of the layer is empty: the first min(T_max, budget) tokens compress nothing and go through the
+    // dense kernel; the rest of the prompt is streamed behind it on the same stream.
+    n0 = std::min(T_max, c->cfg.budget);
+    if (c->bulk_S == nullptr) {
+      c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
+      rc = take(c, &c->bulk_S, (size_t)c->lanes_per_layer * wkv::kBulkRows * c->bulk_stride * 4);
+      if (rc != WKV_OK) return rc;
+    }
+    wkv::PrefillParams P;
+    std::memset(&P, 0, sizeof(P));
+    P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
+    P.lane_state = c->lane_state;
+    P.S = c->bulk_S;
+    P.Q = Q; P.K = K; P.V = V; P.out = out; P.evicted = evicted_pos; P.seq_lens = seq_lens;
+    P.lane0 = layer * c->lanes_per_layer;
+    P.n_kv_heads = c->cfg.n_kv_heads;
+    P.cap = c->cap;
+    P.T_max = T_max;
+    P.n0 = n0;
+    P.s_stride = c->bulk_stride;
+    P.scale = c->scale;
+    cudaError_t e;
+    if (c->cfg.dtype == WKV_BF16)
+      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128>(c->group, P, c->lanes_per_layer, c->stream)
+                                 : launch_bulk<__nv_bfloat16, 64>(c->group, P, c->lanes_per_layer, c->stream);
+    else
+      e = c->cfg.head_dim == 128 ? launch_bulk<float, 128>(c->group, P, c->lanes_per_layer, c->stream)
+                                 : launch_bulk<float, 64>(c->group, P, c->lanes_per_layer, c->stream);
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "bulk prefill launch");
+    c->fresh[layer] = 0;
+    c->last_layer = -1;                  // the next scan of this context waits for this kernel before anything else
+    g_last_launcher.store(nullptr);
+    note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+  }
+  return stream_tokens(c, layer, Q, K, V, seq_lens, n0, T_max, out, evicted_pos);
 }
 
 int wkv_export_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* len, int32_t* tokens, int32_t* pos,
@@ -666,6 +752,7 @@ int wkv_import_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int3
   const long long lane = ((long long)layer * c->cfg.batch + b) * c->cfg.n_kv_heads + kv_head;
   const int cap = c->cap;
   const size_t row = (size_t)c->cfg.head_dim * c->elem;
+  c->fresh[layer] = 0;
   std::vector<int32_t> hpos(cap, -1), hnext(cap, -1), hprev(cap, -1);
   std::vector<float> ha(cap, 0.f);
   for (int i = 0; i < len; ++i) {

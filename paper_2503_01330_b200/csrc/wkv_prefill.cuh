@@ -1,0 +1,311 @@
+// Bulk prompt phase of WeightedKV (Algorithm 1) for sm_100a.
+//
+// Algorithm 1 streams: one token, one pass over the cache.  While a lane holds at most `budget` entries nothing is
+// compressed, so the first n = min(prompt length, budget) iterations are plain causal attention and can be done as one
+// dense problem per lane: logits S = scale * Q K^T (lower triangle), row softmax, outputs O = P V, and the column sums
+// a_i = sum_t mean_g P[t, g, i] that Algorithm 1 accumulates one step at a time.  This kernel computes exactly what
+// those n streamed steps compute: every logit with the reproducible dot, every probability with the reproducible
+// exponential and the integer-sum normaliser, and every a_i by adding its terms in ascending t, so that K, pos, a and
+// the links come out bit-identical to streaming; the outputs (not part of that chain) agree to rounding.
+//
+// One CTA per lane walks the prompt in blocks of 16 query rows (16 / G tokens x G query heads):
+//   phase 1  S block = Q block . K^T tile by tile (fp32 FMAs in the reproducible order), causal mask, parked in an
+//            L2-resident scratch row block; exact row maxima
+//   phase 2  e = exp(s - M) in place, Z as an exact integer sum
+//   phase 3  per key tile: P = e / Z, a_i += group mean (rows in ascending t), O += P . V
+// The work is arithmetic-bound (about n^2 d G FMAs per lane against n d bytes): the roofline is the fp32 pipe.
+#pragma once
+#include "wkv_kernels.cuh"
+
+namespace wkv {
+
+constexpr int kBulkRows = 16;        // query rows per block: 16 / G tokens x G heads
+constexpr int kBulkKeys = 128;       // keys per tile
+constexpr int kBulkThreads = 128;    // 4 warps; warp w owns query rows 4w .. 4w+3
+constexpr int kBulkPadP = 20;        // floats per key in the probability tile (16 rows + padding)
+
+struct PrefillParams {
+  void* Kc;
+  void* Vc;
+  float* a;
+  int32_t* pos;
+  int32_t* next;
+  int32_t* prev;
+  int32_t* lane_state;
+  float* S;                  // [lanes of the layer][kBulkRows][s_stride] logits, then exponentials
+  const void* Q;             // [batch, T_max, n_q_heads, D]
+  const void* K;             // [batch, T_max, n_kv_heads, D]
+  const void* V;
+  void* out;                 // [batch, T_max, n_q_heads, D] or null
+  int32_t* evicted;          // [batch, T_max, n_kv_heads] or null
+  const int32_t* seq_lens;   // [batch] or null
+  int lane0, n_kv_heads, cap, T_max;
+  int n0;                    // tokens this kernel covers at most: min(T_max, budget)
+  int s_stride;              // multiple of kBulkKeys, >= n0
+  float scale;
+};
+
+template <int D>
+constexpr int bulk_smem_bytes() {
+  return (kBulkRows * D + kBulkKeys * (D + 4) + kBulkKeys * kBulkPadP) * 4;
+}
+
+// 4 elements of a row widened to fp32
+__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
+  const uint2 t = *reinterpret_cast<const uint2*>(p);
+  return make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u), __uint_as_float(t.y << 16),
+                     __uint_as_float(t.y & 0xffff0000u));
+}
+__device__ __forceinline__ void store_row_part(float* p, const float (&x)[4]) {
+  *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
+}
+__device__ __forceinline__ void store_row_part(float* p, const float (&x)[2]) {
+  *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]);
+}
+__device__ __forceinline__ void store_row_part(__nv_bfloat16* p, const float (&x)[4]) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(x[0], x[1]), hi = __floats2bfloat162_rn(x[2], x[3]);
+  uint2 t;
+  t.x = *reinterpret_cast<const uint32_t*>(&lo);
+  t.y = *reinterpret_cast<const uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(p) = t;
+}
+__device__ __forceinline__ void store_row_part(__nv_bfloat16* p, const float (&x)[2]) {
+  *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(x[0], x[1]);
+}
+
+// rows [row0, row0 + n_rows) of a [.., T_max, H, D] tensor (head h of sequence b) -> shared memory as fp32, row stride
+// `stride` floats; rows at or beyond `limit` are zero-filled
+template <typename T, int D>
+__device__ __forceinline__ void stage_rows(float* dst, int stride, const T* src, long long row_stride, int row0, int n_rows,
+                                           int limit) {
+  constexpr int Q4 = D / 4;
+  for (int c = threadIdx.x; c < n_rows * Q4; c += kBulkThreads) {
+    const int r = c / Q4, q4 = c % Q4;
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row0 + r < limit) x = load4(src + (long long)(row0 + r) * row_stride + q4 * 4);
+    *reinterpret_cast<float4*>(dst + r * stride + q4 * 4) = x;
+  }
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const PrefillParams P) {
+  constexpr int BQ = kBulkRows / G;              // tokens per row block
+  constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
+  constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
+  constexpr int KS = D + 4;                      // padded row stride of the K / V tile: conflict-free 128-bit reads
+  constexpr int CPT = D / 32;                    // output channels per thread in the P.V phase
+  static_assert(kBulkRows % G == 0 && kBulkThreads == kBulkKeys && kBulkThreads == 8 * kBulkRows, "thread maps");
+  extern __shared__ __align__(16) unsigned char bulk_smem[];
+  float* Qs = reinterpret_cast<float*>(bulk_smem);       // [16][D]
+  float* KV = Qs + kBulkRows * D;                        // [128][D + 4]: the K tile (phase 1), the V tile (phase 3)
+  float* Pt = KV + kBulkKeys * KS;                       // [128][20]: probabilities of the tile, [key][row]
+
+  const int tid = threadIdx.x, w = tid >> 5, ln = tid & 31;
+  const int lane_local = blockIdx.x;
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  const long long lane = (long long)P.lane0 + lane_local;
+  const int Hk = P.n_kv_heads, Hq = Hk * G;
+  int n = P.n0;
+  if (P.seq_lens != nullptr) n = min(n, max(0, P.seq_lens[b]));
+  const T* Qb = reinterpret_cast<const T*>(P.Q) + ((long long)b * P.T_max * Hq + (long long)hk * G) * D;   // + t*Hq*D + g*D
+  const T* Kb = reinterpret_cast<const T*>(P.K) + ((long long)b * P.T_max * Hk + hk) * D;                  // + t*Hk*D
+  const T* Vb = reinterpret_cast<const T*>(P.V) + ((long long)b * P.T_max * Hk + hk) * D;
+  T* Kl = reinterpret_cast<T*>(P.Kc) + lane * (long long)P.cap * D;
+  T* Vl = reinterpret_cast<T*>(P.Vc) + lane * (long long)P.cap * D;
+  float* a_l = P.a + lane * P.cap;
+  float* S = P.S + (long long)lane_local * kBulkRows * P.s_stride;
+
+  // no compression happens in this phase: report "nothing removed" for every token it covers
+  if (P.evicted != nullptr)
+    for (int t = tid; t < P.n0; t += kBulkThreads) P.evicted[((long long)b * P.T_max + t) * Hk + hk] = -1;
+  if (n == 0) return;
+
+  // the cache after n uncompressed steps: token i in slot i, linked in order (Algorithm 1 appends, nothing is removed)
+  {
+    constexpr int Q8 = D * (int)sizeof(T) / 16;          // 16-byte pieces per row
+    for (int c = tid; c < n * Q8; c += kBulkThreads) {
+      const int r = c / Q8, q = c % Q8;
+      reinterpret_cast<uint4*>(Kl + (long long)r * D)[q] = reinterpret_cast<const uint4*>(Kb + (long long)r * Hk * D)[q];
+      reinterpret_cast<uint4*>(Vl + (long long)r * D)[q] = reinterpret_cast<const uint4*>(Vb + (long long)r * Hk * D)[q];
+    }
+    int32_t* pos_l = P.pos + lane * P.cap;
+    int32_t* next_l = P.next + lane * P.cap;
+    int32_t* prev_l = P.prev + lane * P.cap;
+    for (int i = tid; i < n; i += kBulkThreads) {
+      pos_l[i] = i;
+      next_l[i] = i + 1 < n ? i + 1 : -1;
+      prev_l[i] = i - 1;
+    }
+    if (tid == 0) {
+      int32_t* st = P.lane_state + lane * LS_STRIDE;
+      st[LS_LEN] = n;
+      st[LS_T] = n;
+      st[LS_HEAD] = 0;
+      st[LS_TAIL] = n - 1;
+      st[LS_FREE] = n;                                   // while growing, slots fill in arrival order
+    }
+  }
+
+  for (int t0 = 0; t0 < n; t0 += BQ) {
+    const int nk = min(t0 + BQ, n);                      // keys 0 .. nk-1 are visible to some row of the block
+    const int n_tiles = (nk + kBulkKeys - 1) / kBulkKeys;
+    int t_row[4];                                        // token of each of my 4 rows
+    bool act[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      t_row[i] = t0 + (4 * w + i) / G;
+      act[i] = t_row[i] < n;
+    }
+    __syncthreads();                                     // the previous block is done with Qs, KV and Pt
+    // query rows of the block: row rho = token_in_block * G + head; rows of tokens at or beyond n are zero
+    for (int c = tid; c < kBulkRows * (D / 4); c += kBulkThreads) {
+      const int r = c / (D / 4), q4 = c % (D / 4);
+      const int tok = r / G, g = r % G;
+      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (t0 + tok < n) x = load4(Qb + ((long long)(t0 + tok) * Hq + g) * D + q4 * 4);
+      *reinterpret_cast<float4*>(Qs + r * D + q4 * 4) = x;
+    }
+
+    // ---- phase 1: logits of the row block, tile by tile --------------------------------------------------------
+    float row_max[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    for (int kt = 0; kt < n_tiles; ++kt) {
+      const int k0 = kt * kBulkKeys;
+      __syncthreads();
+      stage_rows<T, D>(KV, KS, Kb, (long long)Hk * D, k0, kBulkKeys, nk);
+      __syncthreads();
+      // The reproducible dot: 16 partial sums over blocks of D/16 channels (even- and odd-channel fma chains, added),
+      // combined as the butterfly p_r + p_{r xor off}, off = 8, 4, 2, 1.  The blocks are visited in the order that
+      // lets the butterfly's additions be done as soon as both operands exist (a fixed tree; fp addition commutes).
+      float st1[16], st2[16], st3[16], st4[16], dot[16];
+#pragma unroll
+      for (int s = 0; s < 16; ++s) {
+        const int blk = ((s & 1) << 3) | ((s & 2) << 1) | ((s & 4) >> 1) | ((s & 8) >> 3);   // 0,8,4,12,2,10,6,14,1,...
+        f32x2 qv[4][CP], kv[4][CP];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) load_pairs<CP>(Qs + (4 * w + i) * D + blk * CH, qv[i]);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) load_pairs<CP>(KV + (ln + 32 * j) * KS + blk * CH, kv[j]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int o = i * 4 + j;
+            f32x2 acc = 0ull;
+#pragma unroll
+            for (int e = 0; e < CP; ++e) acc = fma2(qv[i][e], kv[j][e], acc);
+            float v = __fadd_rn(lo_of(acc), hi_of(acc));
+            if (s & 1) {
+              v = __fadd_rn(st1[o], v);
+              if (s & 2) {
+                v = __fadd_rn(st2[o], v);
+                if (s & 4) {
+                  v = __fadd_rn(st3[o], v);
+                  if (s & 8) dot[o] = __fadd_rn(st4[o], v);
+                  else st4[o] = v;
+                } else st3[o] = v;
+              } else st2[o] = v;
+            } else st1[o] = v;
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int key = k0 + ln + 32 * j;
+          const bool ok = act[i] && key <= t_row[i];     // causal: the row's own token is its last key
+          const float sc = ok ? __fmul_rn(P.scale, dot[i * 4 + j]) : -INFINITY;
+          S[(long long)(4 * w + i) * P.s_stride + key] = sc;
+          row_max[i] = fmaxf(row_max[i], sc);
+        }
+      }
+    }
+    // ---- phase 2: exponentials in place and the integer-sum normaliser (each thread re-reads what it wrote) ------
+    float M[4], Z[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float m = row_max[i];
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+      M[i] = m;
+      unsigned long long z = 0ull;
+      float* Srow = S + (long long)(4 * w + i) * P.s_stride;
+      for (int key = ln; key < n_tiles * kBulkKeys; key += 32) {
+        const float sc = Srow[key];
+        const float e = (act[i] && sc != -INFINITY) ? repro_exp(__fsub_rn(sc, m)) : 0.f;
+        Srow[key] = e;
+        z += __float2ull_rz(__fmul_rn(e, 1099511627776.0f));
+      }
+      z = warp_sum_u64(z);
+      Z[i] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
+    }
+    // ---- phase 3: probabilities, score accumulation, outputs -----------------------------------------------------
+    float o_acc[4][CPT];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int c = 0; c < CPT; ++c) o_acc[i][c] = 0.f;
+    for (int kt = 0; kt < n_tiles; ++kt) {
+      const int k0 = kt * kBulkKeys;
+      __syncthreads();
+      stage_rows<T, D>(KV, KS, Vb, (long long)Hk * D, k0, kBulkKeys, nk);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int kk = ln + 32 * j;
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+        *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
+      }
+      __syncthreads();
+      // a_i <- a_i + mean over the group's heads, one token after the other (the order Algorithm 1 adds them in)
+      {
+        const int key = k0 + tid;
+        if (key < nk) {
+          float a_i = key >= t0 ? 0.f : a_l[key];        // the key's own token is in this block: it starts from [a, 0]
+          const float* pr = Pt + tid * kBulkPadP;
+#pragma unroll
+          for (int tok = 0; tok < BQ; ++tok) {
+            float pbar = pr[tok * G];
+#pragma unroll
+            for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pr[tok * G + g]);
+            if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
+            if (key <= t0 + tok && t0 + tok < n) a_i = __fadd_rn(a_i, pbar);
+          }
+          a_l[key] = a_i;
+        }
+      }
+      // O += P . V for my 4 rows and CPT channels
+      const int kmax = min(kBulkKeys, nk - k0);
+      for (int kk = 0; kk < kmax; ++kk) {
+        const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
+        const float pr[4] = {p4.x, p4.y, p4.z, p4.w};
+        float vv[CPT];
+        if constexpr (CPT == 4) {
+          const float4 t = *reinterpret_cast<const float4*>(KV + kk * KS + ln * 4);
+          vv[0] = t.x; vv[1] = t.y; vv[2] = t.z; vv[3] = t.w;
+        } else {
+          const float2 t = *reinterpret_cast<const float2*>(KV + kk * KS + ln * 2);
+          vv[0] = t.x; vv[1] = t.y;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int c = 0; c < CPT; ++c) o_acc[i][c] = fmaf(pr[i], vv[c], o_acc[i][c]);
+      }
+    }
+    if (P.out != nullptr) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (!act[i]) continue;
+        const int g = (4 * w + i) % G;
+        T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t_row[i]) * Hq + (long long)hk * G + g) * D + ln * CPT;
+        store_row_part(dst, o_acc[i]);
+      }
+    }
+  }
+}
+
+}  // namespace wkv

@@ -1,0 +1,101 @@
+"""wkv_prefill_bulk against the CPU oracle (which streams, as Algorithm 1 does) and against wkv_prefill: the dense
+start of the prompt must leave exactly the state that token-by-token processing leaves."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2503_01330_b200 import binding
+from paper_2503_01330_b200.synth import WORKLOADS, TokenStream, Workload
+
+from parity_util import Parity
+
+pytestmark = pytest.mark.gpu
+
+
+def small(layers=1, batch=2, hq=4, hkv=4, d=64, dtype="f32", m=40, W=4, S=0, rank=0):
+    return Workload("s", layers, batch, hq, hkv, d, dtype, m, W, S, 0, 0, 0, rank, 0.05, rank == 0)
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,m,W,S,T", [
+    ("f32", 64, 4, 4, 40, 4, 0, 100),        # budget not a multiple of the row block; streamed tail of 60 tokens
+    ("f32", 128, 2, 2, 300, 8, 0, 300),      # prompt == budget: three key tiles, nothing streamed
+    ("f32", 64, 2, 2, 200, 4, 0, 131),       # prompt shorter than the budget, ragged last tile and last row block
+    ("bf16", 128, 4, 4, 150, 8, 4, 260),     # sinks, bf16
+    ("bf16", 128, 8, 4, 129, 16, 0, 200),    # group of 2, one key past a tile boundary
+    ("bf16", 128, 8, 2, 95, 16, 1, 170),     # group of 4
+    ("f32", 64, 8, 1, 70, 3, 0, 120),        # group of 8: a token's heads span two warps
+    ("bf16", 64, 4, 2, 1, 1, 0, 20),         # smallest cache: one token in bulk, the rest streamed
+    ("f32", 64, 2, 2, 16, 2, 0, 1),          # a single token
+])
+def test_bulk_prefill_matches_oracle_every_token(dtype, d, hq, hkv, m, W, S, T):
+    wl = small(batch=3, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=W, S=S, rank=16 if dtype == "bf16" else 0)
+    p = Parity(wl, seed=40 + m, ragged=[T, T, T])
+    p.prefill(T, chunk=T, bulk=True)
+    p.compare_state()
+    p.decode(m // 2 + 5)
+    p.compare_state()
+    assert p.n_evictions == wl.lanes * max(0, T + m // 2 + 5 - m)
+    p.close()
+
+
+def test_bulk_prefill_ragged_lengths():
+    """Per-sequence lengths: empty, shorter than the budget, exactly the budget, longer."""
+    wl = small(layers=2, batch=4, d=128, dtype="bf16", m=96, W=8, rank=16)
+    p = Parity(wl, seed=9, ragged=[150, 0, 96, 41])
+    p.prefill(150, chunk=150, bulk=True)
+    p.compare_state()
+    p.decode(70)
+    p.compare_state()
+    p.close()
+
+
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+def test_bulk_and_streamed_prefill_leave_identical_state(schedule):
+    wl = small(layers=2, batch=2, hq=8, hkv=2, d=128, dtype="bf16", m=200, W=8, rank=16)
+    st = TokenStream(wl, 21, "cuda:0")
+    Q, K, V = st.tokens(0, 330)
+    lens = torch.tensor([330, 177], dtype=torch.int32, device="cuda:0")
+    states, outs = [], []
+    for bulk in (False, True):
+        ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window,
+                              dtype=binding.WKV_BF16, schedule=schedule)
+        out = torch.zeros(wl.n_layers, wl.batch, 330, wl.n_q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda:0")
+        ev = torch.full((wl.n_layers, wl.batch, 330, wl.n_kv_heads), -7, dtype=torch.int32, device="cuda:0")
+        for layer in range(wl.n_layers):
+            (ctx.wkv_prefill_bulk if bulk else ctx.wkv_prefill)(layer, Q[layer], K[layer], V[layer], lens, out[layer], ev[layer])
+        assert ctx.wkv_status() == 0
+        states.append([ctx.wkv_export_state(l, b, h) for l in range(2) for b in range(2) for h in range(2)])
+        outs.append((out.float().cpu(), ev.cpu()))
+        ctx.close()
+    for s0, s1 in zip(*states):
+        assert s0["len"] == s1["len"] and s0["tokens"] == s1["tokens"]
+        for key in ("pos", "a", "K", "V"):
+            assert torch.equal(s0[key], s1[key]), key
+    assert torch.equal(outs[0][1], outs[1][1])                       # removed positions, -1 where nothing was removed
+    torch.testing.assert_close(outs[1][0], outs[0][0], rtol=2e-2, atol=1e-3)
+
+
+def test_bulk_prefill_on_a_used_layer_streams():
+    """A layer that already holds tokens is continued token by token; the result is still Algorithm 1's."""
+    wl = small(batch=2, d=64, dtype="f32", m=50, W=4)
+    p = Parity(wl, seed=5, ragged=[140, 140])
+    p.prefill(30, chunk=30, bulk=True)      # empty layer: dense
+    p.prefill(60, chunk=60, bulk=True)      # 30 tokens held: streamed
+    p.decode(10)
+    p.prefill(40, chunk=40, bulk=True)
+    p.compare_state()
+    launches = p.ctx.wkv_launch_count()
+    p.ctx.wkv_reset()
+    assert p.ctx.wkv_launch_count() == launches + 1
+    p.close()
+
+
+def test_bulk_prefill_llama7b_layer_shape():
+    """32 heads x 128, bf16, budget 2048: 2048 dense + 2048 streamed prompt tokens, sampled lanes against the oracle."""
+    wl = WORKLOADS["llama7b_layer"]
+    p = Parity(wl, sample=6)
+    p.prefill(wl.prefill, chunk=wl.prefill, bulk=True)
+    p.compare_state()
+    p.decode(64)
+    p.compare_state()
+    p.close()
