@@ -88,13 +88,41 @@ __device__ __forceinline__ void stage_rows(float* dst, int stride, const T* src,
   }
 }
 
+// a_i <- a_i + mean over the group's heads of P[t, g, i], one token after the other (the order Algorithm 1 adds them
+// in).  Thread tid owns key k0 + tid of the tile; Pt is [key][row] with row = token_in_block * G + head.
+template <int G>
+__device__ __forceinline__ void fold_columns(const float* Pt, float* a_l, int k0, int t0, int nk, int n) {
+  constexpr int BQ = kBulkRows / G;
+  const int key = k0 + (int)threadIdx.x;
+  if (key >= nk) return;
+  float a_i = key >= t0 ? 0.f : a_l[key];                // the key's own token is in this block: it starts from [a, 0]
+  const float* pr = Pt + threadIdx.x * kBulkPadP;
+#pragma unroll
+  for (int tok = 0; tok < BQ; ++tok) {
+    float pbar = pr[tok * G];
+#pragma unroll
+    for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pr[tok * G + g]);
+    if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
+    if (key <= t0 + tok && t0 + tok < n) a_i = __fadd_rn(a_i, pbar);
+  }
+  a_l[key] = a_i;
+}
+
+// c[16x8, fp32] += a[16x16, bf16, row-major] . b[16x8, bf16, column-major] on the tensor cores (one warp)
+__device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const PrefillParams P) {
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
   constexpr int KS = D + 4;                      // padded row stride of the K / V tile: conflict-free 128-bit reads
-  constexpr int CPT = D / 32;                    // output channels per thread in the P.V phase
+  constexpr int CPT = D / 32;                    // output channels per thread in the P.V phase (fp32 storage)
+  constexpr bool kTensorPV = sizeof(T) == 2;     // bf16 storage: P.V on the tensor cores
   static_assert(kBulkRows % G == 0 && kBulkThreads == kBulkKeys && kBulkThreads == 8 * kBulkRows, "thread maps");
   extern __shared__ __align__(16) unsigned char bulk_smem[];
   float* Qs = reinterpret_cast<float*>(bulk_smem);       // [16][D]
@@ -241,68 +269,135 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
       Z[i] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
     }
     // ---- phase 3: probabilities, score accumulation, outputs -----------------------------------------------------
-    float o_acc[4][CPT];
+    if constexpr (kTensorPV) {
+      // bf16 storage: O += P . V on the tensor cores (the outputs are not part of the reproducible chain).  Warp w
+      // takes all 16 rows and channels [w*D/4, (w+1)*D/4); P goes in as a bf16 hi + lo pair per probability.
+      constexpr int NTW = D / 32;                        // 8-channel n-tiles per warp
+      constexpr int VS = D + 8;                          // bf16 row stride of the V tile: conflict-free ldmatrix
+      constexpr int PS = kBulkKeys + 8;                  // bf16 row stride of the P tiles
+      __nv_bfloat16* Vt = reinterpret_cast<__nv_bfloat16*>(KV);          // [128][D + 8]
+      __nv_bfloat16* Ph = Vt + kBulkKeys * VS;                           // [16][128 + 8] hi parts
+      __nv_bfloat16* Pl = Ph + kBulkRows * PS;                           // [16][128 + 8] lo parts
+      float cacc[NTW][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-      for (int c = 0; c < CPT; ++c) o_acc[i][c] = 0.f;
-    for (int kt = 0; kt < n_tiles; ++kt) {
-      const int k0 = kt * kBulkKeys;
-      __syncthreads();
-      stage_rows<T, D>(KV, KS, Vb, (long long)Hk * D, k0, kBulkKeys, nk);
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int kk = ln + 32 * j;
-        float p[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
-        *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
-      }
-      __syncthreads();
-      // a_i <- a_i + mean over the group's heads, one token after the other (the order Algorithm 1 adds them in)
-      {
-        const int key = k0 + tid;
-        if (key < nk) {
-          float a_i = key >= t0 ? 0.f : a_l[key];        // the key's own token is in this block: it starts from [a, 0]
-          const float* pr = Pt + tid * kBulkPadP;
-#pragma unroll
-          for (int tok = 0; tok < BQ; ++tok) {
-            float pbar = pr[tok * G];
-#pragma unroll
-            for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pr[tok * G + g]);
-            if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
-            if (key <= t0 + tok && t0 + tok < n) a_i = __fadd_rn(a_i, pbar);
+      for (int nt = 0; nt < NTW; ++nt) cacc[nt][0] = cacc[nt][1] = cacc[nt][2] = cacc[nt][3] = 0.f;
+      for (int kt = 0; kt < n_tiles; ++kt) {
+        const int k0 = kt * kBulkKeys;
+        __syncthreads();
+        {
+          constexpr int Q8 = D / 8;                      // 16-byte pieces per row
+          for (int c = tid; c < kBulkKeys * Q8; c += kBulkThreads) {
+            const int r = c / Q8, q = c % Q8;
+            uint4 x = make_uint4(0u, 0u, 0u, 0u);        // keys beyond the block's range must be zeros, not stale bits
+            if (k0 + r < nk) x = reinterpret_cast<const uint4*>(Vb + (long long)(k0 + r) * Hk * D)[q];
+            *reinterpret_cast<uint4*>(Vt + r * VS + q * 8) = x;
           }
-          a_l[key] = a_i;
-        }
-      }
-      // O += P . V for my 4 rows and CPT channels
-      const int kmax = min(kBulkKeys, nk - k0);
-      for (int kk = 0; kk < kmax; ++kk) {
-        const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
-        const float pr[4] = {p4.x, p4.y, p4.z, p4.w};
-        float vv[CPT];
-        if constexpr (CPT == 4) {
-          const float4 t = *reinterpret_cast<const float4*>(KV + kk * KS + ln * 4);
-          vv[0] = t.x; vv[1] = t.y; vv[2] = t.z; vv[3] = t.w;
-        } else {
-          const float2 t = *reinterpret_cast<const float2*>(KV + kk * KS + ln * 2);
-          vv[0] = t.x; vv[1] = t.y;
         }
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
+        for (int j = 0; j < 4; ++j) {
+          const int kk = ln + 32 * j;
+          float p[4];
 #pragma unroll
-          for (int c = 0; c < CPT; ++c) o_acc[i][c] = fmaf(pr[i], vv[c], o_acc[i][c]);
+          for (int i = 0; i < 4; ++i) {
+            p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+            const __nv_bfloat16 hi = __float2bfloat16_rn(p[i]);
+            Ph[(4 * w + i) * PS + kk] = hi;
+            Pl[(4 * w + i) * PS + kk] = __float2bfloat16_rn(p[i] - __bfloat162float(hi));
+          }
+          *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
+        }
+        __syncthreads();
+        fold_columns<G>(Pt, a_l, k0, t0, nk, n);
+        const int ksteps = (min(kBulkKeys, nk - k0) + 15) / 16;
+        // fragment addresses: A (P, row-major [row][key]): thread i -> row (i%8) + 8*((i/8)&1), key 8*(i/16);
+        //                     B (V, [key][channel], read transposed): thread i -> key (i%8) + 8*((i/8)&1), channel 8*(i/16)
+        const uint32_t a_off = (uint32_t)((((ln & 7) + ((ln >> 3) & 1) * 8) * PS + (ln >> 4) * 8) * 2);
+        const uint32_t ph_base = smem_u32(Ph) + a_off, pl_base = smem_u32(Pl) + a_off;
+        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((((ln & 7) + ((ln >> 3) & 1) * 8) * VS + w * (D / 4) + (ln >> 4) * 8) * 2);
+        for (int ks = 0; ks < ksteps; ++ks) {
+          uint32_t ah[4], al[4];
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(ah[0]), "=r"(ah[1]), "=r"(ah[2]), "=r"(ah[3]) : "r"(ph_base + ks * 32) : "memory");
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(al[0]), "=r"(al[1]), "=r"(al[2]), "=r"(al[3]) : "r"(pl_base + ks * 32) : "memory");
+#pragma unroll
+          for (int np = 0; np < NTW / 2; ++np) {
+            uint32_t bf[4];
+            asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(bf[0]), "=r"(bf[1]), "=r"(bf[2]), "=r"(bf[3])
+                         : "r"(v_base + (uint32_t)(ks * 16 * VS * 2 + np * 32)) : "memory");
+            mma_m16n8k16_bf16(cacc[2 * np], ah, bf[0], bf[1]);
+            mma_m16n8k16_bf16(cacc[2 * np], al, bf[0], bf[1]);
+            mma_m16n8k16_bf16(cacc[2 * np + 1], ah, bf[2], bf[3]);
+            mma_m16n8k16_bf16(cacc[2 * np + 1], al, bf[2], bf[3]);
+          }
+        }
       }
-    }
-    if (P.out != nullptr) {
+      if (P.out != nullptr) {
+        // accumulator fragment: rows ln/4 and ln/4 + 8, channels (ln%4)*2, +1 of each n-tile
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if (!act[i]) continue;
-        const int g = (4 * w + i) % G;
-        T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t_row[i]) * Hq + (long long)hk * G + g) * D + ln * CPT;
-        store_row_part(dst, o_acc[i]);
+        for (int h = 0; h < 2; ++h) {
+          const int rho = (ln >> 2) + 8 * h;
+          const int t = t0 + rho / G, g = rho % G;
+          if (t >= n) continue;
+          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t) * Hq + (long long)hk * G + g) * D + w * (D / 4) + (ln & 3) * 2;
+#pragma unroll
+          for (int nt = 0; nt < NTW; ++nt) {
+            const float x[2] = {cacc[nt][2 * h], cacc[nt][2 * h + 1]};
+            store_row_part(dst + nt * 8, x);
+          }
+        }
+      }
+    } else {
+      // fp32 storage: packed fp32 FMAs; warp w keeps its 4 rows, each thread CPT channels
+      f32x2 o_acc[4][CPT / 2];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = 0ull;
+      for (int kt = 0; kt < n_tiles; ++kt) {
+        const int k0 = kt * kBulkKeys;
+        __syncthreads();
+        stage_rows<T, D>(KV, KS, Vb, (long long)Hk * D, k0, kBulkKeys, nk);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int kk = ln + 32 * j;
+          float p[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+            p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+          *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
+        }
+        __syncthreads();
+        fold_columns<G>(Pt, a_l, k0, t0, nk, n);
+        const int kmax = min(kBulkKeys, nk - k0);
+        for (int kk = 0; kk < kmax; ++kk) {
+          const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
+          const f32x2 pp[4] = {pack2(p4.x, p4.x), pack2(p4.y, p4.y), pack2(p4.z, p4.z), pack2(p4.w, p4.w)};
+          f32x2 vv[CPT / 2];
+          if constexpr (CPT == 4) {
+            load_pairs<2>(KV + kk * KS + ln * 4, vv);
+          } else {
+            const float2 t = *reinterpret_cast<const float2*>(KV + kk * KS + ln * 2);
+            vv[0] = pack2(t.x, t.y);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = fma2(pp[i], vv[c], o_acc[i][c]);
+        }
+      }
+      if (P.out != nullptr) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (!act[i]) continue;
+          const int g = (4 * w + i) % G;
+          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t_row[i]) * Hq + (long long)hk * G + g) * D + ln * CPT;
+          float x[CPT];
+#pragma unroll
+          for (int c = 0; c < CPT / 2; ++c) { x[2 * c] = lo_of(o_acc[i][c]); x[2 * c + 1] = hi_of(o_acc[i][c]); }
+          store_row_part(dst, x);
+        }
       }
     }
   }
