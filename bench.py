@@ -133,6 +133,52 @@ def oracle_lane_steps_per_s(wl, n_lanes: int, steps: int, warmup: int, seed: int
     return n_lanes * steps / dt, min(n_lanes, os.cpu_count() or 1)
 
 
+FP32_LANES_PER_SM = 128          # fp32 FMA lanes per SM (4 sub-partitions x 32); one FMA per lane and clock
+
+
+def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
+    """wkv_prefill_bulk on ONE layer of the workload's shape: every sequence brings a prompt of n_tokens (default:
+    the budget, i.e. the whole dense phase).  The kernel is arithmetic-bound: the roofline is the fp32 FMA pipe,
+    peak = SMs x 128 lanes x max SM clock; algorithmic FMAs = lanes x G x n(n+1)/2 x head_dim x 2 (logits and P.V)."""
+    from paper_2503_01330_b200 import binding
+    one = wl.scaled(n_layers=1)
+    n = n_tokens if n_tokens else one.budget
+    n = min(n, one.budget)
+    ctx = binding.Context(1, one.batch, one.n_q_heads, one.n_kv_heads, one.head_dim, one.budget, one.window, one.sink,
+                          binding.WKV_F32 if one.dtype == "f32" else binding.WKV_BF16, device=dev)
+    Q, K, V = TokenStream(one, seed, dev).tokens(0, n)
+    out = torch.empty(one.batch, n, one.n_q_heads, one.head_dim, dtype=one.torch_dtype, device=dev)
+    times = []
+    for _ in range(reps + 1):                      # the first run also takes the scratch from the allocator
+        ctx.wkv_reset()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.wkv_prefill_bulk(0, Q[0], K[0], V[0], None, out)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert ctx.wkv_status() == 0
+    ctx.close()
+    ms = min(times[1:])
+    lanes = one.batch * one.n_kv_heads
+    fma = lanes * one.group * n * (n + 1) // 2 * one.head_dim * 2
+    props = torch.cuda.get_device_properties(dev)
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(pynvml.nvmlDeviceGetHandleByIndex(dev.index or 0), pynvml.NVML_CLOCK_SM)
+    except Exception:
+        max_mhz = 1965
+    peak = props.multi_processor_count * FP32_LANES_PER_SM * max_mhz * 1e6 / 1e12
+    achieved = fma / (ms * 1e-3) / 1e12
+    return {"value": one.batch * n / (ms * 1e-3), "unit": "prompt tokens/s per layer", "ms_per_layer": ms,
+            "tokens_per_sequence": n, "kernel": "prefill_bulk_kernel",
+            "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFMA/s (fp32)", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": f"{props.multi_processor_count} SMs x {FP32_LANES_PER_SM} lanes x {max_mhz} MHz",
+                         "algorithmic_fma_per_launch": fma}}
+
+
 def run_reference(args, wl):
     """The reference arm: the CPU oracle on the host cores; each step is a bounded sample of the workload."""
     cores = os.cpu_count() or 1
@@ -174,6 +220,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling captures)")
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
+                    help="prefill: time only the dense prompt phase (wkv_prefill_bulk) on one layer and print its line")
+    ap.add_argument("--no-bulk-prefill", action="store_true", help="leave the bulk-prefill figure out of the decode line")
     ap.add_argument("--init", default="prefill", choices=["prefill", "import"],
                     help="import: fill every cache through wkv_import_state with one synthetic full lane instead of "
                          "streaming a prompt (profiling captures: no launches before the steps)")
@@ -209,6 +258,16 @@ def main():
     torch.cuda.set_device(dev)
 
     seed = rank_seed(BASE_SEED, rank)
+    if args.mode == "prefill":
+        fig = bulk_prefill_figures(wl, dev, seed, args.prefill_tokens)
+        if rank == 0:
+            fig.update({"metric": "bulk_prefill_prompt_tokens_per_s_per_layer", "n_gpus": 1, "higher_is_better": True,
+                        "dtype": wl.dtype, "data": "synthetic",
+                        "config": {"workload": wl.name, "layers_timed": 1, "batch": wl.batch, "budget": wl.budget}})
+            print(json.dumps(fig), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     dt_code = binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16
     ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window, wl.sink,
                           dt_code, n_splits=args.n_splits, device=dev, schedule=args.schedule)
@@ -344,6 +403,8 @@ def main():
                          "algorithmic_bytes_per_launch": bytes_launch, "launch_ms": launch_ms},
             "e2e": {"value": e2e_value, "unit": "steps/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": n_e2e, "call": "wkv_decode_step_layers_host: one call per step from pinned host buffers"}}
+    if not args.no_bulk_prefill:
+        line["bulk_prefill"] = bulk_prefill_figures(wl, dev, seed)
     if not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         n_lanes, n_steps = cores, 8

@@ -325,7 +325,7 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
 
 template <typename T, int D>
 cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
-  constexpr int smem = wkv::bulk_smem_bytes<D>();
+  constexpr int smem = wkv::bulk_smem_bytes<T, D>();
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -671,6 +671,7 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     P.n0 = n0;
     P.s_stride = c->bulk_stride;
     P.scale = c->scale;
+    P.status = c->status;
     cudaError_t e;
     if (c->cfg.dtype == WKV_BF16)
       e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128>(c->group, P, c->lanes_per_layer, c->stream)

@@ -12,7 +12,11 @@
 //   phase 1  S block = Q block . K^T tile by tile (fp32 FMAs in the reproducible order), causal mask, parked in an
 //            L2-resident scratch row block; exact row maxima
 //   phase 2  e = exp(s - M) in place, Z as an exact integer sum
-//   phase 3  per key tile: P = e / Z, a_i += group mean (rows in ascending t), O += P . V
+//   phase 3  per key tile: P = e / Z, a_i += group mean (rows in ascending t), O += P . V (bf16 storage: tensor
+//            cores, each probability as a bf16 hi + lo pair; fp32 storage: packed fp32 FMAs)
+// K and V tiles arrive through a two-stage ring of bulk asynchronous copies (one row per thread, byte-counted on an
+// mbarrier), issued two tiles ahead -- the V tiles of a block while its exponentials are computed, the K tiles of the
+// next block while this block's outputs are stored -- so the tile loads overlap the arithmetic.
 // The work is arithmetic-bound (about n^2 d G FMAs per lane against n d bytes): the roofline is the fp32 pipe.
 #pragma once
 #include "wkv_kernels.cuh"
@@ -20,7 +24,7 @@
 namespace wkv {
 
 constexpr int kBulkRows = 16;        // query rows per block: 16 / G tokens x G heads
-constexpr int kBulkKeys = 128;       // keys per tile
+constexpr int kBulkKeys = 128;       // granularity of the scratch rows (a multiple of every tile size)
 constexpr int kBulkThreads = 128;    // 4 warps; warp w owns query rows 4w .. 4w+3
 constexpr int kBulkPadP = 20;        // floats per key in the probability tile (16 rows + padding)
 
@@ -43,20 +47,22 @@ struct PrefillParams {
   int n0;                    // tokens this kernel covers at most: min(T_max, budget)
   int s_stride;              // multiple of kBulkKeys, >= n0
   float scale;
+  uint32_t* status;          // device status word (bounded waits report here)
 };
 
-template <int D>
+// keys per tile: a tile row carries 16 bytes of padding, two tiles of rows live in shared memory
+template <typename T> struct BulkTile { static constexpr int kKeys = sizeof(T) == 2 ? 128 : 64; };
+
+template <typename T, int D>
 constexpr int bulk_smem_bytes() {
-  return (kBulkRows * D + kBulkKeys * (D + 4) + kBulkKeys * kBulkPadP) * 4;
+  constexpr int KT = BulkTile<T>::kKeys;
+  return kBulkRows * D * 4                                   // query rows, fp32
+         + 2 * KT * (D * (int)sizeof(T) + 16)                // two tile stages, storage type, padded rows
+         + KT * kBulkPadP * 4                                // probabilities of a tile, fp32
+         + (sizeof(T) == 2 ? 2 * kBulkRows * (KT + 8) * 2 : 0)   // bf16 hi and lo parts of the probabilities
+         + 64;                                               // mbarriers
 }
 
-// 4 elements of a row widened to fp32
-__device__ __forceinline__ float4 load4(const float* p) { return *reinterpret_cast<const float4*>(p); }
-__device__ __forceinline__ float4 load4(const __nv_bfloat16* p) {
-  const uint2 t = *reinterpret_cast<const uint2*>(p);
-  return make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u), __uint_as_float(t.y << 16),
-                     __uint_as_float(t.y & 0xffff0000u));
-}
 __device__ __forceinline__ void store_row_part(float* p, const float (&x)[4]) {
   *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]);
 }
@@ -74,28 +80,15 @@ __device__ __forceinline__ void store_row_part(__nv_bfloat16* p, const float (&x
   *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(x[0], x[1]);
 }
 
-// rows [row0, row0 + n_rows) of a [.., T_max, H, D] tensor (head h of sequence b) -> shared memory as fp32, row stride
-// `stride` floats; rows at or beyond `limit` are zero-filled
-template <typename T, int D>
-__device__ __forceinline__ void stage_rows(float* dst, int stride, const T* src, long long row_stride, int row0, int n_rows,
-                                           int limit) {
-  constexpr int Q4 = D / 4;
-  for (int c = threadIdx.x; c < n_rows * Q4; c += kBulkThreads) {
-    const int r = c / Q4, q4 = c % Q4;
-    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row0 + r < limit) x = load4(src + (long long)(row0 + r) * row_stride + q4 * 4);
-    *reinterpret_cast<float4*>(dst + r * stride + q4 * 4) = x;
-  }
-}
-
 // a_i <- a_i + mean over the group's heads of P[t, g, i], one token after the other (the order Algorithm 1 adds them
-// in).  Thread tid owns key k0 + tid of the tile; Pt is [key][row] with row = token_in_block * G + head.
-template <int G>
-__device__ __forceinline__ void fold_columns(const float* Pt, float* a_l, int k0, int t0, int nk, int n) {
+// in).  Thread tid < KT owns key k0 + tid of the tile; Pt is [key][row] with row = token_in_block * G + head; a_prev is
+// the key's score before this block (0 if the key's own token is in the block: it starts from [a, 0]).
+template <int G, int KT>
+__device__ __forceinline__ void fold_columns(const float* Pt, float* a_l, float a_prev, int k0, int t0, int nk, int n) {
   constexpr int BQ = kBulkRows / G;
   const int key = k0 + (int)threadIdx.x;
-  if (key >= nk) return;
-  float a_i = key >= t0 ? 0.f : a_l[key];                // the key's own token is in this block: it starts from [a, 0]
+  if ((int)threadIdx.x >= KT || key >= nk) return;
+  float a_i = a_prev;
   const float* pr = Pt + threadIdx.x * kBulkPadP;
 #pragma unroll
   for (int tok = 0; tok < BQ; ++tok) {
@@ -120,14 +113,23 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
-  constexpr int KS = D + 4;                      // padded row stride of the K / V tile: conflict-free 128-bit reads
+  constexpr int KT = BulkTile<T>::kKeys;         // keys per tile
+  constexpr int KPT = KT / 32;                   // keys per thread in the logits phase
+  constexpr int RS = D + 16 / (int)sizeof(T);    // row stride of a tile in elements: 16 bytes of padding, no bank conflicts
+  constexpr int ROWB = D * (int)sizeof(T);       // bytes per row
   constexpr int CPT = D / 32;                    // output channels per thread in the P.V phase (fp32 storage)
   constexpr bool kTensorPV = sizeof(T) == 2;     // bf16 storage: P.V on the tensor cores
-  static_assert(kBulkRows % G == 0 && kBulkThreads == kBulkKeys && kBulkThreads == 8 * kBulkRows, "thread maps");
-  extern __shared__ __align__(16) unsigned char bulk_smem[];
-  float* Qs = reinterpret_cast<float*>(bulk_smem);       // [16][D]
-  float* KV = Qs + kBulkRows * D;                        // [128][D + 4]: the K tile (phase 1), the V tile (phase 3)
-  float* Pt = KV + kBulkKeys * KS;                       // [128][20]: probabilities of the tile, [key][row]
+  constexpr int PS = KT + 8;                     // bf16 row stride of the hi / lo probability tiles
+  constexpr int QV = ROWB / 128;                 // 16-byte pieces of the query block per thread
+  static_assert(kBulkRows % G == 0 && kBulkThreads == 8 * kBulkRows && KT <= kBulkThreads && kBulkKeys % KT == 0, "thread maps");
+  extern __shared__ __align__(128) unsigned char bulk_smem[];
+  float* Qs = reinterpret_cast<float*>(bulk_smem);                       // [16][D] fp32
+  T* stage0 = reinterpret_cast<T*>(Qs + kBulkRows * D);                  // 2 x [KT][RS]
+  float* Pt = reinterpret_cast<float*>(stage0 + 2 * KT * RS);            // [KT][20]: probabilities, [key][row]
+  __nv_bfloat16* Ph = reinterpret_cast<__nv_bfloat16*>(Pt + KT * kBulkPadP);   // [16][KT + 8] (bf16 storage only)
+  __nv_bfloat16* Pl = Ph + kBulkRows * PS;
+  uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(Pt + KT * kBulkPadP) +
+                                               (kTensorPV ? 2 * kBulkRows * PS * 2 : 0));
 
   const int tid = threadIdx.x, w = tid >> 5, ln = tid & 31;
   const int lane_local = blockIdx.x;
@@ -149,9 +151,62 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
     for (int t = tid; t < P.n0; t += kBulkThreads) P.evicted[((long long)b * P.T_max + t) * Hk + hk] = -1;
   if (n == 0) return;
 
+  if (tid == 0) {
+    mbar_init(&full[0], KT);                             // every issuing thread arrives once per fill
+    mbar_init(&full[1], KT);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // The ring.  Thread r < KT fetches row r of a tile: one bulk copy, counted in bytes on the stage's barrier.  Rows
+  // beyond the last key of the block re-fetch that last key (finite values; their probabilities are exactly zero).
+  uint32_t parity = 0;                                   // bit s: parity of stage s's next completion
+  auto issue = [&](const T* base, int kt, int s, int nk_) {
+    if (tid < KT) {
+      const int r = min(kt * KT + tid, nk_ - 1);
+      mbar_expect_tx(&full[s], ROWB);
+      bulk_g2s(stage0 + (s * KT + tid) * RS, base + (long long)r * Hk * D, ROWB, &full[s]);
+    }
+  };
+  auto wait_stage = [&](int s) {
+    mbar_wait(&full[s], (parity >> s) & 1u, P.status);
+    parity ^= 1u << s;
+  };
+  // query rows of a block as 16-byte pieces in registers: piece c -> row c / (ROWB/16); row = token_in_block * G + head
+  uint4 qpre[QV];
+  auto load_q = [&](int t0_) {
+#pragma unroll
+    for (int i = 0; i < QV; ++i) {
+      const int c = tid + kBulkThreads * i;
+      const int r = c / (ROWB / 16), q = c % (ROWB / 16);
+      const int tok = t0_ + r / G, g = r % G;
+      qpre[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (tok < n) qpre[i] = reinterpret_cast<const uint4*>(Qb + ((long long)tok * Hq + g) * D)[q];
+    }
+  };
+  auto store_q = [&]() {
+#pragma unroll
+    for (int i = 0; i < QV; ++i) {
+      const int c = tid + kBulkThreads * i;
+      const int r = c / (ROWB / 16), q = c % (ROWB / 16);
+      if constexpr (sizeof(T) == 2) {
+        float* d = Qs + r * D + q * 8;
+        const uint4 t = qpre[i];
+        *reinterpret_cast<float4*>(d) = make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+                                                    __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+        *reinterpret_cast<float4*>(d + 4) = make_float4(__uint_as_float(t.z << 16), __uint_as_float(t.z & 0xffff0000u),
+                                                        __uint_as_float(t.w << 16), __uint_as_float(t.w & 0xffff0000u));
+      } else {
+        *reinterpret_cast<uint4*>(Qs + r * D + q * 4) = qpre[i];
+      }
+    }
+  };
+  load_q(0);
+  issue(Kb, 0, 0, min(BQ, n));
+  if (min(BQ, n) > KT) issue(Kb, 1, 1, min(BQ, n));
+
   // the cache after n uncompressed steps: token i in slot i, linked in order (Algorithm 1 appends, nothing is removed)
   {
-    constexpr int Q8 = D * (int)sizeof(T) / 16;          // 16-byte pieces per row
+    constexpr int Q8 = ROWB / 16;                        // 16-byte pieces per row
     for (int c = tid; c < n * Q8; c += kBulkThreads) {
       const int r = c / Q8, q = c % Q8;
       reinterpret_cast<uint4*>(Kl + (long long)r * D)[q] = reinterpret_cast<const uint4*>(Kb + (long long)r * Hk * D)[q];
@@ -177,7 +232,7 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
 
   for (int t0 = 0; t0 < n; t0 += BQ) {
     const int nk = min(t0 + BQ, n);                      // keys 0 .. nk-1 are visible to some row of the block
-    const int n_tiles = (nk + kBulkKeys - 1) / kBulkKeys;
+    const int n_tiles = (nk + KT - 1) / KT;
     int t_row[4];                                        // token of each of my 4 rows
     bool act[4];
 #pragma unroll
@@ -185,51 +240,44 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
       t_row[i] = t0 + (4 * w + i) / G;
       act[i] = t_row[i] < n;
     }
-    __syncthreads();                                     // the previous block is done with Qs, KV and Pt
-    // query rows of the block: row rho = token_in_block * G + head; rows of tokens at or beyond n are zero
-    for (int c = tid; c < kBulkRows * (D / 4); c += kBulkThreads) {
-      const int r = c / (D / 4), q4 = c % (D / 4);
-      const int tok = r / G, g = r % G;
-      float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (t0 + tok < n) x = load4(Qb + ((long long)(t0 + tok) * Hq + g) * D + q4 * 4);
-      *reinterpret_cast<float4*>(Qs + r * D + q4 * 4) = x;
-    }
+    store_q();                                           // (the previous block's last barrier freed Qs)
+    __syncthreads();
+    if (t0 + BQ < n) load_q(t0 + BQ);                    // next block's queries: in flight during this whole block
 
-    // ---- phase 1: logits of the row block, tile by tile --------------------------------------------------------
+    // ---- phase 1: logits of the row block, tile by tile (K tiles 0 and 1 are already in flight) -------------------
     float row_max[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
     for (int kt = 0; kt < n_tiles; ++kt) {
-      const int k0 = kt * kBulkKeys;
-      __syncthreads();
-      stage_rows<T, D>(KV, KS, Kb, (long long)Hk * D, k0, kBulkKeys, nk);
-      __syncthreads();
+      const int k0 = kt * KT, s = kt & 1;
+      wait_stage(s);
+      const T* Kt = stage0 + s * KT * RS;
       // The reproducible dot: 16 partial sums over blocks of D/16 channels (even- and odd-channel fma chains, added),
       // combined as the butterfly p_r + p_{r xor off}, off = 8, 4, 2, 1.  The blocks are visited in the order that
       // lets the butterfly's additions be done as soon as both operands exist (a fixed tree; fp addition commutes).
-      float st1[16], st2[16], st3[16], st4[16], dot[16];
+      float st1[4 * KPT], st2[4 * KPT], st3[4 * KPT], st4[4 * KPT], dot[4 * KPT];
 #pragma unroll
-      for (int s = 0; s < 16; ++s) {
-        const int blk = ((s & 1) << 3) | ((s & 2) << 1) | ((s & 4) >> 1) | ((s & 8) >> 3);   // 0,8,4,12,2,10,6,14,1,...
-        f32x2 qv[4][CP], kv[4][CP];
+      for (int sb = 0; sb < 16; ++sb) {
+        const int blk = ((sb & 1) << 3) | ((sb & 2) << 1) | ((sb & 4) >> 1) | ((sb & 8) >> 3);   // 0,8,4,12,2,10,6,14,1,...
+        f32x2 qv[4][CP], kv[KPT][CP];
 #pragma unroll
         for (int i = 0; i < 4; ++i) load_pairs<CP>(Qs + (4 * w + i) * D + blk * CH, qv[i]);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) load_pairs<CP>(KV + (ln + 32 * j) * KS + blk * CH, kv[j]);
+        for (int j = 0; j < KPT; ++j) load_pairs<CP>(Kt + (ln + 32 * j) * RS + blk * CH, kv[j]);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int o = i * 4 + j;
+          for (int j = 0; j < KPT; ++j) {
+            const int o = i * KPT + j;
             f32x2 acc = 0ull;
 #pragma unroll
             for (int e = 0; e < CP; ++e) acc = fma2(qv[i][e], kv[j][e], acc);
             float v = __fadd_rn(lo_of(acc), hi_of(acc));
-            if (s & 1) {
+            if (sb & 1) {
               v = __fadd_rn(st1[o], v);
-              if (s & 2) {
+              if (sb & 2) {
                 v = __fadd_rn(st2[o], v);
-                if (s & 4) {
+                if (sb & 4) {
                   v = __fadd_rn(st3[o], v);
-                  if (s & 8) dot[o] = __fadd_rn(st4[o], v);
+                  if (sb & 8) dot[o] = __fadd_rn(st4[o], v);
                   else st4[o] = v;
                 } else st3[o] = v;
               } else st2[o] = v;
@@ -240,26 +288,31 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < KPT; ++j) {
           const int key = k0 + ln + 32 * j;
           const bool ok = act[i] && key <= t_row[i];     // causal: the row's own token is its last key
-          const float sc = ok ? __fmul_rn(P.scale, dot[i * 4 + j]) : -INFINITY;
+          const float sc = ok ? __fmul_rn(P.scale, dot[i * KPT + j]) : -INFINITY;
           S[(long long)(4 * w + i) * P.s_stride + key] = sc;
           row_max[i] = fmaxf(row_max[i], sc);
         }
       }
+      __syncthreads();                                   // everybody is done with the stage
+      if (kt + 2 < n_tiles) issue(Kb, kt + 2, s, nk);
     }
+    // both stages are free: put the first V tiles in flight, they land while the exponentials are computed
+    issue(Vb, 0, 0, nk);
+    if (n_tiles > 1) issue(Vb, 1, 1, nk);
     // ---- phase 2: exponentials in place and the integer-sum normaliser (each thread re-reads what it wrote) ------
-    float M[4], Z[4];
+    float Z[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       float m = row_max[i];
 #pragma unroll
       for (int off = 16; off >= 1; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-      M[i] = m;
       unsigned long long z = 0ull;
       float* Srow = S + (long long)(4 * w + i) * P.s_stride;
-      for (int key = ln; key < n_tiles * kBulkKeys; key += 32) {
+#pragma unroll 4
+      for (int key = ln; key < n_tiles * KT; key += 32) {
         const float sc = Srow[key];
         const float e = (act[i] && sc != -INFINITY) ? repro_exp(__fsub_rn(sc, m)) : 0.f;
         Srow[key] = e;
@@ -269,51 +322,51 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
       Z[i] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
     }
     // ---- phase 3: probabilities, score accumulation, outputs -----------------------------------------------------
+    constexpr int NTW = D / 32;                          // tensor path: 8-channel n-tiles per warp
+    float cacc[kTensorPV ? NTW : 1][4];
+    f32x2 o_acc[kTensorPV ? 1 : 4][kTensorPV ? 1 : CPT / 2];
     if constexpr (kTensorPV) {
-      // bf16 storage: O += P . V on the tensor cores (the outputs are not part of the reproducible chain).  Warp w
-      // takes all 16 rows and channels [w*D/4, (w+1)*D/4); P goes in as a bf16 hi + lo pair per probability.
-      constexpr int NTW = D / 32;                        // 8-channel n-tiles per warp
-      constexpr int VS = D + 8;                          // bf16 row stride of the V tile: conflict-free ldmatrix
-      constexpr int PS = kBulkKeys + 8;                  // bf16 row stride of the P tiles
-      __nv_bfloat16* Vt = reinterpret_cast<__nv_bfloat16*>(KV);          // [128][D + 8]
-      __nv_bfloat16* Ph = Vt + kBulkKeys * VS;                           // [16][128 + 8] hi parts
-      __nv_bfloat16* Pl = Ph + kBulkRows * PS;                           // [16][128 + 8] lo parts
-      float cacc[NTW][4];
 #pragma unroll
       for (int nt = 0; nt < NTW; ++nt) cacc[nt][0] = cacc[nt][1] = cacc[nt][2] = cacc[nt][3] = 0.f;
-      for (int kt = 0; kt < n_tiles; ++kt) {
-        const int k0 = kt * kBulkKeys;
-        __syncthreads();
-        {
-          constexpr int Q8 = D / 8;                      // 16-byte pieces per row
-          for (int c = tid; c < kBulkKeys * Q8; c += kBulkThreads) {
-            const int r = c / Q8, q = c % Q8;
-            uint4 x = make_uint4(0u, 0u, 0u, 0u);        // keys beyond the block's range must be zeros, not stale bits
-            if (k0 + r < nk) x = reinterpret_cast<const uint4*>(Vb + (long long)(k0 + r) * Hk * D)[q];
-            *reinterpret_cast<uint4*>(Vt + r * VS + q * 8) = x;
-          }
-        }
+    } else {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int kk = ln + 32 * j;
-          float p[4];
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+        for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = 0ull;
+    }
+    for (int kt = 0; kt < n_tiles; ++kt) {
+      const int k0 = kt * KT, s = kt & 1;
+      const int my_key = k0 + tid;
+      const float a_prev = (tid < KT && my_key < nk && my_key < t0) ? a_l[my_key] : 0.f;
+#pragma unroll
+      for (int j = 0; j < KPT; ++j) {
+        const int kk = ln + 32 * j;
+        float p[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+          if constexpr (kTensorPV) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(p[i]);
             Ph[(4 * w + i) * PS + kk] = hi;
             Pl[(4 * w + i) * PS + kk] = __float2bfloat16_rn(p[i] - __bfloat162float(hi));
           }
-          *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
         }
-        __syncthreads();
-        fold_columns<G>(Pt, a_l, k0, t0, nk, n);
-        const int ksteps = (min(kBulkKeys, nk - k0) + 15) / 16;
-        // fragment addresses: A (P, row-major [row][key]): thread i -> row (i%8) + 8*((i/8)&1), key 8*(i/16);
-        //                     B (V, [key][channel], read transposed): thread i -> key (i%8) + 8*((i/8)&1), channel 8*(i/16)
-        const uint32_t a_off = (uint32_t)((((ln & 7) + ((ln >> 3) & 1) * 8) * PS + (ln >> 4) * 8) * 2);
+        *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
+      }
+      wait_stage(s);                                     // the V tile
+      __syncthreads();                                   // the probability tiles
+      const T* Vt = stage0 + s * KT * RS;
+      fold_columns<G, KT>(Pt, a_l, a_prev, k0, t0, nk, n);
+      if constexpr (kTensorPV) {
+        // O += P . V on the tensor cores (the outputs are not part of the reproducible chain).  Warp w takes all 16
+        // rows and channels [w*D/4, (w+1)*D/4).  Fragment addresses: A (P, row-major [row][key]): thread i -> row
+        // (i%8) + 8*((i/8)&1), key 8*(i/16); B (V, [key][channel], read transposed): thread i -> key (i%8) +
+        // 8*((i/8)&1), channel 8*(i/16).
+        const int ksteps = (min(KT, nk - k0) + 15) / 16;
+        const int frow = (ln & 7) + ((ln >> 3) & 1) * 8, fcol = (ln >> 4) * 8;
+        const uint32_t a_off = (uint32_t)((frow * PS + fcol) * 2);
         const uint32_t ph_base = smem_u32(Ph) + a_off, pl_base = smem_u32(Pl) + a_off;
-        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((((ln & 7) + ((ln >> 3) & 1) * 8) * VS + w * (D / 4) + (ln >> 4) * 8) * 2);
+        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((frow * RS + w * (D / 4) + fcol) * 2);
         for (int ks = 0; ks < ksteps; ++ks) {
           uint32_t ah[4], al[4];
           asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -325,15 +378,44 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
             uint32_t bf[4];
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                          : "=r"(bf[0]), "=r"(bf[1]), "=r"(bf[2]), "=r"(bf[3])
-                         : "r"(v_base + (uint32_t)(ks * 16 * VS * 2 + np * 32)) : "memory");
+                         : "r"(v_base + (uint32_t)(ks * 16 * RS * 2 + np * 32)) : "memory");
             mma_m16n8k16_bf16(cacc[2 * np], ah, bf[0], bf[1]);
             mma_m16n8k16_bf16(cacc[2 * np], al, bf[0], bf[1]);
             mma_m16n8k16_bf16(cacc[2 * np + 1], ah, bf[2], bf[3]);
             mma_m16n8k16_bf16(cacc[2 * np + 1], al, bf[2], bf[3]);
           }
         }
+      } else {
+        // fp32 storage: packed fp32 FMAs; warp w keeps its 4 rows, each thread CPT channels
+        const int kmax = min(KT, nk - k0);
+        for (int kk = 0; kk < kmax; ++kk) {
+          const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
+          const f32x2 pp[4] = {pack2(p4.x, p4.x), pack2(p4.y, p4.y), pack2(p4.z, p4.z), pack2(p4.w, p4.w)};
+          f32x2 vv[CPT / 2];
+          const float* vrow = reinterpret_cast<const float*>(Vt) + kk * RS + ln * CPT;
+          if constexpr (CPT == 4) {
+            load_pairs<2>(vrow, vv);
+          } else {
+            const float2 t = *reinterpret_cast<const float2*>(vrow);
+            vv[0] = pack2(t.x, t.y);
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = fma2(pp[i], vv[c], o_acc[i][c]);
+        }
       }
-      if (P.out != nullptr) {
+      __syncthreads();                                   // everybody is done with the stage and the probability tiles
+      if (kt + 2 < n_tiles) issue(Vb, kt + 2, s, nk);
+    }
+    // both stages are free again: the next block's first K tiles travel while this block's outputs are stored
+    if (t0 + BQ < n) {
+      const int nk_next = min(t0 + 2 * BQ, n);
+      issue(Kb, 0, 0, nk_next);
+      if (nk_next > KT) issue(Kb, 1, 1, nk_next);
+    }
+    if (P.out != nullptr) {
+      if constexpr (kTensorPV) {
         // accumulator fragment: rows ln/4 and ln/4 + 8, channels (ln%4)*2, +1 of each n-tile
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -347,47 +429,7 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
             store_row_part(dst + nt * 8, x);
           }
         }
-      }
-    } else {
-      // fp32 storage: packed fp32 FMAs; warp w keeps its 4 rows, each thread CPT channels
-      f32x2 o_acc[4][CPT / 2];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = 0ull;
-      for (int kt = 0; kt < n_tiles; ++kt) {
-        const int k0 = kt * kBulkKeys;
-        __syncthreads();
-        stage_rows<T, D>(KV, KS, Vb, (long long)Hk * D, k0, kBulkKeys, nk);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int kk = ln + 32 * j;
-          float p[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
-          *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
-        }
-        __syncthreads();
-        fold_columns<G>(Pt, a_l, k0, t0, nk, n);
-        const int kmax = min(kBulkKeys, nk - k0);
-        for (int kk = 0; kk < kmax; ++kk) {
-          const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
-          const f32x2 pp[4] = {pack2(p4.x, p4.x), pack2(p4.y, p4.y), pack2(p4.z, p4.z), pack2(p4.w, p4.w)};
-          f32x2 vv[CPT / 2];
-          if constexpr (CPT == 4) {
-            load_pairs<2>(KV + kk * KS + ln * 4, vv);
-          } else {
-            const float2 t = *reinterpret_cast<const float2*>(KV + kk * KS + ln * 2);
-            vv[0] = pack2(t.x, t.y);
-          }
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = fma2(pp[i], vv[c], o_acc[i][c]);
-        }
-      }
-      if (P.out != nullptr) {
+      } else {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           if (!act[i]) continue;
