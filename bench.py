@@ -146,7 +146,7 @@ def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
     n = min(n, one.budget)
     ctx = binding.Context(1, one.batch, one.n_q_heads, one.n_kv_heads, one.head_dim, one.budget, one.window, one.sink,
                           binding.WKV_F32 if one.dtype == "f32" else binding.WKV_BF16, device=dev)
-    Q, K, V = TokenStream(one, seed, dev).tokens(0, n)
+    Q, K, V = TokenStream(one, seed, dev).prompt(0, n)
     out = torch.empty(one.batch, n, one.n_q_heads, one.head_dim, dtype=one.torch_dtype, device=dev)
     times = []
     for _ in range(reps + 1):                      # the first run also takes the scratch from the allocator
@@ -154,7 +154,7 @@ def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        ctx.wkv_prefill_bulk(0, Q[0], K[0], V[0], None, out)
+        ctx.wkv_prefill_bulk(0, Q, K, V, None, out)
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
@@ -200,7 +200,7 @@ def workload_config(wl, args, splits):
     return {"workload": wl.name, "n_layers": wl.n_layers, "batch_per_gpu": wl.batch, "n_q_heads": wl.n_q_heads,
             "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "budget": wl.budget, "window": wl.window,
             "sink": wl.sink, "prefill_tokens": args.prefill_tokens if args.prefill_tokens else wl.budget + 64,
-            "prefill": "streamed through wkv_prefill until every cache is full and compressing" if args.init == "prefill"
+            "prefill": "wkv_prefill_bulk per layer (dense for the first budget tokens, the rest streamed) until every cache is full and compressing" if args.init == "prefill"
             else "synthetic full caches through wkv_import_state (profiling only)",
             "n_splits": splits, "l2": "inputs larger than L2 (cache rows streamed once per step)",
             "parallelism": f"lanes replicated per GPU x{args.gpus}, no collective"}
@@ -276,7 +276,6 @@ def main():
     # ragged prompt lengths in the last 32 tokens of the (shortened) prefill: every cache ends up full
     lens = sequence_lengths(wl.scaled(prefill=n_prefill, prefill_min=max(1, n_prefill - 32)), seed).to(dev)
     t = 0
-    chunk = 16
     if args.init == "import":
         g = torch.Generator().manual_seed(seed)
         m = wl.budget
@@ -290,13 +289,14 @@ def main():
                     ctx.wkv_import_state(layer, b, h, m, p1, a1, K1, V1)
         n_prefill = m
         t = n_prefill
-    while t < n_prefill:
-        tc = min(chunk, n_prefill - t)
-        Q, K, V = stream.tokens(t, tc)
-        rel = (lens - t).clamp(min=0, max=tc).to(torch.int32)
+    if t < n_prefill:
+        # the prompt, layer by layer: the first `budget` tokens through the dense kernel, the rest streamed behind it
+        rel = lens.clamp(max=n_prefill).to(torch.int32)
         for layer in range(wl.n_layers):
-            ctx.wkv_prefill(layer, Q[layer], K[layer], V[layer], rel)
-        t += tc
+            Q, K, V = stream.prompt(layer, n_prefill)
+            ctx.wkv_prefill_bulk(layer, Q, K, V, rel)
+            torch.cuda.synchronize()
+        t = n_prefill
     torch.cuda.synchronize()
     Q = K = V = None
 

@@ -134,3 +134,24 @@ class TokenStream:
         """n consecutive tokens, token-major per sequence: q [n_layers, B, n, Hq, d], k, v [n_layers, B, n, Hkv, d]."""
         qs, ks, vs = zip(*(self.token(t) for t in range(t0, t0 + n)))
         return torch.stack(qs, 2).contiguous(), torch.stack(ks, 2).contiguous(), torch.stack(vs, 2).contiguous()
+
+    def prompt(self, layer: int, n: int):
+        """A whole prompt of n tokens for ONE layer, token-major per sequence: q [B, n, Hq, d], k, v [B, n, Hkv, d].
+        Same distributions as token(), drawn with a few large calls (its own random stream, keyed by the layer)."""
+        wl, dev = self.wl, self.device
+        g = torch.Generator(device=dev)
+        g.manual_seed((self.seed * 1_000_003 + 7_000_000_007 + layer) & 0x7FFFFFFFFFFF)
+        B, Hq, Hk, d = wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+        q = torch.randn(B, n, Hq, d, generator=g, device=dev)
+        v = torch.randn(B, n, Hk, d, generator=g, device=dev)
+        if wl.key_rank > 0:
+            z = torch.randn(B, n, Hk, wl.key_rank, generator=g, device=dev)
+            k = torch.einsum("bnhr,hrd->bnhd", z, self.basis[layer])
+            k = k + wl.key_noise * torch.randn(B, n, Hk, d, generator=g, device=dev)
+        else:
+            k = torch.randn(B, n, Hk, d, generator=g, device=dev) * self.boost[layer][None, None]
+        if wl.unit_scale:
+            s = d ** -0.5
+            q, k, v = q * s, k * s, v * s
+        dt = wl.torch_dtype
+        return q.to(dt).contiguous(), k.to(dt).contiguous(), v.to(dt).contiguous()
