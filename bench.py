@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090291000 + 26968000 + 13558000, "2eaa22dea7b78f4e")}
+NCU_TRAFFIC = {"serving_b16": (1090237000 + 26969000 + 14676000, "5d2f45c1e50b2d8c")}
 
 
 def kernel_source_hash() -> str:
@@ -158,6 +158,15 @@ def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
         e1.record()
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1))
+    # the same prompt token by token (wkv_prefill: one decode launch per token), for scale
+    ctx.wkv_reset()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    ctx.wkv_prefill(0, Q, K, V, None, out)
+    e1.record()
+    torch.cuda.synchronize()
+    streamed_ms = e0.elapsed_time(e1)
     assert ctx.wkv_status() == 0
     ctx.close()
     ms = min(times[1:])
@@ -174,6 +183,7 @@ def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
     achieved = fma / (ms * 1e-3) / 1e12
     return {"value": one.batch * n / (ms * 1e-3), "unit": "prompt tokens/s per layer", "ms_per_layer": ms,
             "tokens_per_sequence": n, "kernel": "prefill_bulk_kernel",
+            "streamed_ms_per_layer": streamed_ms,
             "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "TFMA/s (fp32)", "frac": achieved / peak,
                          "traffic": None, "peak_kind": f"{props.multi_processor_count} SMs x {FP32_LANES_PER_SM} lanes x {max_mhz} MHz",
                          "algorithmic_fma_per_launch": fma}}

@@ -338,13 +338,20 @@ __global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const Prefil
       const int k0 = kt * KT, s = kt & 1;
       const int my_key = k0 + tid;
       const float a_prev = (tid < KT && my_key < nk && my_key < t0) ? a_l[my_key] : 0.f;
+      // all of the tile's exponentials first: the IEEE division below may call its slow path, and a call keeps the
+      // compiler from moving later loads ahead of it (one L2 round trip per value instead of one per tile)
+      float ev[KPT][4];
+#pragma unroll
+      for (int j = 0; j < KPT; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ev[j][i] = S[(long long)(4 * w + i) * P.s_stride + k0 + ln + 32 * j];
 #pragma unroll
       for (int j = 0; j < KPT; ++j) {
         const int kk = ln + 32 * j;
         float p[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          p[i] = act[i] ? __fdiv_rn(S[(long long)(4 * w + i) * P.s_stride + k0 + kk], Z[i]) : 0.f;
+          p[i] = act[i] ? __fdiv_rn(ev[j][i], Z[i]) : 0.f;
           if constexpr (kTensorPV) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(p[i]);
             Ph[(4 * w + i) * PS + kk] = hi;
