@@ -99,3 +99,22 @@ def test_bulk_prefill_llama7b_layer_shape():
     p.decode(64)
     p.compare_state()
     p.close()
+
+
+@pytest.mark.parametrize("name,n_sample", [("serving_b16", 6), ("gqa_b32", 4)])
+def test_bulk_prefill_full_budget_shapes(name, n_sample):
+    """Full batch, full budget and head layout of the large workloads (two of their layers): the whole dense phase
+    (4096 / 3277 tokens, 32 / 26 key tiles) plus a ragged streamed tail, sampled lanes against the oracle."""
+    wl = WORKLOADS[name].scaled(n_layers=2)
+    n_prompt = wl.budget + 48
+    rng = np.random.default_rng(5)
+    lens = rng.integers(wl.budget - 40, n_prompt + 1, wl.batch)        # some prompts end inside the dense phase
+    lens[0] = n_prompt
+    lens[1] = wl.budget - 33
+    p = Parity(wl, sample=n_sample, ragged=lens.tolist())
+    p.prefill(n_prompt, chunk=n_prompt, bulk=True)
+    p.compare_state()
+    p.decode(6)
+    p.compare_state()
+    p.close()
+    torch.cuda.empty_cache()
