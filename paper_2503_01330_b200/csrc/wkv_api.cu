@@ -323,9 +323,9 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
   return WKV_OK;
 }
 
-template <typename T, int D>
+template <typename T, int D, int KT>
 cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
-  constexpr int smem = wkv::bulk_smem_bytes<T, D>();
+  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT>();
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -333,10 +333,10 @@ cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStrea
     return cudaGetLastError();
   };
   switch (G) {
-    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1>);
-    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2>);
-    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4>);
-    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8>);
+    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT>);
+    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT>);
+    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT>);
+    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT>);
   }
   return cudaErrorInvalidValue;
 }
@@ -673,12 +673,19 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     P.scale = c->scale;
     P.status = c->status;
     cudaError_t e;
-    if (c->cfg.dtype == WKV_BF16)
-      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128>(c->group, P, c->lanes_per_layer, c->stream)
-                                 : launch_bulk<__nv_bfloat16, 64>(c->group, P, c->lanes_per_layer, c->stream);
-    else
-      e = c->cfg.head_dim == 128 ? launch_bulk<float, 128>(c->group, P, c->lanes_per_layer, c->stream)
-                                 : launch_bulk<float, 64>(c->group, P, c->lanes_per_layer, c->stream);
+    const int lanes = c->lanes_per_layer;
+    if (c->cfg.dtype == WKV_BF16) {
+      // 128-key tiles (two CTAs per SM) unless the layer has more lanes than that keeps busy
+      if (lanes <= 2 * c->sm_count)
+        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, lanes, c->stream)
+                                   : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, lanes, c->stream);
+      else
+        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64>(c->group, P, lanes, c->stream)
+                                   : launch_bulk<__nv_bfloat16, 64, 64>(c->group, P, lanes, c->stream);
+    } else {
+      e = c->cfg.head_dim == 128 ? launch_bulk<float, 128, 64>(c->group, P, lanes, c->stream)
+                                 : launch_bulk<float, 64, 64>(c->group, P, lanes, c->stream);
+    }
     c->launches += 1;
     if (e != cudaSuccess) return cuda_fail(c, e, "bulk prefill launch");
     c->fresh[layer] = 0;

@@ -50,12 +50,12 @@ struct PrefillParams {
   uint32_t* status;          // device status word (bounded waits report here)
 };
 
-// keys per tile: a tile row carries 16 bytes of padding, two tiles of rows live in shared memory
-template <typename T> struct BulkTile { static constexpr int kKeys = sizeof(T) == 2 ? 128 : 64; };
+// Keys per tile (a template parameter of the kernel): 64, or 128 for 2-byte storage.  Two tiles of padded rows live in
+// shared memory.  128-key tiles amortise the per-tile work better (4 x 4 outputs per thread, two CTAs per SM); 64-key
+// tiles let four CTAs share an SM, which wins once a layer has more lanes than two per SM.
 
-template <typename T, int D>
+template <typename T, int D, int KT>
 constexpr int bulk_smem_bytes() {
-  constexpr int KT = BulkTile<T>::kKeys;
   return kBulkRows * D * 4                                   // query rows, fp32
          + 2 * KT * (D * (int)sizeof(T) + 16)                // two tile stages, storage type, padded rows
          + KT * kBulkPadP * 4                                // probabilities of a tile, fp32
@@ -108,12 +108,11 @@ __device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], const uint32_t 
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kBulkThreads) prefill_bulk_kernel(const PrefillParams P) {
+template <typename T, int D, int G, int KT>
+__global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_kernel(const PrefillParams P) {
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
-  constexpr int KT = BulkTile<T>::kKeys;         // keys per tile
   constexpr int KPT = KT / 32;                   // keys per thread in the logits phase
   constexpr int RS = D + 16 / (int)sizeof(T);    // row stride of a tile in elements: 16 bytes of padding, no bank conflicts
   constexpr int ROWB = D * (int)sizeof(T);       // bytes per row
