@@ -171,7 +171,7 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
  * If the layer is not empty the whole prompt is streamed.  K, positions, accumulated scores and removed positions are
  * bit-identical to wkv_prefill's; outputs and merged values agree within rounding.
  * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider and
- * keeps them until wkv_destroy.  Q, K, V, out must be 16-byte aligned.  Asynchronous. */
+ * keeps them until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos);
 

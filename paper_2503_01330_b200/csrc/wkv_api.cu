@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstdint>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -648,6 +649,9 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
                      int32_t T_max, void* out, int32_t* evicted_pos) {
   int rc = check_prefill_args(c, layer, Q, K, V, T_max);
   if (rc != WKV_OK) return rc;
+  // the dense kernel moves rows with 16-byte bulk copies and vector loads / stores
+  if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15)
+    return fail(c, WKV_ERR_INVALID, "wkv_prefill_bulk: Q, K, V and out must be 16-byte aligned");
   int32_t n0 = 0;
   if (c->fresh[layer] && T_max > 0) {
     // Every lane of the layer is empty: the first min(T_max, budget) tokens compress nothing and go through the

@@ -90,6 +90,20 @@ def test_bulk_prefill_on_a_used_layer_streams():
     p.close()
 
 
+def test_bulk_prefill_rejects_misaligned_rows():
+    wl = small(batch=1, hq=2, hkv=2, d=64, dtype="bf16", m=16, W=2, rank=16)
+    ctx = binding.Context(1, 1, 2, 2, 64, 16, 2, dtype=binding.WKV_BF16)
+    buf = torch.zeros(1 * 8 * 2 * 64 + 8, dtype=torch.bfloat16, device="cuda:0")
+    good = buf[:1024].view(1, 8, 2, 64)
+    odd = buf[4:1028].view(1, 8, 2, 64)                 # 8 bytes past a 16-byte boundary
+    with pytest.raises(binding.WkvError) as e:
+        ctx.wkv_prefill_bulk(0, odd, good, good)
+    assert e.value.code == binding.WKV_ERR_INVALID
+    ctx.wkv_prefill_bulk(0, good, good, good)            # the context is still usable
+    assert ctx.wkv_status() == 0 and ctx.wkv_export_state(0, 0, 0)["len"] == 8
+    ctx.close()
+
+
 def test_bulk_prefill_llama7b_layer_shape():
     """32 heads x 128, bf16, budget 2048: 2048 dense + 2048 streamed prompt tokens, sampled lanes against the oracle."""
     wl = WORKLOADS["llama7b_layer"]
