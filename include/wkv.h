@@ -175,6 +175,19 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos);
 
+/* wkv_prefill_bulk for all layers of a prompt in one call (Algorithm 1 per lane; lanes of different layers are as
+ * independent as lanes of one layer).
+ *   Q device [n_layers, batch, T_max, n_q_heads, head_dim], K, V device [n_layers, batch, T_max, n_kv_heads, head_dim]
+ *   seq_lens device [batch] or NULL (shared by the layers); out like Q or NULL; evicted_pos device
+ *   [n_layers, batch, T_max, n_kv_heads] int32 or NULL.  Inputs and outputs must not overlap; 16-byte alignment as above.
+ * When no layer has consumed a token, the dense phase runs over the lanes of all layers at once if its scratch
+ * (64 * n_layers * lanes_per_layer * round_up(budget, 128) bytes) stays under 256 MB -- what a single sequence needs to
+ * fill the GPU -- and layer by layer otherwise.  The remaining tokens are streamed: one launch per token over the
+ * lanes of all layers where wkv_decode_step_layers does the same, else with the layers interleaved so that one layer's
+ * scan can run alongside the previous layer's lane epilogues.  Results equal wkv_prefill's. */
+int wkv_prefill_bulk_layers(wkv_ctx* ctx, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                            int32_t T_max, void* out, int32_t* evicted_pos);
+
 /* Copies one lane to HOST memory in position order and checks its bookkeeping (links form one chain of
  * `len` entries with strictly increasing positions); waits for the stream.  Any destination may be NULL.
  *   len, tokens : entries held / tokens consumed so far

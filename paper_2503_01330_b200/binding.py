@@ -29,7 +29,7 @@ class wkv_config(C.Structure):
 
 
 EXPORTS = ["wkv_config_error", "wkv_create", "wkv_destroy", "wkv_reset", "wkv_set_stream", "wkv_decode_step",
-           "wkv_decode_step_layers", "wkv_decode_step_static", "wkv_decode_step_host", "wkv_decode_step_layers_host", "wkv_prefill", "wkv_prefill_bulk", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
+           "wkv_decode_step_layers", "wkv_decode_step_static", "wkv_decode_step_host", "wkv_decode_step_layers_host", "wkv_prefill", "wkv_prefill_bulk", "wkv_prefill_bulk_layers", "wkv_export_state", "wkv_export_slots", "wkv_import_state",
            "wkv_status", "wkv_selftest_wait_timeout", "wkv_launch_count", "wkv_device_bytes", "wkv_splits", "wkv_strerror", "wkv_last_error"]
 
 _lib = None
@@ -57,6 +57,7 @@ def lib():
         L.wkv_decode_step_layers_host.argtypes = [vp, vp, vp, vp, vp, vp]
         L.wkv_prefill.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp]
         L.wkv_prefill_bulk.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp]
+        L.wkv_prefill_bulk_layers.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp]
         L.wkv_export_state.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.wkv_export_slots.argtypes = [vp, i32, i32, i32, vp]
         L.wkv_import_state.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -195,6 +196,11 @@ class Context:
         T_max = Q.shape[1]
         self._check(lib().wkv_prefill_bulk(self._h, layer, _dp(Q), _dp(K), _dp(V), _dp(seq_lens), T_max, _dp(out),
                                            _dp(evicted_pos)))
+
+    def wkv_prefill_bulk_layers(self, Q, K, V, seq_lens=None, out=None, evicted_pos=None):
+        T_max = Q.shape[2]
+        self._check(lib().wkv_prefill_bulk_layers(self._h, _dp(Q), _dp(K), _dp(V), _dp(seq_lens), T_max, _dp(out),
+                                                  _dp(evicted_pos)))
 
     def wkv_export_state(self, layer, b, kv_head):
         """Position-ordered host copy of one lane: dict(len, tokens, pos, a, K, V)."""

@@ -45,6 +45,7 @@ struct wkv_ctx {
   float* part[2] = {nullptr, nullptr};
   uint32_t* ticket[2] = {nullptr, nullptr};
   uint32_t* fused_ticket = nullptr;
+  int32_t* fused_seq_lens = nullptr;   // [n_layers * batch]: a caller's per-sequence lengths repeated for every layer
   int parity = 0;
   // what the previous layer call of this context wrote for the caller, and for which layer
   int last_layer = -1;
@@ -61,6 +62,7 @@ struct wkv_ctx {
   // layers have consumed no token since creation / the last reset
   float* bulk_S = nullptr;
   int bulk_stride = 0;
+  long long bulk_lanes = 0;     // lanes the scratch has rows for
   std::vector<char> fresh;
   std::vector<void*> owned;
   long long device_bytes = 0;
@@ -415,6 +417,7 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     T(take(c, &c->fused_logits, (size_t)c->lanes_total * G * cap * 4));
     T(take(c, &c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4));
     T(take(c, &c->fused_ticket, (size_t)c->lanes_total * 4));
+    T(take(c, &c->fused_seq_lens, (size_t)cfg->n_layers * cfg->batch * 4));
   }
   T(take(c, &c->status, 256));
   // staging holds one step of all layers (the host entry points copy through it)
@@ -645,6 +648,53 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
   return stream_tokens(c, layer, Q, K, V, seq_lens, 0, T_max, out, evicted_pos);
 }
 
+// The dense kernel over `lanes` consecutive lanes starting at lane0 (one layer, or all layers at once: to the kernel the
+// lanes of several layers are just more sequences).  Takes the scratch on first use / when more lanes are needed.
+static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void* Q, const void* K, const void* V,
+                        const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos) {
+  if (c->bulk_S == nullptr || c->bulk_lanes < lanes) {
+    c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
+    int rc = take(c, &c->bulk_S, (size_t)lanes * wkv::kBulkRows * c->bulk_stride * 4);
+    if (rc != WKV_OK) return rc;
+    c->bulk_lanes = lanes;
+  }
+  wkv::PrefillParams P;
+  std::memset(&P, 0, sizeof(P));
+  P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
+  P.lane_state = c->lane_state;
+  P.S = c->bulk_S;
+  P.Q = Q; P.K = K; P.V = V; P.out = out; P.evicted = evicted_pos; P.seq_lens = seq_lens;
+  P.batch = c->cfg.batch;
+  P.lane0 = (int)lane0;
+  P.n_kv_heads = c->cfg.n_kv_heads;
+  P.cap = c->cap;
+  P.T_max = T_max;
+  P.n0 = n0;
+  P.s_stride = c->bulk_stride;
+  P.scale = c->scale;
+  P.status = c->status;
+  cudaError_t e;
+  const int n = (int)lanes;
+  if (c->cfg.dtype == WKV_BF16) {
+    // 128-key tiles (two CTAs per SM) unless there are more lanes than that keeps busy
+    if (n <= 2 * c->sm_count)
+      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, n, c->stream)
+                                 : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, n, c->stream);
+    else
+      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64>(c->group, P, n, c->stream)
+                                 : launch_bulk<__nv_bfloat16, 64, 64>(c->group, P, n, c->stream);
+  } else {
+    e = c->cfg.head_dim == 128 ? launch_bulk<float, 128, 64>(c->group, P, n, c->stream)
+                               : launch_bulk<float, 64, 64>(c->group, P, n, c->stream);
+  }
+  c->launches += 1;
+  if (e != cudaSuccess) return cuda_fail(c, e, "bulk prefill launch");
+  c->last_layer = -1;                    // the next scan of this context waits for this kernel before anything else
+  g_last_launcher.store(nullptr);
+  note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+  return WKV_OK;
+}
+
 int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos) {
   int rc = check_prefill_args(c, layer, Q, K, V, T_max);
@@ -657,47 +707,117 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     // Every lane of the layer is empty: the first min(T_max, budget) tokens compress nothing and go through the
     // dense kernel; the rest of the prompt is streamed behind it on the same stream.
     n0 = std::min(T_max, c->cfg.budget);
-    if (c->bulk_S == nullptr) {
-      c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
-      rc = take(c, &c->bulk_S, (size_t)c->lanes_per_layer * wkv::kBulkRows * c->bulk_stride * 4);
-      if (rc != WKV_OK) return rc;
-    }
-    wkv::PrefillParams P;
-    std::memset(&P, 0, sizeof(P));
-    P.Kc = c->Kc; P.Vc = c->Vc; P.a = c->a; P.pos = c->pos; P.next = c->next; P.prev = c->prev;
-    P.lane_state = c->lane_state;
-    P.S = c->bulk_S;
-    P.Q = Q; P.K = K; P.V = V; P.out = out; P.evicted = evicted_pos; P.seq_lens = seq_lens;
-    P.lane0 = layer * c->lanes_per_layer;
-    P.n_kv_heads = c->cfg.n_kv_heads;
-    P.cap = c->cap;
-    P.T_max = T_max;
-    P.n0 = n0;
-    P.s_stride = c->bulk_stride;
-    P.scale = c->scale;
-    P.status = c->status;
-    cudaError_t e;
-    const int lanes = c->lanes_per_layer;
-    if (c->cfg.dtype == WKV_BF16) {
-      // 128-key tiles (two CTAs per SM) unless the layer has more lanes than that keeps busy
-      if (lanes <= 2 * c->sm_count)
-        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, lanes, c->stream)
-                                   : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, lanes, c->stream);
-      else
-        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64>(c->group, P, lanes, c->stream)
-                                   : launch_bulk<__nv_bfloat16, 64, 64>(c->group, P, lanes, c->stream);
-    } else {
-      e = c->cfg.head_dim == 128 ? launch_bulk<float, 128, 64>(c->group, P, lanes, c->stream)
-                                 : launch_bulk<float, 64, 64>(c->group, P, lanes, c->stream);
-    }
-    c->launches += 1;
-    if (e != cudaSuccess) return cuda_fail(c, e, "bulk prefill launch");
+    rc = launch_dense(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, Q, K, V, seq_lens, T_max, n0, out,
+                      evicted_pos);
+    if (rc != WKV_OK) return rc;
     c->fresh[layer] = 0;
-    c->last_layer = -1;                  // the next scan of this context waits for this kernel before anything else
-    g_last_launcher.store(nullptr);
-    note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
   }
   return stream_tokens(c, layer, Q, K, V, seq_lens, n0, T_max, out, evicted_pos);
+}
+
+int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
+                            int32_t T_max, void* out, int32_t* evicted_pos) {
+  int rc = check_prefill_args(c, 0, Q, K, V, T_max);
+  if (rc != WKV_OK) return rc;
+  if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15)
+    return fail(c, WKV_ERR_INVALID, "wkv_prefill_bulk_layers: Q, K, V and out must be 16-byte aligned");
+  const long long D = c->cfg.head_dim, Hq = c->cfg.n_q_heads, Hk = c->cfg.n_kv_heads, B = c->cfg.batch;
+  const int L = c->cfg.n_layers;
+  const size_t q_layer = (size_t)B * T_max * Hq * D * c->elem, kv_layer = (size_t)B * T_max * Hk * D * c->elem;
+  const size_t ev_layer = (size_t)B * T_max * Hk;
+  if (ranges_overlap(Q, q_layer * L, out, q_layer * L) || ranges_overlap(K, kv_layer * L, out, q_layer * L) ||
+      ranges_overlap(V, kv_layer * L, out, q_layer * L) || ranges_overlap(Q, q_layer * L, evicted_pos, ev_layer * 4 * L) ||
+      ranges_overlap(K, kv_layer * L, evicted_pos, ev_layer * 4 * L) || ranges_overlap(V, kv_layer * L, evicted_pos, ev_layer * 4 * L))
+    return fail(c, WKV_ERR_INVALID, "wkv_prefill_bulk_layers: inputs and outputs must not overlap");
+  bool all_fresh = true;
+  for (int l = 0; l < L; ++l) all_fresh = all_fresh && c->fresh[l];
+  int32_t n0 = 0;
+  if (all_fresh && T_max > 0) {
+    n0 = std::min(T_max, c->cfg.budget);
+    const int stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
+    const size_t need_all = (size_t)c->lanes_total * wkv::kBulkRows * stride * 4;
+    if (need_all <= ((size_t)256 << 20)) {
+      // every lane of every layer in one launch
+      rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos);
+      if (rc != WKV_OK) return rc;
+    } else {
+      for (int l = 0; l < L; ++l) {
+        rc = launch_dense(c, (long long)l * c->lanes_per_layer, c->lanes_per_layer, (const char*)Q + l * q_layer,
+                          (const char*)K + l * kv_layer, (const char*)V + l * kv_layer, seq_lens, T_max, n0,
+                          out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr);
+        if (rc != WKV_OK) return rc;
+      }
+    }
+    c->fresh.assign((size_t)L, 0);
+  } else if (!all_fresh) {
+    // some layer already holds tokens: nothing is known to be uncompressed, stream everything
+    n0 = 0;
+  }
+  // The rest of the prompt, token by token with the layers interleaved: consecutive launches then belong to different
+  // layers, and since every input of this call existed before it was issued, a layer's scan may overlap the previous
+  // layer's lane epilogues.
+  if (n0 < T_max) c->fresh.assign((size_t)L, 0);
+  c->last_layer = -1;
+  if (c->fused_ok && n0 < T_max) {
+    // a layer alone cannot fill the GPU: one launch (pair) per token over the lanes of all layers, as in
+    // wkv_decode_step_layers; [n_layers, batch, ...] is [n_layers * batch, ...] to the kernels
+    if (seq_lens != nullptr)
+      for (int l = 0; l < L; ++l)
+        WKV_CUDA(c, cudaMemcpyAsync(c->fused_seq_lens + (size_t)l * B, seq_lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, c->stream));
+    wkv::StepParams P = base_params(c, 0);
+    P.n_splits = c->fused_splits;
+    P.chunk_cap = c->fused_chunk_cap;
+    P.logits = c->fused_logits;
+    P.part = c->fused_part;
+    P.ticket = c->fused_ticket;
+    P.seq_lens = seq_lens != nullptr ? c->fused_seq_lens : nullptr;
+    P.q_bs = (long long)T_max * Hq * D;
+    P.kv_bs = (long long)T_max * Hk * D;
+    P.out_bs = out ? P.q_bs : Hq * D;
+    P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
+    P.wait_at_start = 2;
+    g_last_launcher.store(c);
+    for (int t = n0; t < T_max; ++t) {
+      P.tok_idx = t;
+      P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
+      P.k = (const char*)K + (size_t)t * Hk * D * c->elem;
+      P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
+      P.out = out ? (void*)((char*)out + (size_t)t * Hq * D * c->elem) : c->stage_out;
+      P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
+      cudaError_t e = launch_any(c, P, c->fused_cluster, (int)c->lanes_total);
+      c->launches += c->fused_cluster ? 1 : 2;
+      if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (prefill, all layers at once)");
+    }
+    note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+    return WKV_OK;
+  }
+  for (int t = n0; t < T_max; ++t) {
+    for (int l = 0; l < L; ++l) {
+      wkv::StepParams P = base_params(c, l);
+      P.seq_lens = seq_lens;
+      P.q_bs = (long long)T_max * Hq * D;
+      P.kv_bs = (long long)T_max * Hk * D;
+      P.out_bs = out ? P.q_bs : Hq * D;
+      P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
+      P.tok_idx = t;
+      P.q = (const char*)Q + l * q_layer + (size_t)t * Hq * D * c->elem;
+      P.k = (const char*)K + l * kv_layer + (size_t)t * Hk * D * c->elem;
+      P.v = (const char*)V + l * kv_layer + (size_t)t * Hk * D * c->elem;
+      P.out = out ? (void*)((char*)out + l * q_layer + (size_t)t * Hq * D * c->elem)
+                  : (void*)((char*)c->stage_out + (size_t)l * B * Hq * D * c->elem);
+      P.evicted = evicted_pos ? evicted_pos + l * ev_layer + (size_t)t * Hk : c->stage_ev + (size_t)l * c->lanes_per_layer;
+      // As in wkv_decode_step_layers, the first layer of every token waits for everything before it (the same lanes
+      // were written one token ago); the layers behind it start once its units are in scratch, hence after that wait.
+      if (l == 0) c->last_layer = -1;
+      if (!c->use_cluster) prepare_overlap(c, P, l, 0, 0, true);
+      cudaError_t e = launch_any(c, P, c->use_cluster);
+      c->launches += c->use_cluster ? 1 : 2;
+      if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (prefill, all layers)");
+    }
+  }
+  c->last_layer = -1;
+  note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+  return WKV_OK;
 }
 
 int wkv_export_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* len, int32_t* tokens, int32_t* pos,

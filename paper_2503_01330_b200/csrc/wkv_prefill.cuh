@@ -37,12 +37,13 @@ struct PrefillParams {
   int32_t* prev;
   int32_t* lane_state;
   float* S;                  // [lanes of the layer][kBulkRows][s_stride] logits, then exponentials
-  const void* Q;             // [batch, T_max, n_q_heads, D]
+  const void* Q;             // [batch, T_max, n_q_heads, D] ([n_layers * batch, ...] for a launch over all layers)
   const void* K;             // [batch, T_max, n_kv_heads, D]
   const void* V;
   void* out;                 // [batch, T_max, n_q_heads, D] or null
   int32_t* evicted;          // [batch, T_max, n_kv_heads] or null
   const int32_t* seq_lens;   // [batch] or null
+  int batch;                 // sequences per layer: a launch over several layers indexes seq_lens by b % batch
   int lane0, n_kv_heads, cap, T_max;
   int n0;                    // tokens this kernel covers at most: min(T_max, budget)
   int s_stride;              // multiple of kBulkKeys, >= n0
@@ -136,7 +137,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   const long long lane = (long long)P.lane0 + lane_local;
   const int Hk = P.n_kv_heads, Hq = Hk * G;
   int n = P.n0;
-  if (P.seq_lens != nullptr) n = min(n, max(0, P.seq_lens[b]));
+  if (P.seq_lens != nullptr) n = min(n, max(0, P.seq_lens[b % P.batch]));
   const T* Qb = reinterpret_cast<const T*>(P.Q) + ((long long)b * P.T_max * Hq + (long long)hk * G) * D;   // + t*Hq*D + g*D
   const T* Kb = reinterpret_cast<const T*>(P.K) + ((long long)b * P.T_max * Hk + hk) * D;                  // + t*Hk*D
   const T* Vb = reinterpret_cast<const T*>(P.V) + ((long long)b * P.T_max * Hk + hk) * D;

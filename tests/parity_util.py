@@ -84,7 +84,7 @@ class Parity:
         return qs.cpu(), k[self.li, self.bi, self.hi].cpu(), v[self.li, self.bi, self.hi].cpu()
 
     # ---- prefill through wkv_prefill, chunked ------------------------------------------------------
-    def prefill(self, n_tokens, chunk=32, compare=True, bulk=False):
+    def prefill(self, n_tokens, chunk=32, compare=True, bulk=False, all_layers=False):
         wl = self.wl
         lens_dev = self.lens.to(self.dev)
         t_end = self.t + n_tokens
@@ -94,7 +94,9 @@ class Parity:
             rel = (lens_dev - self.t).clamp(min=0, max=tc).to(torch.int32)
             out = torch.empty(wl.n_layers, wl.batch, tc, wl.n_q_heads, wl.head_dim, dtype=wl.torch_dtype, device=self.dev)
             ev = torch.empty(wl.n_layers, wl.batch, tc, wl.n_kv_heads, dtype=torch.int32, device=self.dev)
-            for layer in range(wl.n_layers):
+            if all_layers:
+                self.ctx.wkv_prefill_bulk_layers(Q, K, V, rel, out, ev)
+            for layer in range(0 if all_layers else wl.n_layers):
                 (self.ctx.wkv_prefill_bulk if bulk else self.ctx.wkv_prefill)(layer, Q[layer], K[layer], V[layer], rel,
                                                                               out[layer], ev[layer])
             Qs = Q.view(wl.n_layers, wl.batch, tc, wl.n_kv_heads, wl.group, wl.head_dim)[self.li, self.bi, :, self.hi].cpu()

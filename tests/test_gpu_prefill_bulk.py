@@ -132,3 +132,65 @@ def test_bulk_prefill_full_budget_shapes(name, n_sample):
     p.compare_state()
     p.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("layers,batch,m,T,schedule", [(3, 2, 60, 150, binding.WKV_SCHEDULE_SPLIT), (2, 1, 40, 90, binding.WKV_SCHEDULE_SPLIT),
+                                                       (1, 2, 33, 70, binding.WKV_SCHEDULE_SPLIT), (4, 1, 50, 50, binding.WKV_SCHEDULE_CLUSTER)])
+def test_all_layers_prompt_call_matches_per_layer_calls(layers, batch, m, T, schedule):
+    """wkv_prefill_bulk_layers (dense phase over the lanes of all layers, streamed tail with the layers interleaved)
+    against wkv_prefill layer by layer: identical state, removed positions and (bf16-rounded) outputs."""
+    wl = small(layers=layers, batch=batch, hq=4, hkv=2, d=128, dtype="bf16", m=m, W=4, rank=16)
+    st = TokenStream(wl, 77, "cuda:0")
+    Q, K, V = st.tokens(0, T)
+    lens = torch.tensor([T, max(1, T - 37)][:batch], dtype=torch.int32, device="cuda:0")
+    res = []
+    for all_layers in (False, True):
+        ctx = binding.Context(layers, batch, 4, 2, 128, m, 4, dtype=binding.WKV_BF16, schedule=schedule, n_splits=2)
+        out = torch.zeros(layers, batch, T, 4, 128, dtype=torch.bfloat16, device="cuda:0")
+        ev = torch.full((layers, batch, T, 2), -7, dtype=torch.int32, device="cuda:0")
+        if all_layers:
+            ctx.wkv_prefill_bulk_layers(Q, K, V, lens, out, ev)
+        else:
+            for layer in range(layers):
+                ctx.wkv_prefill(layer, Q[layer], K[layer], V[layer], lens, out[layer], ev[layer])
+        assert ctx.wkv_status() == 0
+        res.append(([ctx.wkv_export_state(l, b, h) for l in range(layers) for b in range(batch) for h in range(2)],
+                    out.float().cpu(), ev.cpu()))
+        ctx.close()
+    for s0, s1 in zip(res[0][0], res[1][0]):
+        assert s0["len"] == s1["len"] and s0["tokens"] == s1["tokens"]
+        for key in ("pos", "a", "K", "V"):
+            assert torch.equal(s0[key], s1[key]), key
+    assert torch.equal(res[0][2], res[1][2])
+    torch.testing.assert_close(res[1][1], res[0][1], rtol=2e-2, atol=1e-3)
+
+
+def test_all_layers_prompt_paper_cache_setting():
+    """The paper's 256-entry cache (4 initial tokens, 124 recent) on the Llama-2-7B KV shape, one sequence: a
+    1024-token prompt for all 32 layers in one call (dense phase over 1024 lanes, then one launch per token over all
+    layers), sampled lanes against the oracle, then decode."""
+    wl = WORKLOADS["paper_cache256"]
+    p = Parity(wl, sample=10, ragged=[1024])
+    p.prefill(1024, chunk=1024, all_layers=True)
+    p.compare_state()
+    p.decode(12, layers_entry=True)
+    p.compare_state()
+    p.close()
+
+
+def test_all_layers_prompt_many_lanes_interleaves_layers():
+    """16 layers of the serving shape at half its budget (8192 lanes, 72 MB of logit scratch): too much for one launch
+    over all layers, so the dense phase runs layer by layer and the streamed tail interleaves the layers (a layer's scan
+    alongside the previous layer's epilogues)."""
+    wl = WORKLOADS["serving_b16"].scaled(n_layers=16, budget=2048, window=64)
+    n_prompt = wl.budget + 40
+    lens = [n_prompt - (3 * i) % 50 for i in range(wl.batch)]
+    lens[0] = n_prompt
+    p = Parity(wl, sample=8, ragged=lens)
+    assert p.ctx.wkv_device_bytes() > 0
+    p.prefill(n_prompt, chunk=n_prompt, all_layers=True)
+    p.compare_state()
+    p.decode(6)
+    p.compare_state()
+    p.close()
+    torch.cuda.empty_cache()
