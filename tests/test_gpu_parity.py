@@ -213,3 +213,53 @@ def test_two_contexts_interleaved_on_one_stream():
     pb.compare_state()
     pa.close()
     pb.close()
+
+
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+def test_decode_steps_replayed_from_a_cuda_graph(schedule):
+    """wkv_decode_step neither allocates nor synchronises, so a step (all layers) can be captured once and replayed:
+    the replayed steps must leave the same outputs and state as the same steps issued call by call."""
+    wl = small(layers=4, batch=2, hq=4, hkv=2, d=128, dtype="bf16", m=80, W=8, rank=16)
+    dev = torch.device("cuda:0")
+    from paper_2503_01330_b200.synth import TokenStream
+    res = {}
+    for mode in ("calls", "graph"):
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            ctx = binding.Context(4, 2, 4, 2, 128, 80, 8, dtype=binding.WKV_BF16, schedule=schedule, n_splits=2)
+            st = TokenStream(wl, 3, dev)
+            q = torch.empty(4, 2, 4, 128, dtype=torch.bfloat16, device=dev)
+            k = torch.empty(4, 2, 2, 128, dtype=torch.bfloat16, device=dev)
+            v = torch.empty_like(k)
+            out = torch.empty_like(q)
+            ev = torch.empty(4, 2, 2, dtype=torch.int32, device=dev)
+
+            def step():
+                for layer in range(4):
+                    ctx.wkv_decode_step(layer, q[layer], k[layer], v[layer], out[layer], ev[layer])
+
+            graph, outs, evs = None, [], []
+            for t in range(130):
+                a, b, c = st.token(t)
+                q.copy_(a); k.copy_(b); v.copy_(c)
+                if mode == "graph" and t == 2:
+                    s.synchronize()
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=s):
+                        step()
+                if graph is not None:
+                    graph.replay()
+                else:
+                    step()
+                outs.append(out.float().clone())
+                evs.append(ev.clone())
+            s.synchronize()
+            assert ctx.wkv_status() == 0
+            res[mode] = (torch.stack(outs), torch.stack(evs),
+                         [ctx.wkv_export_state(l, b, h) for l in range(4) for b in range(2) for h in range(2)])
+            ctx.close()
+    assert torch.equal(res["calls"][0], res["graph"][0]) and torch.equal(res["calls"][1], res["graph"][1])
+    assert int((res["graph"][1] >= 0).sum()) == 16 * (130 - 80)
+    for x, y in zip(res["calls"][2], res["graph"][2]):
+        for key in ("pos", "a", "K", "V"):
+            assert torch.equal(x[key], y[key]), key
