@@ -201,13 +201,15 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
   lc.blockDim = dim3(wkv::kThreads);
   lc.dynamicSmemBytes = (size_t)smem;
   lc.stream = stream;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = (unsigned)P.n_splits;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // the kernel waits for its predecessor first thing
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   lc.attrs = at;
-  lc.numAttrs = 1;
+  lc.numAttrs = 2;
   return cudaLaunchKernelEx(&lc, wkv::decode_step_cluster_kernel<T, D, G>, P);
 }
 

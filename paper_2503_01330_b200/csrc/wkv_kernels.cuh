@@ -1066,6 +1066,11 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
   const int split = (int)cluster.block_rank();
   const int lane_local = blockIdx.x / S;
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  // Launched with programmatic stream serialization: the next kernel in the stream may be made resident as soon as
+  // every CTA of this grid has started (that hides its launch latency behind this grid's tail, which matters when a
+  // step is a few microseconds long); this grid touches nothing before its predecessor has completed.
+  griddep_launch();
+  griddep_wait();
   if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {      // sequence already consumed: same decision in every CTA
     if (split == 0 && tid == 0 && P.evicted) P.evicted[b * P.ev_bs + hk] = -1;
     return;
