@@ -13,8 +13,8 @@ from parity_util import Parity
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,n_sample,decode,schedule", [("llama7b_b8", 12, 16, 0), ("serving_b16", 12, 12, 0),
-                                                           ("gqa_b32", 10, 8, 0), ("llama7b_b8", 6, 8, 2)])
+@pytest.mark.parametrize("name,n_sample,decode,schedule", [("llama7b_b8", 12, 256, 0), ("serving_b16", 12, 96, 0),
+                                                           ("gqa_b32", 10, 64, 0), ("llama7b_b8", 6, 8, 2)])
 def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     wl = WORKLOADS[name]
     n_prefill = wl.budget + 160
