@@ -189,12 +189,18 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t k2 = {};
     k2.gridDim = dim3((unsigned)lanes);
-    k2.blockDim = dim3(wkv::kEpilogueThreads);
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const bool wide = G <= 2 && lanes <= 2 * sms;        // two wide CTAs per SM hold every lane at once
+    k2.blockDim = dim3(wide ? wkv::kEpilogueThreadsWide : wkv::kEpilogueThreads);
     k2.dynamicSmemBytes = 0;
     k2.stream = stream;
     k2.attrs = pdl;
     k2.numAttrs = 1;
-    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G>, P);
+    if constexpr (G <= 2) {
+      if (wide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P);
+    }
+    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P);
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)n_ctas);

@@ -990,9 +990,12 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
 }
 
 constexpr int kEpilogueThreads = 256;
+constexpr int kEpilogueThreadsWide = 512;     // one or two query heads only (registers: two CTAs per SM)
 
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kEpilogueThreads) lane_epilogue_kernel(const StepParams P) {
+// NT threads per lane: kEpilogueThreads, or kEpilogueThreadsWide when a layer has so few lanes that two wide CTAs per
+// SM still hold them all -- the epilogue is a chain of load -> compute rounds, and twice the threads halve the rounds.
+template <typename T, int D, int G, int NT>
+__global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
   __shared__ __align__(16) unsigned char ep_raw[EpScratch::bytes(G)];
   EpScratch ep;
   ep.carve(ep_raw, G);
@@ -1040,7 +1043,7 @@ __global__ void __launch_bounds__(kEpilogueThreads) lane_epilogue_kernel(const S
       return;
     }
   }
-  lane_epilogue_from_scratch<T, D, G, kEpilogueThreads>(P, v, ep);
+  lane_epilogue_from_scratch<T, D, G, NT>(P, v, ep);
   if (P.ticket != nullptr) {
     if (threadIdx.x == 0) P.ticket[lane_local] = 0u;     // ready for the next call that uses this scratch set
     griddep_wait();                                      // keeps "this grid complete => the scan complete" literally true
