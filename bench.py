@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090275000 + 26967000 + 12748000, "09218991ad536df5")}
+NCU_TRAFFIC = {"serving_b16": (1090369000 + 26967000 + 12972000, "72f613a05dcec82c")}
 
 
 def kernel_source_hash() -> str:
