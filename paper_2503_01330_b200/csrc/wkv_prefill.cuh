@@ -394,6 +394,13 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         }
       } else {
         // fp32 storage: packed fp32 FMAs; warp w keeps its 4 rows, each thread CPT channels
+        // the tile's products are summed on their own and then added to the running output: thousands of keys in one
+        // sequential fp32 chain would cost more accuracy than the 1e-5 output tolerance leaves
+        f32x2 o_tile[4][CPT / 2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int c = 0; c < CPT / 2; ++c) o_tile[i][c] = 0ull;
         const int kmax = min(KT, nk - k0);
         for (int kk = 0; kk < kmax; ++kk) {
           const float4 p4 = *reinterpret_cast<const float4*>(Pt + kk * kBulkPadP + 4 * w);
@@ -409,8 +416,13 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
 #pragma unroll
           for (int i = 0; i < 4; ++i)
 #pragma unroll
-            for (int c = 0; c < CPT / 2; ++c) o_acc[i][c] = fma2(pp[i], vv[c], o_acc[i][c]);
+            for (int c = 0; c < CPT / 2; ++c) o_tile[i][c] = fma2(pp[i], vv[c], o_tile[i][c]);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int c = 0; c < CPT / 2; ++c)
+            o_acc[i][c] = pack2(lo_of(o_acc[i][c]) + lo_of(o_tile[i][c]), hi_of(o_acc[i][c]) + hi_of(o_tile[i][c]));
       }
       __syncthreads();                                   // everybody is done with the stage and the probability tiles
       if (kt + 2 < n_tiles) issue(Vb, kt + 2, s, nk);

@@ -194,3 +194,18 @@ def test_all_layers_prompt_many_lanes_interleaves_layers():
     p.compare_state()
     p.close()
     torch.cuda.empty_cache()
+
+
+def test_large_budget_dense_prompt_then_decode():
+    """A budget of 8192 entries (256 cache tiles per lane, 128 key tiles in the dense phase), fp32: the whole budget
+    filled by the dense kernel, then decode steps that compress, every token against the oracle.  With thousands of
+    keys per output the 1e-5 output tolerance only holds if the products are not summed in one sequential chain."""
+    wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=8192, W=32)
+    p = Parity(wl, seed=123, ragged=[8192])
+    assert p.ctx.wkv_splits() > 1
+    p.prefill(8192, chunk=8192, bulk=True)
+    p.compare_state()
+    p.decode(24)
+    p.compare_state()
+    assert p.n_evictions == wl.lanes * 24
+    p.close()
