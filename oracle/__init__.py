@@ -58,6 +58,8 @@ def lib():
         L.wkvo_dropped_score.argtypes = [C.c_void_p, C.c_int32]
         L.wkvo_last_step.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 4
         L.wkvo_export.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 7
+        L.wkvo_import.restype = C.c_int32
+        L.wkvo_import.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int64] + [C.c_void_p] * 4
         L.wkvo_pinned_exp.restype = C.c_float
         L.wkvo_pinned_exp.argtypes = [C.c_float]
         L.wkvo_pinned_dot.restype = C.c_float
@@ -127,6 +129,16 @@ class Oracle:
         wj, wr, ps = C.c_double(), C.c_double(), C.c_double()
         lib().wkvo_last_step(self._h, lane, C.byref(idx), C.byref(wj), C.byref(wr), C.byref(ps))
         return idx.value, wj.value, wr.value, ps.value
+
+    def import_state(self, lane, tokens, pos, a, K, V):
+        """Replace one lane by a position-ordered state (pos int32 strictly increasing and < tokens; K, V as stored)."""
+        pos = np.ascontiguousarray(pos, np.int32)
+        a = np.ascontiguousarray(a, np.float64)
+        K = np.ascontiguousarray(K, np.float32)
+        V = np.ascontiguousarray(V, np.float32)
+        rc = lib().wkvo_import(self._h, lane, len(pos), int(tokens), _ptr(pos), _ptr(a), _ptr(K), _ptr(V))
+        if rc != 0:
+            raise ValueError("wkvo_import rejected the state")
 
     def export(self, lane=0, coeff=False):
         """Position-ordered state of one lane as a dict of numpy arrays."""

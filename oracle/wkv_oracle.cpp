@@ -396,6 +396,29 @@ void wkvo_export(const wkvo* o, int32_t lane, int32_t* pos, int64_t* n, double* 
   }
 }
 
+// Replaces a lane by the given position-ordered state (test set-up for large caches: filling them token by token
+// would take the tests minutes).  tokens = tokens consumed so far; Algorithm 1's count of entry i is then
+// tokens - pos[i].  Multiplicities restart at 1; not available with coefficient tracking.
+int32_t wkvo_import(wkvo* o, int32_t lane, int32_t len, int64_t tokens, const int32_t* pos, const double* a, const float* K,
+                    const float* V) {
+  if (o->cfg.track || len < 0 || len > o->cfg.budget || tokens < len) return -1;
+  Lane& S = o->lanes[lane];
+  const int d = o->cfg.head_dim;
+  S = Lane();
+  S.t = tokens;
+  for (int32_t i = 0; i < len; ++i) {
+    if (pos[i] < 0 || pos[i] >= tokens || (i > 0 && pos[i] <= pos[i - 1])) return -1;
+    S.K.emplace_back(K + (size_t)i * d, K + (size_t)(i + 1) * d);
+    S.V.emplace_back(V + (size_t)i * d, V + (size_t)(i + 1) * d);
+    S.a_d.push_back(a[i]);
+    S.a_f.push_back((float)a[i]);
+    S.n.push_back(tokens - pos[i]);
+    S.pos.push_back(pos[i]);
+    S.cnt.push_back(1);
+  }
+  return 0;
+}
+
 // The pinned pieces, exposed so the tests can pin them against libm / fp64.
 float wkvo_pinned_exp(float x) { return pinned_exp(x); }
 float wkvo_pinned_dot(const float* q, const float* k, int32_t d, float scale32) { return pinned_dot(q, k, d, scale32); }

@@ -263,3 +263,29 @@ def test_decode_steps_replayed_from_a_cuda_graph(schedule):
     for x, y in zip(res["calls"][2], res["graph"][2]):
         for key in ("pos", "a", "K", "V"):
             assert torch.equal(x[key], y[key]), key
+
+
+def test_maximum_budget_at_the_capacity_limit():
+    """budget = 2^20 - 1, the largest the configuration accepts: a step attends 2^20 entries, the capacity the integer
+    normaliser is specified for (2^20 terms of at most 2^40).  Full caches are imported on both sides; a few steps and
+    the whole exported state must agree."""
+    m = (1 << 20) - 1
+    wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=m, W=16)
+    p = Parity(wl, seed=77)
+    assert p.ctx.wkv_splits() == 64
+    rng = np.random.default_rng(1)
+    tokens = m + 7
+    pos = np.sort(rng.choice(tokens, size=m, replace=False)).astype(np.int32)
+    for i, ln in enumerate(p.lanes):
+        a = (rng.random(m) * (tokens - pos) * 1e-6 + 1e-9).astype(np.float32)
+        K = (rng.standard_normal((m, 64)) * 0.5).astype(np.float32)
+        V = rng.standard_normal((m, 64)).astype(np.float32)
+        p.ctx.wkv_import_state(*ln, tokens=tokens, pos=torch.from_numpy(pos), a=torch.from_numpy(a),
+                               K=torch.from_numpy(K), V=torch.from_numpy(V))
+        p.ref.import_state(i, tokens, pos, a.astype(np.float64), K, V)
+    p.t = tokens
+    p.decode(3)
+    p.compare_state()
+    assert p.n_evictions == 3 * len(p.lanes)
+    p.close()
+    torch.cuda.empty_cache()

@@ -570,3 +570,25 @@ def test_merging_loses_less_than_eviction_on_synthetic_streams(rho):
         e_evict, n0 = compression_output_error(Q, K, V, m, W, merge=0)
         assert n1 == n0 == n * (T - m)                  # same trigger; the ablation changes only what happens to the value
         assert e_merge < 0.97 * e_evict, (rho, m, e_merge, e_evict)
+
+
+def test_imported_state_continues_like_the_streamed_one():
+    """wkvo_import (set-up for the large-cache tests) must put a lane exactly where streaming left it."""
+    rng = np.random.default_rng(0)
+    d, m = 16, 12
+    A = oracle.Oracle(1, d, m, window=2, mode=oracle.MODE_PINNED)
+    B = oracle.Oracle(1, d, m, window=2, mode=oracle.MODE_PINNED)
+    toks = [(rng.standard_normal((1, 1, d)).astype(np.float32), rng.standard_normal((1, d)).astype(np.float32),
+             rng.standard_normal((1, d)).astype(np.float32)) for _ in range(60)]
+    for q, k, v in toks[:30]:
+        A.step(q, k, v)
+    e = A.export(0)
+    B.import_state(0, A.tokens(0), e["pos"], e["a"], e["K"], e["V"])
+    for q, k, v in toks[30:]:
+        oa, ea, _ = A.step(q, k, v)
+        ob, eb, _ = B.step(q, k, v)
+        assert (ea == eb).all() and np.array_equal(oa, ob)
+    ea, eb = A.export(0), B.export(0)
+    assert all(np.array_equal(ea[key], eb[key]) for key in ("pos", "a", "K", "V", "n"))
+    with pytest.raises(ValueError):
+        B.import_state(0, 5, [3, 2], [0.1, 0.2], np.zeros((2, d)), np.zeros((2, d)))     # positions must increase
