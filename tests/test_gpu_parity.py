@@ -289,3 +289,32 @@ def test_maximum_budget_at_the_capacity_limit():
     assert p.n_evictions == 3 * len(p.lanes)
     p.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,m,schedule", [("bf16", 128, 8, 2, 50001, binding.WKV_SCHEDULE_SPLIT),
+                                                      ("f32", 64, 8, 1, 30011, binding.WKV_SCHEDULE_SPLIT),
+                                                      ("bf16", 128, 4, 2, 20003, binding.WKV_SCHEDULE_CLUSTER)])
+def test_large_imported_caches_grouped_heads(dtype, d, hq, hkv, m, schedule):
+    """Tens of thousands of entries per lane with 4, 8 and 2 query heads per key (odd budgets: ragged last tile and
+    uneven units), caches imported on both sides, sinks kept: picks, scores and state after a few compressing steps."""
+    wl = small(batch=2, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=24, S=3, rank=16 if dtype == "bf16" else 0)
+    p = Parity(wl, seed=m, schedule=schedule)
+    rng = np.random.default_rng(m)
+    tokens = m + 1000
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    for i, ln in enumerate(p.lanes):
+        pos = np.sort(np.concatenate([np.arange(3), 3 + rng.choice(tokens - 3, size=m - 3, replace=False)])).astype(np.int32)
+        a = (rng.random(m) * (tokens - pos) * 1e-5 + 1e-8).astype(np.float32)
+        K = torch.from_numpy((rng.standard_normal((m, d)) * 0.3).astype(np.float32)).to(tdt)
+        V = torch.from_numpy(rng.standard_normal((m, d)).astype(np.float32)).to(tdt)
+        p.ctx.wkv_import_state(*ln, tokens=tokens, pos=torch.from_numpy(pos), a=torch.from_numpy(a), K=K, V=V)
+        p.ref.import_state(i, tokens, pos, a.astype(np.float64), K.float().numpy(), V.float().numpy())
+    p.t = tokens
+    p.decode(5)
+    p.decode(2, layers_entry=True)
+    p.compare_state()
+    assert p.n_evictions == 7 * len(p.lanes)
+    for ln in p.lanes:
+        assert p.ctx.wkv_export_state(*ln)["pos"][:3].tolist() == [0, 1, 2]
+    p.close()
+    torch.cuda.empty_cache()
