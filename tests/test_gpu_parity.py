@@ -318,3 +318,29 @@ def test_large_imported_caches_grouped_heads(dtype, d, hq, hkv, m, schedule):
         assert p.ctx.wkv_export_state(*ln)["pos"][:3].tolist() == [0, 1, 2]
     p.close()
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("dtype,schedule", [("f32", binding.WKV_SCHEDULE_SPLIT), ("bf16", binding.WKV_SCHEDULE_CLUSTER)])
+def test_structural_ties_and_saturated_softmax(dtype, schedule):
+    """Degenerate score distributions.  (1) zero queries: every probability is exactly 1/(m+1) (m+1 a power of two), so
+    whole runs of entries tie bit for bit and the pick must be the lowest evictable position.  (2) queries scaled by
+    25: logit gaps far beyond the exponential's cut-off, most probabilities exactly zero, scores stop growing and tie
+    at equal values.  Both against the oracle, every step."""
+    wl = small(batch=2, hq=4, hkv=2, d=64, dtype=dtype, m=63, W=4, rank=16 if dtype == "bf16" else 0)
+    for kind in ("zero_q", "huge_q"):
+        p = Parity(wl, seed=91, schedule=schedule, n_splits=2)
+        draw = p.stream.token
+
+        def token(t, draw=draw, kind=kind):
+            q, k, v = draw(t)
+            return (torch.zeros_like(q) if kind == "zero_q" else (q.float() * 25.0).to(q.dtype)), k, v
+
+        p.stream.token = token
+        p.decode(160)
+        p.compare_state()
+        assert p.n_evictions == wl.lanes * (160 - 63)
+        if kind == "zero_q":
+            # uniform attention: the oldest evictable entry always has the smallest average once all have tied or aged
+            g = p.ctx.wkv_export_state(*p.lanes[0])
+            assert g["len"] == 63
+        p.close()
