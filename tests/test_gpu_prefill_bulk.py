@@ -209,3 +209,23 @@ def test_large_budget_dense_prompt_then_decode():
     p.compare_state()
     assert p.n_evictions == wl.lanes * 24
     p.close()
+
+
+@pytest.mark.parametrize("kind", ["zero_q", "huge_q"])
+def test_bulk_prefill_degenerate_scores(kind):
+    """Uniform attention (zero queries) and a saturated softmax (queries x25: most exponentials cut off to exactly 0)
+    through the dense kernel and the streamed tail."""
+    wl = small(batch=2, hq=4, hkv=2, d=128, dtype="bf16", m=140, W=6, rank=16)
+    p = Parity(wl, seed=19, ragged=[230, 131])
+    draw = p.stream.token
+
+    def token(t):
+        q, k, v = draw(t)
+        return (torch.zeros_like(q) if kind == "zero_q" else (q.float() * 25.0).to(q.dtype)), k, v
+
+    p.stream.token = token
+    p.prefill(230, chunk=230, bulk=True)
+    p.compare_state()
+    p.decode(20)
+    p.compare_state()
+    p.close()
