@@ -42,20 +42,20 @@ def pick_lanes(wl, n, seed):
 
 class Parity:
     def __init__(self, wl, seed=BASE_SEED, sample=None, n_splits=0, sink=None, merge=1, device="cuda:0", ragged=None,
-                 check_probs=False, schedule=0):
+                 check_probs=False, schedule=0, scale=0.0):
         self.wl, self.dev = wl, torch.device(device)
         self.sink = wl.sink if sink is None else sink
         self.dtype_code = binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16
         self.ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window,
                                    self.sink, self.dtype_code, merge=merge, n_splits=n_splits, device=self.dev,
-                                   schedule=schedule)
+                                   schedule=schedule, scale=scale)
         self.lanes = pick_lanes(wl, sample, seed)
         self.li = torch.tensor([l for l, _, _ in self.lanes], device=self.dev)
         self.bi = torch.tensor([b for _, b, _ in self.lanes], device=self.dev)
         self.hi = torch.tensor([h for _, _, h in self.lanes], device=self.dev)
         self.ref = oracle.Oracle(len(self.lanes), wl.head_dim, wl.budget, window=wl.window, sink=self.sink,
                                  group=wl.group, dtype=oracle.F32 if wl.dtype == "f32" else oracle.BF16,
-                                 mode=oracle.MODE_PINNED, merge=merge)
+                                 mode=oracle.MODE_PINNED, merge=merge, scale=scale)
         self.stream = TokenStream(wl, seed, self.dev)
         self.lens = sequence_lengths(wl, seed) if ragged is None else torch.as_tensor(ragged, dtype=torch.int32)
         self.t = 0

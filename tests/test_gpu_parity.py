@@ -344,3 +344,15 @@ def test_structural_ties_and_saturated_softmax(dtype, schedule):
             g = p.ctx.wkv_export_state(*p.lanes[0])
             assert g["len"] == 63
         p.close()
+
+
+@pytest.mark.parametrize("scale", [0.03125, 0.3])
+def test_softmax_scale_override(scale):
+    """A caller-chosen softmax scale (a power of two and one that is not) in place of 1/sqrt(head_dim): the one
+    multiplication after the dot, same on both sides; dense prompt phase, streamed tail and decode."""
+    wl = small(batch=2, hq=4, hkv=2, d=64, dtype="f32", m=50, W=4)
+    p = Parity(wl, seed=8, scale=scale, ragged=[90, 90])
+    p.prefill(90, chunk=90, bulk=True)
+    p.decode(40)
+    p.compare_state()
+    p.close()
