@@ -229,3 +229,24 @@ def test_bulk_prefill_degenerate_scores(kind):
     p.decode(20)
     p.compare_state()
     p.close()
+
+
+def test_bulk_prefill_eviction_ablation_and_stream_switch():
+    """merge = 0 (plain eviction with the same picks) through the dense phase and the streamed tail; halfway the
+    context is moved to another CUDA stream (wkv_set_stream) and must carry on from the same state."""
+    wl = small(layers=2, batch=2, hq=4, hkv=4, d=64, dtype="f32", m=48, W=4)
+    p = Parity(wl, seed=15, merge=0, ragged=[120, 77])
+    p.prefill(120, chunk=120, bulk=True)
+    p.compare_state()
+    p.decode(10)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    p.ctx.wkv_set_stream(side.cuda_stream)
+    with torch.cuda.stream(side):
+        p.decode(25)
+        p.compare_state()
+    side.synchronize()
+    p.ctx.wkv_set_stream(torch.cuda.current_stream().cuda_stream)
+    p.decode(5)
+    p.compare_state()
+    p.close()
