@@ -592,3 +592,30 @@ def test_imported_state_continues_like_the_streamed_one():
     assert all(np.array_equal(ea[key], eb[key]) for key in ("pos", "a", "K", "V", "n"))
     with pytest.raises(ValueError):
         B.import_state(0, 5, [3, 2], [0.1, 0.2], np.zeros((2, d)), np.zeros((2, d)))     # positions must increase
+
+
+# ---------------------------------------------------------------------------------------------
+# while nothing is compressed, Algorithm 1's accumulated scores are the column sums of the causal attention matrix
+# (what the dense prompt kernel computes in one go): textbook form in numpy, fp64
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("G", [1, 4])
+def test_scores_before_compression_are_causal_column_sums(G):
+    rng = np.random.default_rng(3)
+    n, d, lanes = 37, 16, 3
+    Q = rng.standard_normal((n, lanes, G, d))
+    K = rng.standard_normal((n, lanes, d))
+    V = rng.standard_normal((n, lanes, d))
+    ref = Oracle(lanes, d, n + 5, window=2, group=G, dtype=F32, mode=MODE_DOUBLE)
+    outs = [ref.step(Q[t].astype(np.float32), K[t].astype(np.float32), V[t].astype(np.float32))[0] for t in range(n)]
+    Qf, Kf, Vf = (x.astype(np.float32).astype(np.float64) for x in (Q, K, V))
+    for lane in range(lanes):
+        S = np.einsum("tgd,id->tgi", Qf[:, lane], Kf[:, lane]) / math.sqrt(d)          # [t, g, i]
+        S = np.where(np.arange(n)[None, None, :] <= np.arange(n)[:, None, None], S, -np.inf)
+        P = scipy_softmax(S, axis=-1)
+        want_a = P.mean(axis=1).sum(axis=0)                                                # column sums of the group mean
+        got = ref.export(lane)
+        np.testing.assert_allclose(got["a"], want_a, rtol=1e-12, atol=1e-15)
+        np.testing.assert_array_equal(got["pos"], np.arange(n))
+        np.testing.assert_array_equal(got["n"], n - np.arange(n))
+        want_o = np.einsum("tgi,id->tgd", P, Vf[:, lane])
+        np.testing.assert_allclose(np.stack([o[lane] for o in outs]), want_o, rtol=1e-10, atol=1e-12)
