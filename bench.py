@@ -189,6 +189,47 @@ def bulk_prefill_figures(wl, dev, seed, n_tokens=0, reps=3):
                          "algorithmic_fma_per_launch": fma}}
 
 
+def whole_prompt_figures(wl, dev, seed, n_tokens):
+    """A prompt of n_tokens per sequence for ALL layers in one wkv_prefill_bulk_layers call, and the same prompt streamed
+    layer by layer through wkv_prefill (Algorithm 1 as printed), for workloads whose prompt tensors fit beside the cache."""
+    from paper_2503_01330_b200 import binding
+    per_layer = wl.batch * n_tokens * (wl.n_q_heads + 2 * wl.n_kv_heads) * wl.head_dim * wl.elem_bytes
+    if per_layer * wl.n_layers > (24 << 30):
+        raise SystemExit("prompt tensors of all layers would take more than 24 GB: use --mode prefill (one layer)")
+    ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window, wl.sink,
+                          binding.WKV_F32 if wl.dtype == "f32" else binding.WKV_BF16, device=dev)
+    st = TokenStream(wl, seed, dev)
+    parts = [st.prompt(layer, n_tokens) for layer in range(wl.n_layers)]
+    Q, K, V = (torch.stack([p[i] for p in parts]) for i in range(3))
+    parts = None
+
+    def timed(fn):
+        ctx.wkv_reset()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def streamed():
+        for layer in range(wl.n_layers):
+            ctx.wkv_prefill(layer, Q[layer], K[layer], V[layer])
+
+    timed(lambda: ctx.wkv_prefill_bulk_layers(Q, K, V))            # takes the scratch, warms the path
+    bulk_ms = min(timed(lambda: ctx.wkv_prefill_bulk_layers(Q, K, V)) for _ in range(2))
+    streamed_ms = timed(streamed)
+    assert ctx.wkv_status() == 0
+    ctx.close()
+    return {"metric": "whole_prompt_ms_all_layers", "value": bulk_ms, "unit": "ms", "higher_is_better": False,
+            "streamed_layer_by_layer_ms": streamed_ms, "prompt_tokens_per_s": wl.batch * n_tokens / (bulk_ms * 1e-3),
+            "n_gpus": 1, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": wl.name, "n_layers": wl.n_layers, "batch": wl.batch, "budget": wl.budget,
+                       "window": wl.window, "sink": wl.sink, "prompt_tokens": n_tokens,
+                       "call": "wkv_prefill_bulk_layers: dense phase for the first budget tokens, the rest streamed"}}
+
+
 def run_reference(args, wl):
     """The reference arm: the CPU oracle on the host cores; each step is a bounded sample of the workload."""
     cores = os.cpu_count() or 1
@@ -230,8 +271,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the workload's layer count (profiling captures)")
-    ap.add_argument("--mode", default="decode", choices=["decode", "prefill"],
-                    help="prefill: time only the dense prompt phase (wkv_prefill_bulk) on one layer and print its line")
+    ap.add_argument("--mode", default="decode", choices=["decode", "prefill", "prompt"],
+                    help="prefill: time only the dense prompt phase (wkv_prefill_bulk) on one layer and print its line; "
+                         "prompt: a whole prompt of --prefill-tokens (default: the workload's prefill length) for all "
+                         "layers through wkv_prefill_bulk_layers, beside the same prompt streamed")
     ap.add_argument("--no-bulk-prefill", action="store_true", help="leave the bulk-prefill figure out of the decode line")
     ap.add_argument("--init", default="prefill", choices=["prefill", "import"],
                     help="import: fill every cache through wkv_import_state with one synthetic full lane instead of "
@@ -268,6 +311,13 @@ def main():
     torch.cuda.set_device(dev)
 
     seed = rank_seed(BASE_SEED, rank)
+    if args.mode == "prompt":
+        fig = whole_prompt_figures(wl, dev, seed, args.prefill_tokens if args.prefill_tokens else wl.prefill)
+        if rank == 0:
+            print(json.dumps(fig), flush=True)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     if args.mode == "prefill":
         fig = bulk_prefill_figures(wl, dev, seed, args.prefill_tokens)
         if rank == 0:
