@@ -162,14 +162,17 @@ int wkv_decode_step_layers_host(wkv_ctx* ctx, const void* q, const void* k, cons
 int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                 int32_t T_max, void* out, int32_t* evicted_pos);
 
-/* The same prompt, same arguments and same results as wkv_prefill, with the uncompressed start of the prompt done as
- * one dense problem per lane.  Algorithm 1 compresses only once a lane holds more than `budget` entries, so its first
- * min(T_max, budget) iterations are causal attention (Background section) plus the running sums of the attention
- * columns; when no lane of the layer has consumed a token since wkv_create / wkv_reset, one kernel computes those
- * iterations for all lanes of the layer (every logit, probability and accumulated score with the arithmetic of the
- * streamed step, scores added in the order of the tokens), and the remaining tokens are streamed as in wkv_prefill.
- * If the layer is not empty the whole prompt is streamed.  K, positions, accumulated scores and removed positions are
- * bit-identical to wkv_prefill's; outputs and merged values agree within rounding.
+/* The same prompt, same arguments and same results as wkv_prefill, with the uncompressed part of the prompt done as
+ * one dense problem per lane.  Algorithm 1 compresses only once a lane holds more than `budget` entries; until then
+ * its iterations are causal attention (Background section) plus the running sums of the attention columns.  The
+ * library keeps, per layer, an upper bound on the tokens any lane has consumed since wkv_create / wkv_reset (calls of
+ * every kind count; an imported lane counts as its token count if nothing of it was removed, as full otherwise).
+ * While that bound is below the budget, the first min(T_max, budget - bound) tokens of the call go through one kernel
+ * for all lanes of the layer -- on top of what each lane already holds, whose keys and values it reads from the cache
+ * -- with every logit, probability and accumulated score computed by the arithmetic of the streamed step and the
+ * scores added in the order of the tokens; the remaining tokens are streamed as in wkv_prefill.  So a prompt may come
+ * in one call or in chunks.  K, positions, accumulated scores and removed positions are bit-identical to
+ * wkv_prefill's; outputs and merged values agree within rounding.
  * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider and
  * keeps them until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
@@ -180,7 +183,7 @@ int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, 
  *   Q device [n_layers, batch, T_max, n_q_heads, head_dim], K, V device [n_layers, batch, T_max, n_kv_heads, head_dim]
  *   seq_lens device [batch] or NULL (shared by the layers); out like Q or NULL; evicted_pos device
  *   [n_layers, batch, T_max, n_kv_heads] int32 or NULL.  Inputs and outputs must not overlap; 16-byte alignment as above.
- * When no layer has consumed a token, the dense phase runs over the lanes of all layers at once if its scratch
+ * While no lane of any layer can have reached the budget, the dense phase runs over the lanes of all layers at once if its scratch
  * (64 * n_layers * lanes_per_layer * round_up(budget, 128) bytes) stays under 256 MB -- what a single sequence needs to
  * fill the GPU -- and layer by layer otherwise.  The remaining tokens are streamed: one launch per token over the
  * lanes of all layers where wkv_decode_step_layers does the same, else with the layers interleaved so that one layer's

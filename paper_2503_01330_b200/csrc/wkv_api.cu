@@ -63,7 +63,9 @@ struct wkv_ctx {
   float* bulk_S = nullptr;
   int bulk_stride = 0;
   long long bulk_lanes = 0;     // lanes the scratch has rows for
-  std::vector<char> fresh;
+  // per layer: an upper bound on the tokens any lane of the layer has consumed since creation / reset; while it is
+  // below the budget no lane has compressed and token i of every lane sits in slot i (kCompressed: unknown / beyond)
+  std::vector<long long> tokens_hi;
   std::vector<void*> owned;
   long long device_bytes = 0;
   long long launches = 0;
@@ -300,7 +302,7 @@ void note_outputs(wkv_ctx* c, const void* out, size_t out_bytes, const void* ev,
 }
 
 int run_reset(wkv_ctx* c) {
-  c->fresh.assign((size_t)c->cfg.n_layers, 1);
+  c->tokens_hi.assign((size_t)c->cfg.n_layers, 0);
   for (int i = 0; i < 2; ++i) WKV_CUDA(c, cudaMemsetAsync(c->ticket[i], 0, (size_t)c->lanes_per_layer * 4, c->stream));
   if (c->fused_ticket) WKV_CUDA(c, cudaMemsetAsync(c->fused_ticket, 0, (size_t)c->lanes_total * 4, c->stream));
   wkv::reset_kernel<<<592, 256, 0, c->stream>>>(c->lane_state, c->pos, c->a, c->next, c->prev, c->lanes_total, c->cap,
@@ -479,7 +481,7 @@ static int decode_step_impl(wkv_ctx* c, int32_t layer, const void* q, const void
   P.tok_idx = 0;
   const size_t row = (size_t)D * c->elem;
   const size_t q_bytes = (size_t)c->cfg.batch * c->cfg.n_q_heads * row, kv_bytes = (size_t)c->lanes_per_layer * row;
-  c->fresh[layer] = 0;
+  c->tokens_hi[layer] += 1;
   if (!c->use_cluster) prepare_overlap(c, P, layer, q_bytes, kv_bytes, inputs_ready);
   cudaError_t e = launch_any(c, P, c->use_cluster);
   c->launches += c->use_cluster ? 1 : 2;
@@ -523,7 +525,7 @@ int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void*
     P.ev_bs = c->cfg.n_kv_heads;
     P.wait_at_start = 2;
     g_last_launcher.store(c);
-    c->fresh.assign((size_t)c->cfg.n_layers, 0);
+    for (auto& th : c->tokens_hi) th += 1;
     cudaError_t e = launch_any(c, P, c->fused_cluster, (int)c->lanes_total);
     c->launches += c->fused_cluster ? 1 : 2;
     if (e != cudaSuccess) return cuda_fail(c, e, "decode step launch (all layers)");
@@ -571,7 +573,7 @@ int wkv_decode_step_static(wkv_ctx* c, int32_t layer, const void* q, const void*
   // kernel writes every logit and every partial of an active lane before the epilogue kernel reads them.
   P.wait_at_start = 2;                 // one array for everybody: never start before the previous kernel has finished
   c->last_layer = -1;
-  c->fresh[layer] = 0;
+  c->tokens_hi[layer] += 1;
   g_last_launcher.store(nullptr);
   e = launch_any(c, P, false);
   c->launches += 2;
@@ -624,7 +626,7 @@ static int stream_tokens(wkv_ctx* c, int32_t layer, const void* Q, const void* K
   P.kv_bs = (long long)T_max * Hk * D;
   P.out_bs = out ? P.q_bs : Hq * D;
   P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
-  if (t_begin < T_max) c->fresh[layer] = 0;
+  if (t_begin < T_max) c->tokens_hi[layer] += T_max - t_begin;
   for (int t = t_begin; t < T_max; ++t) {
     P.tok_idx = t;
     P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
@@ -711,14 +713,16 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15)
     return fail(c, WKV_ERR_INVALID, "wkv_prefill_bulk: Q, K, V and out must be 16-byte aligned");
   int32_t n0 = 0;
-  if (c->fresh[layer] && T_max > 0) {
-    // Every lane of the layer is empty: the first min(T_max, budget) tokens compress nothing and go through the
-    // dense kernel; the rest of the prompt is streamed behind it on the same stream.
-    n0 = std::min(T_max, c->cfg.budget);
+  const long long room = (long long)c->cfg.budget - c->tokens_hi[layer];
+  if (room > 0 && T_max > 0) {
+    // No lane of the layer can hold more than budget - room tokens, so none has compressed and the next `room` tokens
+    // compress nothing either: the first min(T_max, room) tokens of this call go through the dense kernel (on top of
+    // whatever each lane already holds), the rest is streamed behind it on the same stream.
+    n0 = (int32_t)std::min<long long>(T_max, room);
     rc = launch_dense(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, Q, K, V, seq_lens, T_max, n0, out,
                       evicted_pos);
     if (rc != WKV_OK) return rc;
-    c->fresh[layer] = 0;
+    c->tokens_hi[layer] += n0;
   }
   return stream_tokens(c, layer, Q, K, V, seq_lens, n0, T_max, out, evicted_pos);
 }
@@ -737,11 +741,11 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
       ranges_overlap(V, kv_layer * L, out, q_layer * L) || ranges_overlap(Q, q_layer * L, evicted_pos, ev_layer * 4 * L) ||
       ranges_overlap(K, kv_layer * L, evicted_pos, ev_layer * 4 * L) || ranges_overlap(V, kv_layer * L, evicted_pos, ev_layer * 4 * L))
     return fail(c, WKV_ERR_INVALID, "wkv_prefill_bulk_layers: inputs and outputs must not overlap");
-  bool all_fresh = true;
-  for (int l = 0; l < L; ++l) all_fresh = all_fresh && c->fresh[l];
+  long long room = c->cfg.budget;
+  for (int l = 0; l < L; ++l) room = std::min(room, (long long)c->cfg.budget - c->tokens_hi[l]);
   int32_t n0 = 0;
-  if (all_fresh && T_max > 0) {
-    n0 = std::min(T_max, c->cfg.budget);
+  if (room > 0 && T_max > 0) {
+    n0 = (int32_t)std::min<long long>(T_max, room);        // uncompressed in every lane of every layer (see wkv_prefill_bulk)
     const int stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
     const size_t need_all = (size_t)c->lanes_total * wkv::kBulkRows * stride * 4;
     if (need_all <= ((size_t)256 << 20)) {
@@ -756,15 +760,12 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
         if (rc != WKV_OK) return rc;
       }
     }
-    c->fresh.assign((size_t)L, 0);
-  } else if (!all_fresh) {
-    // some layer already holds tokens: nothing is known to be uncompressed, stream everything
-    n0 = 0;
+    for (auto& th : c->tokens_hi) th += n0;
   }
   // The rest of the prompt, token by token with the layers interleaved: consecutive launches then belong to different
   // layers, and since every input of this call existed before it was issued, a layer's scan may overlap the previous
   // layer's lane epilogues.
-  if (n0 < T_max) c->fresh.assign((size_t)L, 0);
+  for (auto& th : c->tokens_hi) th += T_max - n0;
   c->last_layer = -1;
   if (c->fused_ok && n0 < T_max) {
     // a layer alone cannot fill the GPU: one launch (pair) per token over the lanes of all layers, as in
@@ -892,7 +893,8 @@ int wkv_import_state(wkv_ctx* c, int32_t layer, int32_t b, int32_t kv_head, int3
   const long long lane = ((long long)layer * c->cfg.batch + b) * c->cfg.n_kv_heads + kv_head;
   const int cap = c->cap;
   const size_t row = (size_t)c->cfg.head_dim * c->elem;
-  c->fresh[layer] = 0;
+  // an imported lane counts as uncompressed only if it is: every token still there, hence token i in slot i
+  c->tokens_hi[layer] = tokens == len ? std::max<long long>(c->tokens_hi[layer], tokens) : (long long)c->cfg.budget;
   std::vector<int32_t> hpos(cap, -1), hnext(cap, -1), hprev(cap, -1);
   std::vector<float> ha(cap, 0.f);
   for (int i = 0; i < len; ++i) {

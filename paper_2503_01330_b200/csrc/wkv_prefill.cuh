@@ -6,7 +6,9 @@
 // a_i = sum_t mean_g P[t, g, i] that Algorithm 1 accumulates one step at a time.  This kernel computes exactly what
 // those n streamed steps compute: every logit with the reproducible dot, every probability with the reproducible
 // exponential and the integer-sum normaliser, and every a_i by adding its terms in ascending t, so that K, pos, a and
-// the links come out bit-identical to streaming; the outputs (not part of that chain) agree to rounding.
+// the links come out bit-identical to streaming; the outputs (not part of that chain) agree to rounding.  A lane may
+// already hold uncompressed tokens from earlier calls (a prompt fed in chunks): their keys and values are read from
+// the cache, where token i still sits in slot i, and the new rows attend to them as well.
 //
 // One CTA per lane walks the prompt in blocks of 16 query rows (16 / G tokens x G query heads):
 //   phase 1  S block = Q block . K^T tile by tile (fp32 FMAs in the reproducible order), causal mask, parked in an
@@ -136,8 +138,14 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
   const long long lane = (long long)P.lane0 + lane_local;
   const int Hk = P.n_kv_heads, Hq = Hk * G;
-  int n = P.n0;
-  if (P.seq_lens != nullptr) n = min(n, max(0, P.seq_lens[b % P.batch]));
+  // The lane may already hold n_old tokens from earlier calls -- uncompressed, so token i sits in slot i with its
+  // score a_i so far; the host only sends lanes here whose n_old + n0 cannot exceed the budget.  This call adds n_new
+  // tokens (input rows 0 .. n_new-1, global token index n_old + row); n = tokens held afterwards.
+  const int n_old = P.lane_state[lane * LS_STRIDE + LS_T];
+  const bool consistent = P.lane_state[lane * LS_STRIDE + LS_LEN] == n_old && n_old + P.n0 <= P.s_stride && n_old + P.n0 < P.cap;
+  int n_new = P.n0;
+  if (P.seq_lens != nullptr) n_new = min(n_new, max(0, P.seq_lens[b % P.batch]));
+  const int n = n_old + n_new;
   const T* Qb = reinterpret_cast<const T*>(P.Q) + ((long long)b * P.T_max * Hq + (long long)hk * G) * D;   // + t*Hq*D + g*D
   const T* Kb = reinterpret_cast<const T*>(P.K) + ((long long)b * P.T_max * Hk + hk) * D;                  // + t*Hk*D
   const T* Vb = reinterpret_cast<const T*>(P.V) + ((long long)b * P.T_max * Hk + hk) * D;
@@ -149,7 +157,11 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // no compression happens in this phase: report "nothing removed" for every token it covers
   if (P.evicted != nullptr)
     for (int t = tid; t < P.n0; t += kBulkThreads) P.evicted[((long long)b * P.T_max + t) * Hk + hk] = -1;
-  if (n == 0) return;
+  if (!consistent) {                                     // cannot happen through the library's entry points
+    if (tid == 0) atomicOr(P.status, kStatusBadLink);
+    return;
+  }
+  if (n_new == 0) return;
 
   if (tid == 0) {
     mbar_init(&full[0], KT);                             // every issuing thread arrives once per fill
@@ -160,13 +172,16 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // The ring.  Thread r < KT fetches row r of a tile: one bulk copy, counted in bytes on the stage's barrier.  Rows
   // beyond the last key of the block re-fetch that last key (finite values; their probabilities are exactly zero).
   uint32_t parity = 0;                                   // bit s: parity of stage s's next completion
-  auto issue = [&](const T* base, int kt, int s, int nk_) {
+  // Keys / values of tokens before n_old come from the cache (slot = token), the others from this call's input.
+  auto issue = [&](bool values, int kt, int s, int nk_) {
     if (tid < KT) {
       const int r = min(kt * KT + tid, nk_ - 1);
+      const T* src = r < n_old ? (values ? Vl : Kl) + (long long)r * D : (values ? Vb : Kb) + (long long)(r - n_old) * Hk * D;
       mbar_expect_tx(&full[s], ROWB);
-      bulk_g2s(stage0 + (s * KT + tid) * RS, base + (long long)r * Hk * D, ROWB, &full[s]);
+      bulk_g2s(stage0 + (s * KT + tid) * RS, src, ROWB, &full[s]);
     }
   };
+  constexpr bool kKeys = false, kValues = true;
   auto wait_stage = [&](int s) {
     mbar_wait(&full[s], (parity >> s) & 1u, P.status);
     parity ^= 1u << s;
@@ -180,7 +195,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
       const int r = c / (ROWB / 16), q = c % (ROWB / 16);
       const int tok = t0_ + r / G, g = r % G;
       qpre[i] = make_uint4(0u, 0u, 0u, 0u);
-      if (tok < n) qpre[i] = reinterpret_cast<const uint4*>(Qb + ((long long)tok * Hq + g) * D)[q];
+      if (tok < n) qpre[i] = reinterpret_cast<const uint4*>(Qb + ((long long)(tok - n_old) * Hq + g) * D)[q];
     }
   };
   auto store_q = [&]() {
@@ -200,27 +215,28 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
       }
     }
   };
-  load_q(0);
-  issue(Kb, 0, 0, min(BQ, n));
-  if (min(BQ, n) > KT) issue(Kb, 1, 1, min(BQ, n));
+  load_q(n_old);
+  issue(kKeys, 0, 0, min(n_old + BQ, n));
+  if (min(n_old + BQ, n) > KT) issue(kKeys, 1, 1, min(n_old + BQ, n));
 
   // the cache after n uncompressed steps: token i in slot i, linked in order (Algorithm 1 appends, nothing is removed)
   {
     constexpr int Q8 = ROWB / 16;                        // 16-byte pieces per row
-    for (int c = tid; c < n * Q8; c += kBulkThreads) {
+    for (int c = tid; c < n_new * Q8; c += kBulkThreads) {
       const int r = c / Q8, q = c % Q8;
-      reinterpret_cast<uint4*>(Kl + (long long)r * D)[q] = reinterpret_cast<const uint4*>(Kb + (long long)r * Hk * D)[q];
-      reinterpret_cast<uint4*>(Vl + (long long)r * D)[q] = reinterpret_cast<const uint4*>(Vb + (long long)r * Hk * D)[q];
+      reinterpret_cast<uint4*>(Kl + (long long)(n_old + r) * D)[q] = reinterpret_cast<const uint4*>(Kb + (long long)r * Hk * D)[q];
+      reinterpret_cast<uint4*>(Vl + (long long)(n_old + r) * D)[q] = reinterpret_cast<const uint4*>(Vb + (long long)r * Hk * D)[q];
     }
     int32_t* pos_l = P.pos + lane * P.cap;
     int32_t* next_l = P.next + lane * P.cap;
     int32_t* prev_l = P.prev + lane * P.cap;
-    for (int i = tid; i < n; i += kBulkThreads) {
+    for (int i = n_old + tid; i < n; i += kBulkThreads) {
       pos_l[i] = i;
       next_l[i] = i + 1 < n ? i + 1 : -1;
       prev_l[i] = i - 1;
     }
     if (tid == 0) {
+      if (n_old > 0) next_l[n_old - 1] = n_old;          // the old tail gets a right neighbour
       int32_t* st = P.lane_state + lane * LS_STRIDE;
       st[LS_LEN] = n;
       st[LS_T] = n;
@@ -230,7 +246,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
     }
   }
 
-  for (int t0 = 0; t0 < n; t0 += BQ) {
+  for (int t0 = n_old; t0 < n; t0 += BQ) {
     const int nk = min(t0 + BQ, n);                      // keys 0 .. nk-1 are visible to some row of the block
     const int n_tiles = (nk + KT - 1) / KT;
     int t_row[4];                                        // token of each of my 4 rows
@@ -297,11 +313,11 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         }
       }
       __syncthreads();                                   // everybody is done with the stage
-      if (kt + 2 < n_tiles) issue(Kb, kt + 2, s, nk);
+      if (kt + 2 < n_tiles) issue(kKeys, kt + 2, s, nk);
     }
     // both stages are free: put the first V tiles in flight, they land while the exponentials are computed
-    issue(Vb, 0, 0, nk);
-    if (n_tiles > 1) issue(Vb, 1, 1, nk);
+    issue(kValues, 0, 0, nk);
+    if (n_tiles > 1) issue(kValues, 1, 1, nk);
     // ---- phase 2: exponentials in place and the integer-sum normaliser (each thread re-reads what it wrote) ------
     float Z[4];
 #pragma unroll
@@ -425,13 +441,13 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
             o_acc[i][c] = pack2(lo_of(o_acc[i][c]) + lo_of(o_tile[i][c]), hi_of(o_acc[i][c]) + hi_of(o_tile[i][c]));
       }
       __syncthreads();                                   // everybody is done with the stage and the probability tiles
-      if (kt + 2 < n_tiles) issue(Vb, kt + 2, s, nk);
+      if (kt + 2 < n_tiles) issue(kValues, kt + 2, s, nk);
     }
     // both stages are free again: the next block's first K tiles travel while this block's outputs are stored
     if (t0 + BQ < n) {
       const int nk_next = min(t0 + 2 * BQ, n);
-      issue(Kb, 0, 0, nk_next);
-      if (nk_next > KT) issue(Kb, 1, 1, nk_next);
+      issue(kKeys, 0, 0, nk_next);
+      if (nk_next > KT) issue(kKeys, 1, 1, nk_next);
     }
     if (P.out != nullptr) {
       if constexpr (kTensorPV) {
@@ -441,7 +457,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
           const int rho = (ln >> 2) + 8 * h;
           const int t = t0 + rho / G, g = rho % G;
           if (t >= n) continue;
-          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t) * Hq + (long long)hk * G + g) * D + w * (D / 4) + (ln & 3) * 2;
+          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + (t - n_old)) * Hq + (long long)hk * G + g) * D + w * (D / 4) + (ln & 3) * 2;
 #pragma unroll
           for (int nt = 0; nt < NTW; ++nt) {
             const float x[2] = {cacc[nt][2 * h], cacc[nt][2 * h + 1]};
@@ -453,7 +469,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         for (int i = 0; i < 4; ++i) {
           if (!act[i]) continue;
           const int g = (4 * w + i) % G;
-          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + t_row[i]) * Hq + (long long)hk * G + g) * D + ln * CPT;
+          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + (t_row[i] - n_old)) * Hq + (long long)hk * G + g) * D + ln * CPT;
           float x[CPT];
 #pragma unroll
           for (int c = 0; c < CPT / 2; ++c) { x[2 * c] = lo_of(o_acc[i][c]); x[2 * c + 1] = hi_of(o_acc[i][c]); }

@@ -75,18 +75,39 @@ def test_bulk_and_streamed_prefill_leave_identical_state(schedule):
     torch.testing.assert_close(outs[1][0], outs[0][0], rtol=2e-2, atol=1e-3)
 
 
-def test_bulk_prefill_on_a_used_layer_streams():
-    """A layer that already holds tokens is continued token by token; the result is still Algorithm 1's."""
+def test_bulk_prefill_continues_uncompressed_layers_and_streams_the_rest():
+    """A prompt that arrives in pieces: while no lane of the layer can have reached the budget, each piece goes through
+    the dense kernel on top of what the lanes hold; afterwards the pieces are streamed.  Decode steps in between count
+    as tokens too.  The result is Algorithm 1's throughout."""
     wl = small(batch=2, d=64, dtype="f32", m=50, W=4)
     p = Parity(wl, seed=5, ragged=[140, 140])
     p.prefill(30, chunk=30, bulk=True)      # empty layer: dense
-    p.prefill(60, chunk=60, bulk=True)      # 30 tokens held: streamed
+    n1 = p.ctx.wkv_launch_count()
+    p.prefill(12, chunk=12, bulk=True)      # 30 tokens held, 42 after: still dense (one launch)
+    assert p.ctx.wkv_launch_count() == n1 + 1
+    p.decode(3)                             # 45
+    p.prefill(45, chunk=45, bulk=True)      # 5 more fit densely, 40 streamed
     p.decode(10)
-    p.prefill(40, chunk=40, bulk=True)
+    p.prefill(40, chunk=40, bulk=True)      # full: streamed
     p.compare_state()
     launches = p.ctx.wkv_launch_count()
     p.ctx.wkv_reset()
     assert p.ctx.wkv_launch_count() == launches + 1
+    p.close()
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,m,chunk,all_layers", [("bf16", 128, 8, 2, 300, 37, False), ("f32", 64, 4, 4, 190, 64, False),
+                                                               ("bf16", 128, 4, 4, 260, 50, True), ("bf16", 64, 8, 1, 150, 16, True)])
+def test_chunked_prompts_through_the_dense_kernel(dtype, d, hq, hkv, m, chunk, all_layers):
+    """Prompts fed in chunks (chunked prefill): every chunk that still fits under the budget is a dense launch that
+    reads the earlier tokens' keys and values from the cache; ragged sequence ends fall inside and between chunks."""
+    wl = small(layers=2, batch=3, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=6, rank=16 if dtype == "bf16" else 0)
+    T = m + 2 * chunk + 5
+    p = Parity(wl, seed=60 + m, ragged=[T, m - chunk // 2, 2 * chunk + 3])
+    p.prefill(T, chunk=chunk, bulk=True, all_layers=all_layers)
+    p.compare_state()
+    p.decode(12)
+    p.compare_state()
     p.close()
 
 
