@@ -2,6 +2,8 @@
 configuration bench.py times, on sampled lanes the oracle computes one by one.  The streamed prompt is shortened
 to budget + 160 tokens: every cache is then full and has compressed 160 times, which is the state the decode phase
 runs in."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -49,3 +51,35 @@ def test_paper_cache_settings(name):
     for ln in p.lanes:                                     # the four initial tokens are never removed
         assert p.ctx.wkv_export_state(*ln)["pos"][:4].tolist() == [0, 1, 2, 3]
     p.close()
+
+
+def test_llama7b_b8_full_prompt_length():
+    """The 32-layer, batch-8 configuration with its whole 8192-token prompt (budget 1638: 6554 compressions per lane
+    before the first decode step), fed in chunks of 256 tokens for all layers at once -- dense while the lanes are below
+    the budget, streamed with interleaved layers afterwards -- then decode; sampled lanes against the oracle."""
+    wl = WORKLOADS["llama7b_b8"]
+    p = Parity(wl, sample=6, ragged=[wl.prefill] * wl.batch)
+    p.prefill(wl.prefill, chunk=256, all_layers=True)
+    p.compare_state()
+    p.decode(24)
+    p.compare_state()
+    assert p.n_evictions == len(p.lanes) * (wl.prefill + 24 - wl.budget)
+    p.close()
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.skipif(os.environ.get("WKV_LONG_TESTS") != "1", reason="several minutes each: set WKV_LONG_TESTS=1")
+@pytest.mark.parametrize("name,n_sample", [("serving_b16", 6), ("gqa_b32", 4)])
+def test_serving_and_gqa_full_prompt_lengths(name, n_sample):
+    """The two largest configurations with their whole prompts (16384 tokens with per-sequence lengths drawn from
+    8192..16384, and 32768 tokens), in chunks of 256 tokens for all layers at once, then decode; sampled lanes against
+    the oracle.  Tens of thousands of compressions per lane."""
+    wl = WORKLOADS[name]
+    p = Parity(wl, sample=n_sample)
+    assert int(p.lens.max()) == wl.prefill and int(p.lens.min()) >= wl.prefill_min
+    p.prefill(wl.prefill, chunk=256, all_layers=True)
+    p.compare_state()
+    p.decode(8)
+    p.compare_state()
+    p.close()
+    torch.cuda.empty_cache()
