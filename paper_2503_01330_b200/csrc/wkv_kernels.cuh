@@ -657,7 +657,9 @@ __device__ __forceinline__ void exp_and_zsum(float* lg, long long stride, int n,
 }
 
 // Group-wide sums of G 64-bit integers; x[g] holds the total in every thread after the call.  scratch: G*NT/32 entries.
-template <int G, int NT>
+// kRelease = false leaves out the trailing barrier: the caller then must not write the scratch again before a later
+// barrier of its own.
+template <int G, int NT, bool kRelease = true>
 __device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsigned long long* scratch) {
   const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
 #pragma unroll
@@ -673,7 +675,7 @@ __device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsign
     for (int w = 0; w < NT / 32; ++w) z += scratch[g * (NT / 32) + w];
     x[g] = z;
   }
-  group_sync<NT>();
+  if constexpr (kRelease) group_sync<NT>();
 }
 
 // A_t over a range of slots, a = [a,0] + A_t, abar = a/n and the range's pick key (Algorithm 1).
@@ -822,19 +824,28 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
   float* lg = P.logits + (long long)v.lane_local * G * P.cap;
   const float* part = P.part + (long long)v.lane_local * P.n_splits * G * (D + 2);
   // (1) split weights and the global max / normaliser of every query head
-  if (tid < G) {
-    const int g = tid;
+  // (warp g takes head g, a lane takes splits lane and lane + 32: one round of loads instead of a serial loop)
+  static_assert(NT / 32 >= G && kMaxSplits <= 64, "one warp per query head, two splits per lane");
+  if ((tid >> 5) < G) {
+    const int g = tid >> 5, lq = tid & 31;
     const float* pg = part + g * (D + 2);
-    float M = -INFINITY;
-    for (int s = 0; s < P.n_splits; ++s) M = fmaxf(M, __ldcg(pg + (long long)s * G * (D + 2)));
-    float lsum = 0.f;
-    for (int s = 0; s < P.n_splits; ++s) {
-      const float w = fast_exp2((__ldcg(pg + (long long)s * G * (D + 2)) - M) * kLog2e);
-      ep.w[g * kMaxSplits + s] = w;
-      lsum += w * __ldcg(pg + (long long)s * G * (D + 2) + 1);
+    const long long st = (long long)G * (D + 2);
+    const bool has0 = lq < P.n_splits, has1 = lq + 32 < P.n_splits;
+    const float m0 = has0 ? __ldcg(pg + lq * st) : -INFINITY, l0 = has0 ? __ldcg(pg + lq * st + 1) : 0.f;
+    const float m1 = has1 ? __ldcg(pg + (lq + 32) * st) : -INFINITY, l1 = has1 ? __ldcg(pg + (lq + 32) * st + 1) : 0.f;
+    float M = fmaxf(m0, m1);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, off));
+    const float w0 = has0 ? fast_exp2((m0 - M) * kLog2e) : 0.f, w1 = has1 ? fast_exp2((m1 - M) * kLog2e) : 0.f;
+    if (has0) ep.w[g * kMaxSplits + lq] = w0;
+    if (has1) ep.w[g * kMaxSplits + lq + 32] = w1;
+    float lsum = w0 * l0 + w1 * l1;
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, off);
+    if (lq == 0) {
+      ep.M[g] = M;                  // max of the reproducible logits: exact, order-free
+      ep.linv[g] = 1.f / lsum;
     }
-    ep.M[g] = M;                    // max of the reproducible logits: exact, order-free
-    ep.linv[g] = 1.f / lsum;
   }
   group_sync<NT>();
   // (2) o_t = A_t^T V_t (Background section), V as it was before this step's merge
@@ -849,22 +860,19 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
     }
   }
   // (3) Z_g as an exact integer sum
+  float Zr[G];
   {
     unsigned long long zl[G];
     exp_and_zsum<G, true, NT>(lg, P.cap, L, ep.M, zl);
-    group_sum_u64<G, NT>(zl, ep.u64);
-    if (tid < G) {
+    group_sum_u64<G, NT, false>(zl, ep.u64);          // every thread holds the totals; the scratch is not written again
 #pragma unroll
-      for (int g = 0; g < G; ++g)
-        if (g == tid) ep.Z[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
-    }
-    group_sync<NT>();
+    for (int g = 0; g < G; ++g) Zr[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
   }
   // (4) probabilities, score fold, pick
   const bool compress = L > P.budget;                 // "length of V_t exceeds m"
   unsigned long long best = ~0ull;
   int best_slot = -1;
-  fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, ep.Z, compress, best, best_slot);
+  fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, Zr, compress, best, best_slot);
   if (P.probs) {
     for (int i = L + tid; i < P.budget + 1; i += NT)
 #pragma unroll
