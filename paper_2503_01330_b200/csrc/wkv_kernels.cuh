@@ -765,6 +765,15 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
   float vj = 0.f;
   const bool merging = compress && P.merge && j_slot >= 0;
   if (merging && tid < D) vj = to_f32(j_slot == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)j_slot * D + tid));
+  // ... and so can the right neighbour's row, without waiting for thread 0's walk: r = next[j], which this step
+  // changes only if j is the old tail (then r is the new entry).  One round trip less on the lane's critical path.
+  int r_early = -1;
+  float vr_early = 0.f;
+  if (merging && tid < D) {
+    r_early = j_slot == v.tail ? new_slot : __ldcg(next_l + j_slot);
+    if (r_early >= 0 && r_early < P.cap)
+      vr_early = to_f32(r_early == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r_early * D + tid));
+  }
   if (tid == 0) {
     int head = v.head, tail = v.tail;
     next_l[new_slot] = -1;
@@ -810,7 +819,7 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
   if (merging && ep.i32[2] >= 0 && tid < D) {
     const int r = ep.i32[3];
     const float wj = ep.misc[0], wr = ep.misc[1];
-    const float vr = to_f32(r == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r * D + tid));
+    const float vr = r == r_early ? vr_early : to_f32(r == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r * D + tid));
     Vw[(long long)r * D + tid] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
   }
 }
