@@ -10,6 +10,8 @@
 #include <string>
 #include <vector>
 
+#include <cuda.h>                      // tensor-map types only; the driver entry point is looked up at run time
+
 #include "../../include/wkv.h"
 #include "wkv_kernels.cuh"
 #include "wkv_prefill.cuh"
@@ -52,6 +54,8 @@ struct wkv_ctx {
   const char* last_out[3] = {nullptr, nullptr, nullptr};
   size_t last_out_bytes[3] = {0, 0, 0};
   uint32_t* status = nullptr;
+  // four query heads on bf16 rows: the scan takes its V tiles through this tensor map (see StepParams::vmap)
+  alignas(64) unsigned char vmap[128] = {};
   // staging for the host-buffer entry point and for discarded prefill outputs
   void* stage_q = nullptr;
   void* stage_k = nullptr;
@@ -111,6 +115,33 @@ int take(wkv_ctx* c, P** dst, size_t bytes) {
   return WKV_OK;
 }
 
+// Tensor map over the value cache as a [rows][head_dim] bf16 matrix, boxes of 64 elements x one tile of rows, 128-byte
+// swizzle, zero fill past the last row.  The driver's encoder is found through the runtime: the library does not
+// link against the driver.
+int encode_value_map(wkv_ctx* c, void* base, unsigned long long rows, int head_dim) {
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static_assert(sizeof(CUtensorMap) == sizeof(c->vmap), "tensor map size");
+  void* sym = nullptr;
+  cudaDriverEntryPointQueryResult qr = cudaDriverEntryPointSymbolNotFound;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
+  if (qr != cudaDriverEntryPointSuccess || !sym) return fail(c, WKV_ERR_CUDA, "the driver has no cuTensorMapEncodeTiled");
+  if (rows >= 0x7fffffffULL) return fail(c, WKV_ERR_INVALID, "n_layers * batch * n_kv_heads * (budget + 1) must stay below 2^31 rows with four query heads per key");
+  const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)wkv::kTileSlots};
+  const cuuint32_t estr[2] = {1u, 1u};
+  CUtensorMap m;
+  const CUresult r = reinterpret_cast<encode_fn>(sym)(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(c, WKV_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+  std::memcpy(c->vmap, &m, sizeof(m));
+  return WKV_OK;
+}
+
 const char* check_config(const wkv_config* c) {
   if (!c) return "config is NULL";
   if (c->n_layers < 1 || c->batch < 1) return "n_layers and batch must be >= 1";
@@ -132,9 +163,37 @@ const char* check_config(const wkv_config* c) {
   return nullptr;
 }
 
+// Scan CTAs that fit on one SM together (registers and shared memory of the instantiation this configuration runs).
+template <typename T, int D, int G>
+int scan_ctas_per_sm_of() {
+  using C = wkv::Cfg<T, D, G>;
+  int n = 0;
+  if (cudaFuncSetAttribute(wkv::scan_entry<T, D, G>(), cudaFuncAttributeMaxDynamicSharedMemorySize, C::kFixedBytes) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, wkv::scan_entry<T, D, G>(), wkv::kThreads, C::kFixedBytes) != cudaSuccess) {
+    cudaGetLastError();
+    return 4;
+  }
+  return n < 1 ? 1 : n;
+}
+template <typename T, int D>
+int scan_ctas_per_sm_by_group(int G) {
+  switch (G) {
+    case 1: return scan_ctas_per_sm_of<T, D, 1>();
+    case 2: return scan_ctas_per_sm_of<T, D, 2>();
+    case 4: return scan_ctas_per_sm_of<T, D, 4>();
+    default: return scan_ctas_per_sm_of<T, D, 8>();
+  }
+}
+int scan_ctas_per_sm(const wkv_config& c) {
+  const int G = c.n_q_heads / c.n_kv_heads;
+  if (c.dtype == WKV_BF16) return c.head_dim == 128 ? scan_ctas_per_sm_by_group<__nv_bfloat16, 128>(G) : scan_ctas_per_sm_by_group<__nv_bfloat16, 64>(G);
+  return c.head_dim == 128 ? scan_ctas_per_sm_by_group<float, 128>(G) : scan_ctas_per_sm_by_group<float, 64>(G);
+}
+
 // Splits per lane when the caller leaves the choice to the library: a power of two (so the lane's CTAs can form a
 // thread-block cluster), enough CTAs to fill 148 SMs several times over, at least ~4 tiles of work per CTA.
-int auto_splits(const wkv_config& c, long long lanes) {
+// `slots` = scan CTAs the whole GPU holds at once.
+int auto_splits(const wkv_config& c, long long lanes, long long slots) {
   const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
   int s = 1;
   while (s < 16 && lanes * s < 1776 && tiles / (2 * s) >= 4) s *= 2;
@@ -143,6 +202,13 @@ int auto_splits(const wkv_config& c, long long lanes) {
     s = (tiles + 31) / 32;
     if (s > wkv::kMaxSplits) s = wkv::kMaxSplits;
     if (s < 1) s = 1;
+    // ... unless the units then fill the last round of resident CTAs badly: a layer's time is about (rounds of resident
+    // CTAs) x (tiles per unit + a start-up of ~3 tiles); take the split count that makes that product clearly smaller.
+    auto cost = [&](int k) { return ((lanes * k + slots - 1) / slots) * ((tiles + k - 1) / k + 3); };
+    int best = s;
+    for (int k = 1; k <= 16 && tiles / k >= 8; ++k)
+      if (cost(k) < cost(best)) best = k;
+    if (cost(best) * 26 < cost(s) * 25) s = best;
   }
   return s;
 }
@@ -163,7 +229,7 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   const int smem = C::kFixedBytes + (cluster ? G * P.chunk_cap * 4 : 0);
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
-  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_kernel<T, D, G>;
+  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_entry<T, D, G>();
   if (attr_done[dev][cluster] < smem) {
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -187,7 +253,7 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
     k1.stream = stream;
     k1.attrs = pdl;
     k1.numAttrs = 1;
-    e = cudaLaunchKernelEx(&k1, wkv::scan_kernel<T, D, G>, P);
+    e = cudaLaunchKernelEx(&k1, wkv::scan_entry<T, D, G>(), P);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t k2 = {};
     k2.gridDim = dim3((unsigned)lanes);
@@ -256,6 +322,7 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   P.chunk_cap = c->chunk_cap;
   P.merge = c->cfg.merge;
   P.scale = c->scale;
+  std::memcpy(P.vmap, c->vmap, sizeof(P.vmap));
   return P;
 }
 
@@ -375,7 +442,8 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   c->lanes_per_layer = cfg->batch * cfg->n_kv_heads;
   c->lanes_total = (long long)cfg->n_layers * c->lanes_per_layer;
   c->cap = (cfg->budget + 1 + 3) & ~3;
-  c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_per_layer);
+  const long long slots = (long long)c->sm_count * scan_ctas_per_sm(*cfg);
+  c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_per_layer, slots);
   {
     const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
     c->chunk_cap = ((tiles + c->n_splits - 1) / c->n_splits) * wkv::kTileSlots;   // the largest share of an even deal
@@ -395,7 +463,7 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     // One launch for all layers: the lanes of all layers are just more lanes.  Worth it when a layer alone cannot
     // fill the GPU; allowed when the scratch for every lane at once stays small.
     const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
-    c->fused_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_total);
+    c->fused_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_total, slots);
     c->fused_chunk_cap = ((tiles + c->fused_splits - 1) / c->fused_splits) * wkv::kTileSlots;
     const bool can_cluster = is_cluster_size(c->fused_splits) && c->group * c->fused_chunk_cap * 4 <= 64 * 1024;
     c->fused_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ? can_cluster
@@ -436,6 +504,8 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   T(take(c, &c->stage_v, (size_t)c->lanes_total * row));
   T(take(c, &c->stage_out, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row));
   T(take(c, &c->stage_ev, (size_t)c->lanes_total * 4));
+  if (rc == WKV_OK && c->group == 4 && cfg->dtype == WKV_BF16)
+    rc = encode_value_map(c, c->Vc, (unsigned long long)c->lanes_total * cap, cfg->head_dim);
   if (rc == WKV_OK) rc = run_reset(c);
   if (rc != WKV_OK) {
     wkv_destroy(c);

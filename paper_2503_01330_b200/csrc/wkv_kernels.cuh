@@ -85,6 +85,9 @@ struct StepParams {
   int merge;
   int wait_at_start;     // scan kernel: how it orders itself against the preceding kernel, 0 / 1 / 2 (see scan_kernel)
   float scale;
+  // Tensor map over the value cache as a [lanes_total * cap][D] matrix: boxes of 64 elements x 32 rows, 128-byte
+  // swizzle.  Encoded by the host for configurations whose scan takes its V tiles that way (Cfg::kMmaPV), else unused.
+  alignas(64) unsigned char vmap[128];
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -135,6 +138,14 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                    smem_u32(dst)),
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Tiled tensor-map copy global -> this CTA's shared memory: the box of `tmap` whose first element is (x, y) = (element
+// in the row, row).  x * element size must be a multiple of 16 bytes; dst 128-byte aligned (1024 for swizzled boxes).
+__device__ __forceinline__ void tensor_g2s_2d(void* dst, const void* tmap, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                   smem_u32(dst)),
+               "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
                : "memory");
 }
 // Hint: bring [src, src + bytes) into L2.  src 16-byte aligned, bytes a multiple of 16.
@@ -241,6 +252,21 @@ __device__ __forceinline__ void load_pairs(const __nv_bfloat16* p, f32x2 (&x)[NP
   }
 }
 
+// Tensor-core pieces of the P.V half for four query heads (bf16 rows).  D[16x8] += A[16x8] * B[8x8], fp32 accumulate.
+__device__ __forceinline__ void mma_m16n8k8_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5}, {%6}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(b0));
+}
+// Four transposed 8x8 bf16 matrices; lanes 8i..8i+7 give the row addresses of matrix i (16 bytes each, shared memory).
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], const void* row_addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(smem_u32(row_addr))
+               : "memory");
+}
+__device__ __forceinline__ uint32_t bf16_bits(__nv_bfloat16 x) { return (uint32_t)__bfloat16_as_ushort(x); }
+
 // ------------------------------------------------------------------------------------------------
 // reproducible exp (see the header comment)
 // ------------------------------------------------------------------------------------------------
@@ -304,11 +330,19 @@ struct EpScratch {
 template <typename T, int D, int G>
 struct Cfg {
   static constexpr int kRowBytes = D * (int)sizeof(T);
-  static constexpr int kTileBytes = kTileSlots * kRowBytes; // one of K or V
+  static constexpr int kTileBytes = kTileSlots * kRowBytes; // the K tile of a stage
   static constexpr int kLanesPerRow = G <= 2 ? 8 : 16;      // threads that share one cache row in the scan
+  // Four query heads on bf16 rows: the P.V half of the scan (outside the reproducible chain) runs on mma.m16n8k8 with
+  // the value fragments fetched by ldmatrix.trans.  The V tile of a stage is then written by tensor-map copies with the
+  // 128-byte swizzle, one per 128-byte half of the rows ([half][32 rows][128 B], the 16-byte chunk index XORed with
+  // row % 8), so that the eight rows of a fragment fall into eight different bank groups.
+  static constexpr bool kMmaPV = G == 4 && sizeof(T) == 2 && D % 64 == 0;
+  static constexpr int kVHalves = kRowBytes / 128;          // kMmaPV only
+  static constexpr int kVHalfBytes = kTileSlots * 128;
+  static constexpr int kStageBytes = 2 * kTileBytes;
   static constexpr int kFit = WKV_RING_BYTES / (2 * kTileBytes);
   static constexpr int kStages = kFit < 2 ? 2 : (kFit > 8 ? 8 : kFit);
-  static constexpr int kRingBytes = kStages * 2 * kTileBytes;
+  static constexpr int kRingBytes = kStages * kStageBytes;
   static constexpr int kAuxBytes = 2 * kRowBytes;           // k row and v row of the new token
   static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
   static constexpr int kCtaPartFloats = G * (D + 2);
@@ -382,6 +416,28 @@ __device__ __forceinline__ void fill_view(LaneView<T>& v, const StepParams& P, i
   v.slot_end = min(v.L, (v.tile_begin + v.n_tiles) * kTileSlots);
 }
 
+// Producer side of one ring stage (one thread): `rows` cache rows of K in one bulk copy and the same rows of V in one
+// more -- or, where the stage keeps its V rows swizzled (Cfg::kMmaPV), whole 32-row boxes of V through the tensor map
+// `vmap` over the value cache as a [rows_total][D] matrix, starting at row `vrow0` (rows past the lane's entries are
+// other slots' bytes or, past the end of the cache, zero fill; the consumers never use them).
+template <typename T, int D, int G>
+__device__ __forceinline__ void fill_stage(unsigned char* dst, const T* Ksrc, const T* Vsrc, int rows, uint64_t* bar,
+                                           const void* vmap, int vrow0) {
+  using C = Cfg<T, D, G>;
+  const uint32_t bytes = (uint32_t)rows * C::kRowBytes;
+  if constexpr (!C::kMmaPV) {
+    mbar_expect_tx(bar, 2 * bytes);
+    bulk_g2s(dst, Ksrc, bytes, bar);
+    bulk_g2s(dst + C::kTileBytes, Vsrc, bytes, bar);
+  } else {
+    mbar_expect_tx(bar, bytes + C::kVHalves * C::kVHalfBytes);
+    bulk_g2s(dst, Ksrc, bytes, bar);
+#pragma unroll
+    for (int h = 0; h < C::kVHalves; ++h)
+      tensor_g2s_2d(dst + C::kTileBytes + h * C::kVHalfBytes, vmap, h * 64, vrow0, bar);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // the scan: per-thread state of the four consumer warps (each warp owns 8 rows of every tile)
 // ------------------------------------------------------------------------------------------------
@@ -402,9 +458,15 @@ struct Scanner {
   // bookkeeping is done once per head instead of once per thread.  The additions are those of the plain butterfly.
   static constexpr int LH = LPR / G;             // threads per (row, head) after the reduce-scatter
   static_assert(G <= LPR && LH >= 1, "at most one head per thread of a row");
+  // P.V on the tensor cores (C::kMmaPV): per warp and tile, (V rows)^T [channels x 8 rows] times the probabilities
+  // [8 rows x (4 heads as bf16 high parts | 4 heads as bf16 low parts)], in blocks of 16 channels.  Lane t = 4*c + q holds
+  // channels 16*blk + c and 16*blk + 8 + c of columns 2q and 2q+1; end() adds the low-part columns to the high-part ones.
+  static constexpr bool MMA = C::kMmaPV;
+  static constexpr int NB = D / 16;              // channel blocks
   f32x2 qf[G][NP][CP];
   float m_run, l_run;                            // online softmax of this thread's head: head_of(l) = l / LH
-  f32x2 o_acc[G][NP][CP];
+  f32x2 o_acc[MMA ? 1 : G][NP][CP];
+  float oc[MMA ? NB : 1][4];
 
   __device__ __forceinline__ void begin(const T* q) {      // q: [G][D], 16-byte aligned (global or shared)
     const int l = (threadIdx.x & 31) % LPR;
@@ -414,11 +476,25 @@ struct Scanner {
     for (int g = 0; g < G; ++g) {
 #pragma unroll
       for (int j = 0; j < NP; ++j) load_pairs<CP>(q + g * D + (l + LPR * j) * CH, qf[g][j]);
+      if constexpr (!MMA) {
 #pragma unroll
-      for (int j = 0; j < NP; ++j)
+        for (int j = 0; j < NP; ++j)
 #pragma unroll
-        for (int e = 0; e < CP; ++e) o_acc[g][j][e] = 0ull;
+          for (int e = 0; e < CP; ++e) o_acc[g][j][e] = 0ull;
+      }
     }
+    if constexpr (MMA) {
+#pragma unroll
+      for (int j = 0; j < NB; ++j) oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.f;
+    }
+  }
+  // 32-bit word w of row `row` of a stage's V tile: plain rows, or (MMA) the swizzled halves that the tensor-map copies
+  // leave -- [half][row][128 B] with address bits 4..6 XORed with bits 7..9 (the tile starts on a 1024-byte boundary).
+  __device__ __forceinline__ static uint32_t* v_word(T* tV, int row, int w) {
+    if constexpr (!MMA) return reinterpret_cast<uint32_t*>(tV + row * D) + w;
+    unsigned char* base = reinterpret_cast<unsigned char*>(tV);
+    const int chunk = w >> 2;                                           // 16-byte chunk of the row
+    return reinterpret_cast<uint32_t*>(base + (chunk >> 3) * C::kVHalfBytes + row * 128 + ((((chunk & 7) ^ (row & 7)) << 4) | ((w & 3) << 2)));
   }
 
   // value of head g's owner threads, for every thread of the row group
@@ -441,10 +517,9 @@ struct Scanner {
       const int ns_row = new_slot - slot0;
       if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
         uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
-        uint32_t* dv = reinterpret_cast<uint32_t*>(tV + ns_row * D);
         const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
         const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
-        for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; dv[w] = sv_[w]; }
+        for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; *v_word(tV, ns_row, w) = sv_[w]; }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
         __syncwarp();
       }
@@ -503,6 +578,7 @@ struct Scanner {
       float mt = sv[0];
 #pragma unroll
       for (int ps = 1; ps < PASSES; ++ps) mt = fmaxf(mt, sv[ps]);
+      if constexpr (MMA) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 16));   // one accumulator for the warp's 8 rows
       const float m_new = fmaxf(m_run, mt);
       const float m_use = m_new == -INFINITY ? 0.f : m_new;
       corr = fast_exp2((m_run - m_use) * kLog2e);
@@ -514,6 +590,41 @@ struct Scanner {
         l_run += sv[ps];
       }
     }
+    if constexpr (MMA) {
+      static_assert(PASSES == 4 && LH == 4 && RPP == 2, "fragment layout below assumes 16 threads per row, 4 heads");
+      if (__any_sync(0xffffffffu, corr != 1.0f)) {
+        const int src = (lane_id & 1) * 8;                             // my columns' heads: 2*(q & 1) and the next one
+        const float ca = __shfl_sync(0xffffffffu, corr, src), cb = __shfl_sync(0xffffffffu, corr, src + LH);
+#pragma unroll
+        for (int j = 0; j < NB; ++j) { oc[j][0] *= ca; oc[j][1] *= cb; oc[j][2] *= ca; oc[j][3] *= cb; }
+      }
+      if (slot0 + kTileSlots > L) {
+        // ragged tile: rows beyond L hold stale bytes, possibly NaN patterns, and 0 * NaN would reach the accumulators
+        for (int w = lane_id; w < 8 * (C::kRowBytes / 4); w += 32) {
+          const int r = w / (C::kRowBytes / 4);
+          if (slot0 + warp * 8 + r >= L) *v_word(tV, warp * 8 + r, w % (C::kRowBytes / 4)) = 0u;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+      }
+      // B fragment: lane t = 4*n + q supplies rows 2q, 2q+1 of column n (n < 4: head n, high part; else head n-4, low
+      // part).  Row 2q is pass q of row group 0, row 2q+1 pass q of row group 1; head n % 4 is this lane's own head.
+      const float mine = li == 0 ? sv[0] : (li == 1 ? sv[1] : (li == 2 ? sv[2] : sv[3]));
+      const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
+      const bool up = lane_id >= 16;
+      const float pe = up ? other : mine, po = up ? mine : other;
+      const __nv_bfloat16 he = __float2bfloat16_rn(pe), ho = __float2bfloat16_rn(po);
+      const __nv_bfloat16 le = __float2bfloat16_rn(pe - __bfloat162float(he)), lo = __float2bfloat16_rn(po - __bfloat162float(ho));
+      const uint32_t b0 = up ? (bf16_bits(le) | (bf16_bits(lo) << 16)) : (bf16_bits(he) | (bf16_bits(ho) << 16));
+      // lanes 8i..8i+7 address rows 0..7 of the warp's share, 16-byte chunk 4*jj + i of the row (channels 32*jj + 8*i ...)
+#pragma unroll
+      for (int jj = 0; jj < NB / 2; ++jj) {
+        uint32_t af[4];
+        ldmatrix_x4_trans(af, v_word(tV, warp * 8 + (lane_id & 7), (4 * jj + (lane_id >> 3)) * 4));
+        mma_m16n8k8_bf16(oc[2 * jj], af[0], af[1], b0);
+        mma_m16n8k8_bf16(oc[2 * jj + 1], af[2], af[3], b0);
+      }
+    } else {
     // the running maxima settle after a few tiles: rescale the output accumulators only when some head's maximum moved
     if (__any_sync(0xffffffffu, corr != 1.0f)) {
 #pragma unroll
@@ -546,6 +657,7 @@ struct Scanner {
         }
       }
     }
+    }  // !MMA
   }
 
   // Fold the warp's row groups and leave the warp's partial (m, l, o[D]) per query head in shared memory.
@@ -554,6 +666,30 @@ struct Scanner {
     const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
     const int rg = lane_id / LPR, l = lane_id % LPR;
     const int my_head = l / LH, li = l % LH;
+    if constexpr (MMA) {
+      l_run += __shfl_xor_sync(0xffffffffu, l_run, 16);               // both row groups ran on the same maximum
+      const int c = lane_id >> 2, q = lane_id & 3;
+#pragma unroll
+      for (int j = 0; j < NB; ++j)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) oc[j][i] += __shfl_xor_sync(0xffffffffu, oc[j][i], 2);   // high-part + low-part columns
+      if (q < 2) {
+        float* wa = warp_part + (warp * G + 2 * q) * (D + 2) + 2;
+        float* wb = wa + (D + 2);
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+          wa[16 * j + c] = oc[j][0];
+          wb[16 * j + c] = oc[j][1];
+          wa[16 * j + 8 + c] = oc[j][2];
+          wb[16 * j + 8 + c] = oc[j][3];
+        }
+      }
+      if (rg == 0 && li == 0) {
+        float* wp = warp_part + (warp * G + my_head) * (D + 2);
+        wp[0] = m_run;
+        wp[1] = l_run;
+      }
+    } else {
 #pragma unroll
     for (int off = 16; off >= LPR; off >>= 1) {
       const float m_o = __shfl_xor_sync(0xffffffffu, m_run, off);     // same head on both sides
@@ -594,6 +730,7 @@ struct Scanner {
         wp[1] = l_run;
       }
     }
+    }  // !MMA
   }
 };
 
@@ -899,11 +1036,11 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
 // on the finished scratch: o_t, probabilities, score fold, pick, merge, relink.
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
+__device__ __forceinline__ void scan_body(const StepParams& P) {
   using C = Cfg<T, D, G>;
   constexpr int kStages = C::kStages;
   constexpr int NT = kThreads;
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
   const Smem<T, D, G> sm(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
   const int split = blockIdx.x % P.n_splits;
@@ -944,11 +1081,8 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
   auto issue_tile = [&](int i) {
     const int s = i % kStages;
     const int slot0 = (v.tile_begin + i) * kTileSlots;
-    const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
-    unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
-    mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
-    bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
-    bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+    fill_stage<T, D, G>(sm.ring + (size_t)s * C::kStageBytes, v.Kl + (long long)slot0 * D, v.Vl + (long long)slot0 * D,
+                        min(kTileSlots, v.L - slot0), &sm.full_bar[s], P.vmap, (int)(v.lane * P.cap) + slot0);
   };
   if (tid == kConsumerWarps * 32) {
     for (int s = 0; s < kStages; ++s) {
@@ -986,8 +1120,8 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
     for (int i = 0; i < v.n_tiles; ++i) {
       const int s = i % kStages;
       mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
-      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
-      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes);
+      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes + C::kTileBytes);
       sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, lg, P.cap, 0);
       release_stage(&sm.empty_bar[s]);
     }
@@ -1004,6 +1138,23 @@ __global__ void __launch_bounds__(kThreads) scan_kernel(const StepParams P) {
     }
   }
   if (!P.wait_at_start) griddep_wait();
+}
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads) scan_kernel(const __grid_constant__ StepParams P) {
+  scan_body<T, D, G>(P);
+}
+// The same scan for the instantiations with the tensor-core P.V half (Cfg::kMmaPV), held to the registers of four CTAs
+// per SM (a second argument to __launch_bounds__ changes the compiler's choices even when it is 1, hence two entries).
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kThreads, 4) scan_kernel_mma(const __grid_constant__ StepParams P) {
+  scan_body<T, D, G>(P);
+}
+// the entry that a configuration's scan is launched through
+template <typename T, int D, int G>
+inline auto scan_entry() -> void (*)(const StepParams) {
+  if constexpr (Cfg<T, D, G>::kMmaPV) return scan_kernel_mma<T, D, G>;
+  else return scan_kernel<T, D, G>;
 }
 
 constexpr int kEpilogueThreads = 256;
@@ -1072,12 +1223,12 @@ __global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
 // co-scheduled CTAs; every CTA of an active lane reaches every barrier.
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const StepParams P) {
+__global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const __grid_constant__ StepParams P) {
   namespace cg = cooperative_groups;
   using C = Cfg<T, D, G>;
   constexpr int kStages = C::kStages;
   constexpr int NT = kThreads;
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
   const Smem<T, D, G> sm(smem_raw);
   const float kLog2e = 1.4426950408889634f;
   cg::cluster_group cluster = cg::this_cluster();
@@ -1140,11 +1291,9 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
         const int s = i % kStages;
         if (i >= kStages) mbar_wait(&sm.empty_bar[s], ((i / kStages) - 1) & 1, P.status);
         const int slot0 = (v.tile_begin + i) * kTileSlots;
-        const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
-        unsigned char* dst = sm.ring + (size_t)s * 2 * C::kTileBytes;
-        mbar_expect_tx(&sm.full_bar[s], 2 * bytes);
-        bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
-        bulk_g2s(dst + C::kTileBytes, v.Vl + (long long)slot0 * D, bytes, &sm.full_bar[s]);
+        fill_stage<T, D, G>(sm.ring + (size_t)s * C::kStageBytes, v.Kl + (long long)slot0 * D,
+                            v.Vl + (long long)slot0 * D, min(kTileSlots, v.L - slot0), &sm.full_bar[s], P.vmap,
+                            (int)(v.lane * P.cap) + slot0);
       }
     }
   } else {
@@ -1153,8 +1302,8 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const Ste
     for (int i = 0; i < v.n_tiles; ++i) {
       const int s = i % kStages;
       mbar_wait(&sm.full_bar[s], (i / kStages) & 1, P.status);
-      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes);
-      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * 2 * C::kTileBytes + C::kTileBytes);
+      T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes);
+      T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes + C::kTileBytes);
       sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, sm.chunk_logits,
               P.chunk_cap, v.slot_begin);
       release_stage(&sm.empty_bar[s]);
