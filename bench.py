@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090246000 + 26968000 + 12905000, "f5e624d6f4906d22")}
+NCU_TRAFFIC = {"serving_b16": (1090240000 + 26967000 + 12462000, "a41d72c730b10507")}
 
 
 def kernel_source_hash() -> str:

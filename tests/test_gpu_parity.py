@@ -36,6 +36,8 @@ def test_tiny_config_every_step():
     ("bf16", 64, 4, 4, 33, 5, 2, 5, 100),      # more splits than tiles
     ("bf16", 128, 8, 4, 64, 16, 0, 2, 160),    # group of 2
     ("bf16", 128, 8, 2, 95, 16, 1, 0, 200),    # group of 4
+    ("bf16", 64, 8, 2, 70, 4, 0, 3, 170),      # group of 4 on 128-byte rows (one swizzled half per value tile), ragged tail
+    ("bf16", 128, 16, 4, 45, 6, 2, 5, 130),    # group of 4: the last tile's box reaches past the lane and, for the last lane, past the cache
     ("f32", 64, 8, 1, 31, 3, 0, 1, 90),        # group of 8, exactly one tile
     ("f32", 64, 2, 2, 1, 1, 0, 0, 20),         # smallest possible cache
     ("bf16", 128, 2, 2, 8, 8, 0, 0, 40),       # window == budget: a single candidate
