@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090240000 + 26967000 + 12462000, "a41d72c730b10507")}
+NCU_TRAFFIC = {"serving_b16": (1090404000 + 26966000 + 12344000, "bee9d73b4de8119d")}
 
 
 def kernel_source_hash() -> str:

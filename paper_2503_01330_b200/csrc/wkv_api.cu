@@ -268,6 +268,12 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
     if constexpr (G <= 2) {
       if (wide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P);
     }
+    if constexpr (G == 4) {
+      if (lanes <= 2 * sms) {
+        k2.blockDim = dim3(wkv::kEpilogueThreadsMid);
+        return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel_mid<T, D, G>, P);
+      }
+    }
     return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P);
   }
   cudaLaunchConfig_t lc = {};

@@ -1163,7 +1163,7 @@ constexpr int kEpilogueThreadsWide = 512;     // one or two query heads only (re
 // NT threads per lane: kEpilogueThreads, or kEpilogueThreadsWide when a layer has so few lanes that two wide CTAs per
 // SM still hold them all -- the epilogue is a chain of load -> compute rounds, and twice the threads halve the rounds.
 template <typename T, int D, int G, int NT>
-__global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
+__device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
   __shared__ __align__(16) unsigned char ep_raw[EpScratch::bytes(G)];
   EpScratch ep;
   ep.carve(ep_raw, G);
@@ -1216,6 +1216,17 @@ __global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
     if (threadIdx.x == 0) P.ticket[lane_local] = 0u;     // ready for the next call that uses this scratch set
     griddep_wait();                                      // keeps "this grid complete => the scan complete" literally true
   }
+}
+
+template <typename T, int D, int G, int NT>
+__global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
+  lane_epilogue_body<T, D, G, NT>(P);
+}
+// Four query heads, a layer of at most two lanes per SM: 384 threads per lane, held to the registers of two CTAs per SM.
+constexpr int kEpilogueThreadsMid = 384;
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kEpilogueThreadsMid, 2) lane_epilogue_kernel_mid(const StepParams P) {
+  lane_epilogue_body<T, D, G, kEpilogueThreadsMid>(P);
 }
 
 // ------------------------------------------------------------------------------------------------
