@@ -80,7 +80,9 @@ const char* wkv_config_error(const wkv_config* cfg);
 
 /* Validates cfg, allocates the cache and bookkeeping for n_layers*batch*n_kv_heads lanes on the current
  * CUDA device through the provider and clears them.  *out is NULL on failure.  (Algorithm 1: "a, n are
- * empty lists".) */
+ * empty lists".)  With four query heads per key on bf16 rows the cache scan takes its value tiles through a
+ * tensor map, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
+ * the driver lacks it, WKV_ERR_INVALID if the value cache would have 2^31 rows or more. */
 int wkv_create(const wkv_config* cfg, wkv_ctx** out);
 
 /* Releases everything obtained from the provider.  NULL is accepted. */
