@@ -38,6 +38,7 @@ def test_tiny_config_every_step():
     ("bf16", 128, 8, 2, 95, 16, 1, 0, 200),    # group of 4
     ("bf16", 64, 8, 2, 70, 4, 0, 3, 170),      # group of 4 on 128-byte rows (one swizzled half per value tile), ragged tail
     ("bf16", 128, 16, 4, 45, 6, 2, 5, 130),    # group of 4: the last tile's box reaches past the lane and, for the last lane, past the cache
+    ("f32", 128, 8, 2, 60, 4, 1, 2, 140),      # group of 4 on fp32 rows (plain value tiles, 384-thread lane epilogue)
     ("f32", 64, 8, 1, 31, 3, 0, 1, 90),        # group of 8, exactly one tile
     ("f32", 64, 2, 2, 1, 1, 0, 0, 20),         # smallest possible cache
     ("bf16", 128, 2, 2, 8, 8, 0, 0, 40),       # window == budget: a single candidate
