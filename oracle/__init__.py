@@ -57,6 +57,8 @@ def lib():
         L.wkvo_dropped_score.restype = C.c_double
         L.wkvo_dropped_score.argtypes = [C.c_void_p, C.c_int32]
         L.wkvo_last_step.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 4
+        L.wkvo_impose_pick.argtypes = [C.c_void_p, C.c_void_p]
+        L.wkvo_last_pick.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 4
         L.wkvo_export.argtypes = [C.c_void_p, C.c_int32] + [C.c_void_p] * 7
         L.wkvo_import.restype = C.c_int32
         L.wkvo_import.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int64] + [C.c_void_p] * 4
@@ -129,6 +131,21 @@ class Oracle:
         wj, wr, ps = C.c_double(), C.c_double(), C.c_double()
         lib().wkvo_last_step(self._h, lane, C.byref(idx), C.byref(wj), C.byref(wr), C.byref(ps))
         return idx.value, wj.value, wr.value, ps.value
+
+    def impose_pick(self, pos):
+        """Every lane with pos[lane] >= 0 removes the entry at that original position on its next compressing step
+        instead of its own argmin (one shot; used to keep two arithmetic modes on one trajectory across a near-tie)."""
+        pos = np.ascontiguousarray(pos, np.int32).reshape(self.n_lanes)
+        lib().wkvo_impose_pick(self._h, _ptr(pos))
+
+    def last_pick(self, lane=0):
+        """(position the lane's own argmin chose, its average score, the average score of the entry actually removed,
+        1 if an imposed position was outside the evictable range) for the lane's last compressing step."""
+        own = C.c_int32()
+        bad = C.c_int32()
+        oa, ta = C.c_double(), C.c_double()
+        lib().wkvo_last_pick(self._h, lane, C.byref(own), C.byref(oa), C.byref(ta), C.byref(bad))
+        return own.value, oa.value, ta.value, bad.value
 
     def import_state(self, lane, tokens, pos, a, K, V):
         """Replace one lane by a position-ordered state (pos int32 strictly increasing and < tokens; K, V as stored)."""

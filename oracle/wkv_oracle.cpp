@@ -161,6 +161,12 @@ struct Lane {
   int32_t last_evicted_index = -1;
   double last_wj = 0.0, last_wr = 0.0;
   double last_prob_sum = 0.0;
+  // the pick of the last compressing step: what the lane's own argmin chose and what was removed (they differ only
+  // when the caller imposed the removal, see wkvo_impose_pick)
+  int32_t last_own_pos = -1;
+  double last_own_abar = 0.0, last_taken_abar = 0.0;
+  int32_t imposed_pos = -1;                // one-shot: position to remove at the next compressing step, -1 = own argmin
+  int32_t last_imposed_bad = 0;            // the imposed position was not in the evictable range (own argmin used)
 };
 
 }  // namespace
@@ -241,23 +247,27 @@ void wkvo_step(wkvo* o, const float* q, const float* k, const float* v, const ui
     }
     const int L = (int)S.K.size();
 
-    std::vector<std::vector<double>> pd(G, std::vector<double>(L));
+    // In mode 1 the fp64 probabilities serve the output only: a caller that asks for no output does not pay for them.
+    const bool need_fp64 = c.mode == 0 || out != nullptr;
+    std::vector<std::vector<double>> pd(G, std::vector<double>(need_fp64 ? L : 0));
     std::vector<std::vector<float>> pf(G);
     for (int g = 0; g < G; ++g) {
       std::vector<float> qr(d);
       for (int ch = 0; ch < d; ++ch) qr[ch] = store_from_float(q[((size_t)ln * G + g) * d + ch], c.dtype);
-      // Background: A_t = softmax(q_t^T K_t) (scaled), o_t = A_t^T V_t -- the fp64 definition.
-      std::vector<double> s(L);
-      double M = -INFINITY;
-      for (int i = 0; i < L; ++i) {
-        double acc = 0.0;
-        for (int ch = 0; ch < d; ++ch) acc += (double)qr[ch] * (double)S.K[i][ch];
-        s[i] = o->scale * acc;
-        M = std::max(M, s[i]);
+      if (need_fp64) {
+        // Background: A_t = softmax(q_t^T K_t) (scaled), o_t = A_t^T V_t -- the fp64 definition.
+        std::vector<double> s(L);
+        double M = -INFINITY;
+        for (int i = 0; i < L; ++i) {
+          double acc = 0.0;
+          for (int ch = 0; ch < d; ++ch) acc += (double)qr[ch] * (double)S.K[i][ch];
+          s[i] = o->scale * acc;
+          M = std::max(M, s[i]);
+        }
+        double Z = 0.0;
+        for (int i = 0; i < L; ++i) { pd[g][i] = std::exp(s[i] - M); Z += pd[g][i]; }
+        for (int i = 0; i < L; ++i) pd[g][i] /= Z;
       }
-      double Z = 0.0;
-      for (int i = 0; i < L; ++i) { pd[g][i] = std::exp(s[i] - M); Z += pd[g][i]; }
-      for (int i = 0; i < L; ++i) pd[g][i] /= Z;
       if (out) {
         for (int ch = 0; ch < d; ++ch) {
           double acc = 0.0;
@@ -318,6 +328,21 @@ void wkvo_step(wkvo* o, const float* q, const float* k, const float* v, const ui
         }
       }
       // (budget >= sink + window guarantees lo <= hi, so j >= 0 and j+1 exists)
+      auto abar_of = [&](int i) {
+        return c.mode == 1 ? (double)(S.a_f[i] / (float)S.n[i]) : S.a_d[i] / (double)S.n[i];
+      };
+      S.last_own_pos = S.pos[j];
+      S.last_own_abar = abar_of(j);
+      S.last_imposed_bad = 0;
+      if (S.imposed_pos >= 0) {
+        // A caller-imposed removal (wkvo_impose_pick) replaces the lane's own argmin for this one step.
+        int forced = -1;
+        for (int i = lo; i <= hi; ++i)
+          if (S.pos[i] == S.imposed_pos) forced = i;
+        if (forced >= 0) j = forced; else S.last_imposed_bad = 1;
+        S.imposed_pos = -1;
+      }
+      S.last_taken_abar = abar_of(j);
       const int r = j + 1;
       double wj, wr;
       if (c.mode == 1) {
@@ -374,6 +399,24 @@ void wkvo_last_step(const wkvo* o, int32_t lane, int32_t* index, double* wj, dou
   if (wj) *wj = S.last_wj;
   if (wr) *wr = S.last_wr;
   if (prob_sum) *prob_sum = S.last_prob_sum;
+}
+
+// Test hook for comparing two arithmetic modes on one stream.  Algorithm 1 removes the argmin of the average scores;
+// where the two smallest averages lie closer together than binary32 rounding noise, mode 0 and mode 1 may legitimately
+// pick different entries, after which their states are no longer comparable.  wkvo_impose_pick makes every lane with
+// pos[lane] >= 0 remove the entry at that original position on its NEXT compressing step instead of its own argmin
+// (the position must lie in the evictable range, else the lane keeps its own choice and reports it); wkvo_last_pick
+// then tells what the lane would have picked by itself and the average scores of both entries, so that the caller can
+// check that the imposed entry was a near-minimum.  Everything else of the step is unchanged.
+void wkvo_impose_pick(wkvo* o, const int32_t* pos) {
+  for (int32_t ln = 0; ln < o->cfg.n_lanes; ++ln) o->lanes[ln].imposed_pos = pos ? pos[ln] : -1;
+}
+void wkvo_last_pick(const wkvo* o, int32_t lane, int32_t* own_pos, double* own_abar, double* taken_abar, int32_t* imposed_bad) {
+  const Lane& S = o->lanes[lane];
+  if (own_pos) *own_pos = S.last_own_pos;
+  if (own_abar) *own_abar = S.last_own_abar;
+  if (taken_abar) *taken_abar = S.last_taken_abar;
+  if (imposed_bad) *imposed_bad = S.last_imposed_bad;
 }
 
 // Position-ordered copy of a lane.  Any destination may be NULL.

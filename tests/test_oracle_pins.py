@@ -519,6 +519,76 @@ def test_pinned_mode_tracks_double_mode(dtype):
         np.testing.assert_allclose(sp["V"], sd["V"], rtol=tol, atol=tol)
 
 
+def _adopt_and_count(wl, lanes_hk, n_tokens, seed):
+    """Both arithmetic modes on one seeded stream of workload `wl` (kv heads `lanes_hk` of layer 0, sequence 0).
+
+    The binary32 mode decides; the fp64 mode (the definition) must agree with every pick, except where its own two
+    smallest averages are closer than binary32 noise: there the binary32 pick must be within 1e-5 relative of the fp64
+    minimum, and the fp64 side then removes that entry too so that both stay on one trajectory.  Returns
+    (compressions, adoptions, worst relative gap at an adoption)."""
+    from paper_2503_01330_b200.synth import TokenStream
+    dt = F32 if wl.dtype == "f32" else BF16
+    n = len(lanes_hk)
+    od = Oracle(n, wl.head_dim, wl.budget, window=wl.window, sink=wl.sink, group=wl.group, mode=MODE_DOUBLE, dtype=dt)
+    op = Oracle(n, wl.head_dim, wl.budget, window=wl.window, sink=wl.sink, group=wl.group, mode=MODE_PINNED, dtype=dt)
+    stream = TokenStream(wl, seed, "cpu")
+    hk = torch.tensor(lanes_hk)
+    compressions = adoptions = 0
+    worst_gap = 0.0
+    out_tol = 2e-2 if dt == BF16 else 1e-5
+    for t in range(n_tokens):
+        q, k, v = stream.token(t)
+        qs = q[0, 0].view(wl.n_kv_heads, wl.group, wl.head_dim)[hk].float().numpy()
+        ks, vs = k[0, 0][hk].float().numpy(), v[0, 0][hk].float().numpy()
+        out_p, ev_p, _ = op.step(qs, ks, vs)
+        od.impose_pick(ev_p)
+        out_d, ev_d, _ = od.step(qs, ks, vs)
+        np.testing.assert_array_equal(ev_d, ev_p)                   # the imposed entry was removed
+        for lane in range(n):
+            if ev_p[lane] < 0:
+                continue
+            compressions += 1
+            own_pos, own_abar, taken_abar, bad = od.last_pick(lane)
+            assert not bad, (t, lane, "the binary32 pick lies outside the fp64 side's evictable range")
+            if own_pos != ev_p[lane]:
+                adoptions += 1
+                gap = (taken_abar - own_abar) / own_abar
+                worst_gap = max(worst_gap, gap)
+                assert 0.0 <= gap <= 1e-5, (t, lane, own_pos, int(ev_p[lane]), own_abar, taken_abar)
+        # outputs: both are the fp64 definition on values that differ only by the rounding of the merge weights
+        np.testing.assert_allclose(out_p, out_d, rtol=0, atol=out_tol)
+    for lane in range(n):
+        sd, sp = od.export(lane), op.export(lane)
+        np.testing.assert_array_equal(sd["pos"], sp["pos"])
+        np.testing.assert_allclose(sp["a"], sd["a"], rtol=2e-5, atol=1e-9)
+    od.close()
+    op.close()
+    return compressions, adoptions, worst_gap
+
+
+def test_pinned_sequence_is_the_fp64_sequence_up_to_near_ties_tiny_config():
+    """The whole `tiny` configuration (4 lanes, 256 + 256 tokens): the binary32 eviction sequence against Algorithm 1
+    in fp64, adopt-and-count."""
+    from paper_2503_01330_b200.synth import BASE_SEED, WORKLOADS
+    wl = WORKLOADS["tiny"]
+    comp, adopted, gap = _adopt_and_count(wl, list(range(wl.n_kv_heads)), wl.prefill + wl.decode, BASE_SEED)
+    assert comp == wl.n_kv_heads * (wl.prefill + wl.decode - wl.budget)
+    print(f"tiny: {comp} compressions, {adopted} adoptions, worst relative gap {gap:.2e}")
+    assert adopted <= 2
+
+
+def test_pinned_sequence_is_the_fp64_sequence_up_to_near_ties_llama7b_layer():
+    """Two lanes of the single-layer Llama-2-7B-shaped configuration (bf16, budget 2048, window 64) over the whole
+    4096-token prompt and 256 decode steps: 2304 compressions per lane."""
+    from paper_2503_01330_b200.synth import BASE_SEED, WORKLOADS
+    wl = WORKLOADS["llama7b_layer"]
+    n_tokens = wl.prefill + 256
+    comp, adopted, gap = _adopt_and_count(wl, [3, 29], n_tokens, BASE_SEED + 1)
+    assert comp == 2 * (n_tokens - wl.budget)
+    print(f"llama7b_layer: {comp} compressions, {adopted} adoptions, worst relative gap {gap:.2e}")
+    assert adopted <= 8                                              # near-ties are rare: a handful in 4608 decisions
+
+
 # ---------------------------------------------------------------------------------------------
 # the Ideal Merging section: the closed form really leaves the output unchanged; its two-term cut is convex
 # ---------------------------------------------------------------------------------------------
