@@ -38,7 +38,8 @@ typedef enum {
   WKV_ERR_INVALID = -1, /* bad configuration or argument                                   */
   WKV_ERR_ALLOC = -2,   /* the memory provider returned NULL                               */
   WKV_ERR_CUDA = -3,    /* a CUDA runtime call or launch failed (text in wkv_last_error)    */
-  WKV_ERR_STATE = -4,   /* call order misuse, or exported bookkeeping found inconsistent    */
+  WKV_ERR_STATE = -4,   /* a lane's bookkeeping found inconsistent (host check of an export,
+                           or a kernel's own check of its slot links)                       */
   WKV_ERR_TIMEOUT = -5  /* a bounded device-side wait gave up (device status word)          */
 } wkv_error;
 
@@ -79,8 +80,9 @@ typedef struct {
 const char* wkv_config_error(const wkv_config* cfg);
 
 /* Validates cfg, allocates the cache and bookkeeping for n_layers*batch*n_kv_heads lanes on the current
- * CUDA device through the provider and clears them.  *out is NULL on failure.  (Algorithm 1: "a, n are
- * empty lists".)  With four query heads per key on bf16 rows the cache scan takes its value tiles through a
+ * CUDA device through the provider and clears them (Algorithm 1 starts from empty score and count lists).  *out is
+ * NULL on failure; when the provider returns NULL for one of the blocks the call returns WKV_ERR_ALLOC after handing
+ * every block it had obtained back to `release`.  With four query heads per key on bf16 rows the cache scan takes its value tiles through a
  * tensor map, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
  * the driver lacks it, WKV_ERR_INVALID if the value cache would have 2^31 rows or more. */
 int wkv_create(const wkv_config* cfg, wkv_ctx** out);
@@ -140,7 +142,9 @@ int wkv_decode_step_layers(wkv_ctx* ctx, const void* q, const void* k, const voi
  *          in it has to start at zero: every word the second kernel reads has been written by the first
  *          kernel of the same call.  Calls that can overlap on the GPU (different streams, or different contexts
  *          without ordering between them) race on the array: serialise them.
- *   Calls no cudaMalloc, cudaFree or other allocating routine. */
+ *   Calls no cudaMalloc, cudaFree or other allocating routine.  (The CUDA runtime may load a kernel's code the
+ *          first time that kernel is launched on a device and take device memory for it: run one step of the same
+ *          shape outside the region that must not allocate.) */
 #define WKV_STATIC_SCRATCH_BYTES (4u << 20)
 int wkv_decode_step_static(wkv_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, void* out,
                            int32_t* evicted_pos);
@@ -211,15 +215,21 @@ int wkv_export_slots(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, in
 int wkv_import_state(wkv_ctx* ctx, int32_t layer, int32_t b, int32_t kv_head, int32_t len, int32_t tokens,
                      const int32_t* pos, const float* a, const void* K, const void* V);
 
-/* Reads and clears the device status word (waits for the stream): WKV_OK, or WKV_ERR_TIMEOUT if a bounded
- * wait inside a kernel gave up since the last call. */
+/* Reads and clears the device status word (waits for the stream): WKV_OK, WKV_ERR_TIMEOUT if a bounded wait inside
+ * a kernel gave up since the last call, or WKV_ERR_STATE if a kernel found inconsistent slot links.
+ * After WKV_ERR_TIMEOUT the context accepts calls as before (this call also clears the per-lane arrival counters of
+ * the kernels), but a lane whose step was abandoned has consumed one token less than the others and its outputs of
+ * that step are undefined: wkv_reset the context or wkv_import_state the affected lanes before decoding on. */
 int wkv_status(wkv_ctx* ctx);
 
-/* Self-test of the error path for device-side waits.  Every wait inside the kernels (on a shared-memory barrier fed
- * by a bulk copy) is bounded: after a fixed number of polls the waiting thread sets a bit in the device status word
- * and carries on, so a kernel always terminates.  This call launches a one-thread kernel that waits on a barrier
- * nothing will complete (20000 polls, a few milliseconds); afterwards wkv_status returns WKV_ERR_TIMEOUT once and the
- * context is as usable as before.  Nothing faults or hangs.  Asynchronous. */
+/* Self-test of the error path for device-side waits.  Every wait inside the kernels is bounded: the waits on a
+ * shared-memory barrier fed by a bulk copy, and the lane epilogue's poll of its lane's arrival counter, which the scan
+ * kernel in front of it increments (that kernel's CTAs have all started before an epilogue CTA becomes resident, so
+ * the poll never waits for work that waits for it; at most 2^22 polls of about 100 ns).  After its limit the waiting
+ * thread sets a bit in the device status word and carries on, so a kernel always terminates.  This call launches a
+ * one-thread kernel that waits on a barrier nothing will complete (20000 polls, a few milliseconds); afterwards
+ * wkv_status returns WKV_ERR_TIMEOUT once and the context is as usable as before.  Nothing faults or hangs.
+ * Asynchronous. */
 int wkv_selftest_wait_timeout(wkv_ctx* ctx);
 
 /* Number of kernels this context has launched so far, and bytes it obtained from the provider. */

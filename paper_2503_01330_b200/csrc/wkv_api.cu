@@ -168,8 +168,9 @@ template <typename T, int D, int G>
 int scan_ctas_per_sm_of() {
   using C = wkv::Cfg<T, D, G>;
   int n = 0;
-  if (cudaFuncSetAttribute(wkv::scan_entry<T, D, G>(), cudaFuncAttributeMaxDynamicSharedMemorySize, C::kFixedBytes) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, wkv::scan_entry<T, D, G>(), wkv::kThreads, C::kFixedBytes) != cudaSuccess) {
+  constexpr int smem = wkv::scan_smem_bytes<T, D, G>();
+  if (cudaFuncSetAttribute(wkv::scan_entry<T, D, G>(), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, wkv::scan_entry<T, D, G>(), wkv::kThreads, smem) != cudaSuccess) {
     cudaGetLastError();
     return 4;
   }
@@ -222,22 +223,24 @@ constexpr int kMaxDynSmem = 200 * 1024;
 template <typename T, int D, int G>
 cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaStream_t stream) {
   using C = wkv::Cfg<T, D, G>;
-  static int attr_done[64][2] = {};            // largest dynamic shared memory size configured per device and kernel
+  // largest dynamic shared memory size configured per device and kernel (contexts may be driven from several host
+  // threads: two of them setting the same attribute twice is harmless, a torn read is not)
+  static std::atomic<int> attr_done[64][2];
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  const int smem = C::kFixedBytes + (cluster ? G * P.chunk_cap * 4 : 0);
+  const int smem = cluster ? C::kFixedBytes + G * P.chunk_cap * 4 : wkv::scan_smem_bytes<T, D, G>();
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
   const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_entry<T, D, G>();
-  if (attr_done[dev][cluster] < smem) {
+  if (attr_done[dev][cluster].load(std::memory_order_acquire) < smem) {
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     if (cluster) {
       e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       if (e != cudaSuccess) return e;
     }
-    attr_done[dev][cluster] = smem;
+    attr_done[dev][cluster].store(smem, std::memory_order_release);
   }
   const int n_ctas = lanes * P.n_splits;
   if (!cluster) {
@@ -260,21 +263,24 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const bool wide = G <= 2 && lanes <= 2 * sms;        // two wide CTAs per SM hold every lane at once
-    k2.blockDim = dim3(wide ? wkv::kEpilogueThreadsWide : wkv::kEpilogueThreads);
-    k2.dynamicSmemBytes = 0;
+    const bool mid = G == 4 && lanes <= 2 * sms;
+    const int nt = wide ? wkv::kEpilogueThreadsWide : (mid ? wkv::kEpilogueThreadsMid : wkv::kEpilogueThreads);
+    k2.blockDim = dim3(nt);
     k2.stream = stream;
     k2.attrs = pdl;
     k2.numAttrs = 1;
+    // room to stage a lane's scores and positions in shared memory, when the lane can be finished out of registers
+    wkv::StepParams P2 = P;
+    const int e_slots = wkv::epilogue_slots_per_thread(G, nt) * nt;
+    P2.ep_stage_slots = (e_slots > 0 && P.budget + 1 <= e_slots) ? P.cap : 0;
+    k2.dynamicSmemBytes = (size_t)P2.ep_stage_slots * 8;
     if constexpr (G <= 2) {
-      if (wide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P);
+      if (wide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P2);
     }
     if constexpr (G == 4) {
-      if (lanes <= 2 * sms) {
-        k2.blockDim = dim3(wkv::kEpilogueThreadsMid);
-        return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel_mid<T, D, G>, P);
-      }
+      if (mid) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel_mid<T, D, G>, P2);
     }
-    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P);
+    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P2);
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)n_ctas);
@@ -387,18 +393,18 @@ int run_reset(wkv_ctx* c) {
 
 // Device address of g_static_scratch on the current device, looked up once per device.
 cudaError_t static_scratch_base(unsigned char** base) {
-  static unsigned char* per_device[64] = {};
+  static std::atomic<unsigned char*> per_device[64];       // zero-initialised; every thread would store the same address
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  if (per_device[dev] == nullptr) {
-    unsigned char* p = nullptr;
+  unsigned char* p = per_device[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
     e = cudaGetSymbolAddress((void**)&p, g_static_scratch);
     if (e != cudaSuccess) return e;
-    per_device[dev] = p;
+    per_device[dev].store(p, std::memory_order_release);
   }
-  *base = per_device[dev];
+  *base = p;
   return cudaSuccess;
 }
 
@@ -484,32 +490,34 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   const size_t D = cfg->head_dim, cap = c->cap, G = c->group;
   const size_t row = D * c->elem;
   int rc = WKV_OK;
-  auto T = [&](int r) { if (rc == WKV_OK) rc = r; };
-  T(take(c, &c->Kc, (size_t)c->lanes_total * cap * row));
-  T(take(c, &c->Vc, (size_t)c->lanes_total * cap * row));
-  T(take(c, &c->a, (size_t)c->lanes_total * cap * 4));
-  T(take(c, &c->pos, (size_t)c->lanes_total * cap * 4));
-  T(take(c, &c->next, (size_t)c->lanes_total * cap * 4));
-  T(take(c, &c->prev, (size_t)c->lanes_total * cap * 4));
-  T(take(c, &c->lane_state, (size_t)c->lanes_total * wkv::LS_STRIDE * 4));
+  // one request after the other; after the first refusal the provider is not asked again
+#define WKV_TAKE(dst, bytes) do { if (rc == WKV_OK) rc = take(c, dst, bytes); } while (0)
+  WKV_TAKE(&c->Kc, (size_t)c->lanes_total * cap * row);
+  WKV_TAKE(&c->Vc, (size_t)c->lanes_total * cap * row);
+  WKV_TAKE(&c->a, (size_t)c->lanes_total * cap * 4);
+  WKV_TAKE(&c->pos, (size_t)c->lanes_total * cap * 4);
+  WKV_TAKE(&c->next, (size_t)c->lanes_total * cap * 4);
+  WKV_TAKE(&c->prev, (size_t)c->lanes_total * cap * 4);
+  WKV_TAKE(&c->lane_state, (size_t)c->lanes_total * wkv::LS_STRIDE * 4);
   for (int i = 0; i < 2; ++i) {
-    T(take(c, &c->logits[i], (size_t)c->lanes_per_layer * G * cap * 4));
-    T(take(c, &c->part[i], (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4));
-    T(take(c, &c->ticket[i], (size_t)c->lanes_per_layer * 4));
+    WKV_TAKE(&c->logits[i], (size_t)c->lanes_per_layer * G * cap * 4);
+    WKV_TAKE(&c->part[i], (size_t)c->lanes_per_layer * c->n_splits * G * (D + 2) * 4);
+    WKV_TAKE(&c->ticket[i], (size_t)c->lanes_per_layer * 4);
   }
   if (c->fused_ok) {
-    T(take(c, &c->fused_logits, (size_t)c->lanes_total * G * cap * 4));
-    T(take(c, &c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4));
-    T(take(c, &c->fused_ticket, (size_t)c->lanes_total * 4));
-    T(take(c, &c->fused_seq_lens, (size_t)cfg->n_layers * cfg->batch * 4));
+    WKV_TAKE(&c->fused_logits, (size_t)c->lanes_total * G * cap * 4);
+    WKV_TAKE(&c->fused_part, (size_t)c->lanes_total * c->fused_splits * G * (D + 2) * 4);
+    WKV_TAKE(&c->fused_ticket, (size_t)c->lanes_total * 4);
+    WKV_TAKE(&c->fused_seq_lens, (size_t)cfg->n_layers * cfg->batch * 4);
   }
-  T(take(c, &c->status, 256));
+  WKV_TAKE(&c->status, 256);
   // staging holds one step of all layers (the host entry points copy through it)
-  T(take(c, &c->stage_q, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row));
-  T(take(c, &c->stage_k, (size_t)c->lanes_total * row));
-  T(take(c, &c->stage_v, (size_t)c->lanes_total * row));
-  T(take(c, &c->stage_out, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row));
-  T(take(c, &c->stage_ev, (size_t)c->lanes_total * 4));
+  WKV_TAKE(&c->stage_q, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row);
+  WKV_TAKE(&c->stage_k, (size_t)c->lanes_total * row);
+  WKV_TAKE(&c->stage_v, (size_t)c->lanes_total * row);
+  WKV_TAKE(&c->stage_out, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row);
+  WKV_TAKE(&c->stage_ev, (size_t)c->lanes_total * 4);
+#undef WKV_TAKE
   if (rc == WKV_OK && c->group == 4 && cfg->dtype == WKV_BF16)
     rc = encode_value_map(c, c->Vc, (unsigned long long)c->lanes_total * cap, cfg->head_dim);
   if (rc == WKV_OK) rc = run_reset(c);
@@ -1000,7 +1008,15 @@ int wkv_status(wkv_ctx* c) {
   WKV_CUDA(c, cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost));
   if (w) {
     WKV_CUDA(c, cudaMemset(c->status, 0, 4));
-    if (w & wkv::kStatusWaitTimeout) return fail(c, WKV_ERR_TIMEOUT, "a bounded wait inside a kernel gave up");
+    if (w & wkv::kStatusWaitTimeout) {
+      // A lane epilogue that gave up on its units left their reports uncounted: clear the counters (the stream is
+      // idle), so that the next call's epilogues wait for that call's units and not for stale ones.  The lanes that were
+      // skipped are one token behind; the caller resets or re-imports them (see wkv.h).
+      for (int i = 0; i < 2; ++i) WKV_CUDA(c, cudaMemset(c->ticket[i], 0, (size_t)c->lanes_per_layer * 4));
+      if (c->fused_ticket) WKV_CUDA(c, cudaMemset(c->fused_ticket, 0, (size_t)c->lanes_total * 4));
+      c->last_layer = -1;
+      return fail(c, WKV_ERR_TIMEOUT, "a bounded wait inside a kernel gave up");
+    }
     return fail(c, WKV_ERR_STATE, "a kernel found inconsistent slot links");
   }
   return WKV_OK;
@@ -1025,7 +1041,7 @@ const char* wkv_strerror(int code) {
     case WKV_ERR_INVALID: return "invalid configuration or argument";
     case WKV_ERR_ALLOC: return "device memory provider failed";
     case WKV_ERR_CUDA: return "CUDA runtime error";
-    case WKV_ERR_STATE: return "inconsistent state or call order";
+    case WKV_ERR_STATE: return "inconsistent lane bookkeeping";
     case WKV_ERR_TIMEOUT: return "device-side wait timed out";
   }
   return "unknown error";

@@ -48,7 +48,7 @@ constexpr int kTileSlots = 32;        // cache entries per pipeline stage
 constexpr int kConsumerWarps = 4;     // each owns 8 rows of a tile
 constexpr int kThreads = (kConsumerWarps + 1) * 32;   // + one producer warp
 constexpr int kMaxSplits = 64;
-constexpr uint32_t kSpinLimit = 1u << 22;             // bounded mbarrier polling (each poll sleeps briefly)
+constexpr uint32_t kSpinLimit = 1u << 22;             // polls of a bounded wait (mbarrier, or a lane's arrival counter; each poll sleeps briefly)
 
 enum StatusBits : uint32_t { kStatusWaitTimeout = 1u, kStatusBadLink = 2u };
 
@@ -84,6 +84,7 @@ struct StepParams {
   int chunk_cap;         // cluster kernel: logits one CTA can hold per query head (its tiles * 32)
   int merge;
   int wait_at_start;     // scan kernel: how it orders itself against the preceding kernel, 0 / 1 / 2 (see scan_kernel)
+  int ep_stage_slots;    // lane epilogue kernel: entries of a and pos its dynamic shared memory can stage (0: none)
   float scale;
   // Tensor map over the value cache as a [lanes_total * cap][D] matrix: boxes of 64 elements x 32 rows, 128-byte
   // swizzle.  Encoded by the host for configurations whose scan takes its V tiles that way (Cfg::kMmaPV), else unused.
@@ -311,7 +312,7 @@ struct EpScratch {
   float* Z;                  // [8]
   float* misc;               // [8] w_j, w_r
   int* i32;                  // [64] flags, j, r
-  unsigned long long* u64;   // [128]: [0..63] sums, [64..71] minima, [80..87] Z partial per head, [88..89] pick key
+  unsigned long long* u64;   // [128]: [0..63] sums, [64..95] minima and their slots, [96..103] Z partial per head, [104..105] pick key
   __host__ __device__ static constexpr int bytes(int G) { return (G * kMaxSplits + 32 + 64) * 4 + 128 * 8; }
   __device__ __forceinline__ void carve(unsigned char* base, int G) {
     w = reinterpret_cast<float*>(base);
@@ -504,28 +505,58 @@ struct Scanner {
     return __shfl_sync(0xffffffffu, mine, (lane_id & ~(LPR - 1)) | (g * LH));
   }
 
-  // One tile of up to 32 rows starting at slot0; logits parked at logit_dst[g*logit_stride + slot - logit_off].
-  __device__ __forceinline__ void tile(T* tK, T* tV, int slot0, int L, int new_slot, const T* new_k, const T* new_v,
-                                       float scale, float* logit_dst, long long logit_stride, int logit_off) {
-    const float kLog2e = 1.4426950408889634f;
+  // Tensor-core P.V of one tile (MMA configurations): oc += (the warp's 8 value rows)^T . (their probabilities).
+  // `mine` is the probability of this thread's own (row, head): row 2*li + rg of the warp's eight, head my_head.
+  __device__ __forceinline__ void pv_mma(T* tV, float mine, int slot0, int L) {
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    if (slot0 + kTileSlots > L) {
+      // ragged tile: rows beyond L hold stale bytes, possibly NaN patterns, and 0 * NaN would reach the accumulators
+      for (int w = lane_id; w < 8 * (C::kRowBytes / 4); w += 32) {
+        const int r = w / (C::kRowBytes / 4);
+        if (slot0 + warp * 8 + r >= L) *v_word(tV, warp * 8 + r, w % (C::kRowBytes / 4)) = 0u;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+    }
+    // B fragment: lane t = 4*n + q supplies rows 2q, 2q+1 of column n (n < 4: head n, high part; else head n-4, low
+    // part).  Row 2q is pass q of row group 0, row 2q+1 pass q of row group 1; head n % 4 is this lane's own head.
+    const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
+    const bool up = lane_id >= 16;
+    const float pe = up ? other : mine, po = up ? mine : other;
+    const __nv_bfloat16 he = __float2bfloat16_rn(pe), ho = __float2bfloat16_rn(po);
+    const __nv_bfloat16 le = __float2bfloat16_rn(pe - __bfloat162float(he)), lo = __float2bfloat16_rn(po - __bfloat162float(ho));
+    const uint32_t b0 = up ? (bf16_bits(le) | (bf16_bits(lo) << 16)) : (bf16_bits(he) | (bf16_bits(ho) << 16));
+    // lanes 8i..8i+7 address rows 0..7 of the warp's share, 16-byte chunk 4*jj + i of the row (channels 32*jj + 8*i ...)
+#pragma unroll
+    for (int jj = 0; jj < NB / 2; ++jj) {
+      uint32_t af[4];
+      ldmatrix_x4_trans(af, v_word(tV, warp * 8 + (lane_id & 7), (4 * jj + (lane_id >> 3)) * 4));
+      mma_m16n8k8_bf16(oc[2 * jj], af[0], af[1], b0);
+      mma_m16n8k8_bf16(oc[2 * jj + 1], af[2], af[3], b0);
+    }
+  }
+
+  // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the row in the
+  // tile (the K tile, the V tile or both: a null pointer skips one) with the token's k and v before anybody reads it.
+  __device__ __forceinline__ static void patch_new_token(T* tK, T* tV, int slot0, int new_slot, const T* new_k, const T* new_v) {
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int ns_row = new_slot - slot0;
+    if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
+      const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
+      const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
+      for (int w = lane_id; w < C::kRowBytes / 4; w += 32) {
+        if (tK != nullptr) reinterpret_cast<uint32_t*>(tK + ns_row * D)[w] = sk[w];
+        if (tV != nullptr) *v_word(tV, ns_row, w) = sv_[w];
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
+      __syncwarp();
+    }
+  }
+
+  // Logits of my head for the rows of my row group, one per pass (the reproducible dot; -inf for rows beyond L).
+  __device__ __forceinline__ void logits(const T* tK, int slot0, int L, float scale, float (&sv)[PASSES], bool (&valid)[PASSES]) const {
     const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
     const int rg = lane_id / LPR, l = lane_id % LPR;
-    const int my_head = l / LH, li = l % LH;
-    {
-      // The cache copy of this step's token may still be in flight: the warp that owns its row overwrites the
-      // row in the tile with the token's k and v before anybody reads it.
-      const int ns_row = new_slot - slot0;
-      if (ns_row >= warp * 8 && ns_row < warp * 8 + 8) {
-        uint32_t* dk = reinterpret_cast<uint32_t*>(tK + ns_row * D);
-        const uint32_t* sk = reinterpret_cast<const uint32_t*>(new_k);
-        const uint32_t* sv_ = reinterpret_cast<const uint32_t*>(new_v);
-        for (int w = lane_id; w < C::kRowBytes / 4; w += 32) { dk[w] = sk[w]; *v_word(tV, ns_row, w) = sv_[w]; }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled by a bulk copy
-        __syncwarp();
-      }
-    }
-    float sv[PASSES];                                                // logits of my head, one row per pass
-    bool valid[PASSES];
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
       const int row = warp * 8 + ps * RPP + rg;
@@ -566,12 +597,34 @@ struct Scanner {
       const float sc = __fmul_rn(scale, vals[0]);
       sv[ps] = valid[ps] ? sc : -INFINITY;
     }
-    // park the logits of my head: thread li of the head's LH threads takes the passes ps with ps % LH == li
+  }
+
+  // Park the logits of my head at logit_dst[head * logit_stride + slot - logit_off]: thread li of the head's LH threads
+  // takes the passes ps with ps % LH == li.
+  __device__ __forceinline__ static void park(const float (&sv)[PASSES], int slot0, int L, float* logit_dst,
+                                              long long logit_stride, int logit_off) {
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
+    const int my_head = l / LH, li = l % LH;
 #pragma unroll
     for (int ps = 0; ps < PASSES; ++ps) {
       const int slot = slot0 + warp * 8 + ps * RPP + rg;
       if ((ps % LH) == li && slot < L) logit_dst[(long long)my_head * logit_stride + (slot - logit_off)] = sv[ps];
     }
+  }
+
+  // One tile of up to 32 rows starting at slot0; logits parked at logit_dst[g*logit_stride + slot - logit_off].
+  __device__ __forceinline__ void tile(T* tK, T* tV, int slot0, int L, int new_slot, const T* new_k, const T* new_v,
+                                       float scale, float* logit_dst, long long logit_stride, int logit_off) {
+    const float kLog2e = 1.4426950408889634f;
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
+    const int li = l % LH;
+    patch_new_token(tK, tV, slot0, new_slot, new_k, new_v);
+    float sv[PASSES];                                                // logits of my head, one row per pass
+    bool valid[PASSES];
+    logits(tK, slot0, L, scale, sv, valid);
+    park(sv, slot0, L, logit_dst, logit_stride, logit_off);
     // online softmax update of my head, one rescale per tile
     float corr;
     {
@@ -598,32 +651,8 @@ struct Scanner {
 #pragma unroll
         for (int j = 0; j < NB; ++j) { oc[j][0] *= ca; oc[j][1] *= cb; oc[j][2] *= ca; oc[j][3] *= cb; }
       }
-      if (slot0 + kTileSlots > L) {
-        // ragged tile: rows beyond L hold stale bytes, possibly NaN patterns, and 0 * NaN would reach the accumulators
-        for (int w = lane_id; w < 8 * (C::kRowBytes / 4); w += 32) {
-          const int r = w / (C::kRowBytes / 4);
-          if (slot0 + warp * 8 + r >= L) *v_word(tV, warp * 8 + r, w % (C::kRowBytes / 4)) = 0u;
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-      }
-      // B fragment: lane t = 4*n + q supplies rows 2q, 2q+1 of column n (n < 4: head n, high part; else head n-4, low
-      // part).  Row 2q is pass q of row group 0, row 2q+1 pass q of row group 1; head n % 4 is this lane's own head.
       const float mine = li == 0 ? sv[0] : (li == 1 ? sv[1] : (li == 2 ? sv[2] : sv[3]));
-      const float other = __shfl_xor_sync(0xffffffffu, mine, 16);
-      const bool up = lane_id >= 16;
-      const float pe = up ? other : mine, po = up ? mine : other;
-      const __nv_bfloat16 he = __float2bfloat16_rn(pe), ho = __float2bfloat16_rn(po);
-      const __nv_bfloat16 le = __float2bfloat16_rn(pe - __bfloat162float(he)), lo = __float2bfloat16_rn(po - __bfloat162float(ho));
-      const uint32_t b0 = up ? (bf16_bits(le) | (bf16_bits(lo) << 16)) : (bf16_bits(he) | (bf16_bits(ho) << 16));
-      // lanes 8i..8i+7 address rows 0..7 of the warp's share, 16-byte chunk 4*jj + i of the row (channels 32*jj + 8*i ...)
-#pragma unroll
-      for (int jj = 0; jj < NB / 2; ++jj) {
-        uint32_t af[4];
-        ldmatrix_x4_trans(af, v_word(tV, warp * 8 + (lane_id & 7), (4 * jj + (lane_id >> 3)) * 4));
-        mma_m16n8k8_bf16(oc[2 * jj], af[0], af[1], b0);
-        mma_m16n8k8_bf16(oc[2 * jj + 1], af[2], af[3], b0);
-      }
+      pv_mma(tV, mine, slot0, L);
     } else {
     // the running maxima settle after a few tiles: rescale the output accumulators only when some head's maximum moved
     if (__any_sync(0xffffffffu, corr != 1.0f)) {
@@ -658,6 +687,44 @@ struct Scanner {
       }
     }
     }  // !MMA
+  }
+
+  // Two-phase scan (MMA configurations): the value phase starts from zero accumulators and ends with the warp's partial
+  // (m = the unit's maximum of the head, l = sum of the warp's probabilities, o[D]) in shared memory.  l_mine is the sum
+  // over the tiles of this thread's own (row, head) probabilities.
+  __device__ __forceinline__ void begin_pv() {
+#pragma unroll
+    for (int j = 0; j < NB; ++j) oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.f;
+  }
+  __device__ __forceinline__ void end_pv(float* warp_part, float m_unit, float l_mine) {
+    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+    const int rg = lane_id / LPR, l = lane_id % LPR;
+    const int my_head = l / LH, li = l % LH;
+    // the head's eight rows of every tile: four threads (li) in each of the two row groups
+    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 1);
+    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 2);
+    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 16);
+    const int c = lane_id >> 2, q = lane_id & 3;
+#pragma unroll
+    for (int j = 0; j < NB; ++j)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) oc[j][i] += __shfl_xor_sync(0xffffffffu, oc[j][i], 2);   // high-part + low-part columns
+    if (q < 2) {
+      float* wa = warp_part + (warp * G + 2 * q) * (D + 2) + 2;
+      float* wb = wa + (D + 2);
+#pragma unroll
+      for (int j = 0; j < NB; ++j) {
+        wa[16 * j + c] = oc[j][0];
+        wb[16 * j + c] = oc[j][1];
+        wa[16 * j + 8 + c] = oc[j][2];
+        wb[16 * j + 8 + c] = oc[j][3];
+      }
+    }
+    if (rg == 0 && li == 0) {
+      float* wp = warp_part + (warp * G + my_head) * (D + 2);
+      wp[0] = m_unit;
+      wp[1] = l_mine;
+    }
   }
 
   // Fold the warp's row groups and leave the warp's partial (m, l, o[D]) per query head in shared memory.
@@ -815,6 +882,33 @@ __device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsign
   if constexpr (kRelease) group_sync<NT>();
 }
 
+// One slot's share of a step: p = e / Z per query head (written to the optional probability output), the group mean
+// folded into the slot's accumulated score (Algorithm 1: a = [a,0] + A_t), abar = a / n and the pick key.
+template <typename T, int G>
+__device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>& v, float* a_l, int32_t* pos_l, int slot,
+                                         const float (&e)[G], const float* Z, float a_old, int pos_i, bool compress,
+                                         unsigned long long& best, int& best_slot) {
+  float pg[G];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    pg[g] = __fdiv_rn(e[g], Z[g]);
+    if (P.probs)
+      P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + slot] = pg[g];
+  }
+  float pbar = pg[0];
+#pragma unroll
+  for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pg[g]);
+  if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
+  const float a_new = __fadd_rn(a_old, pbar);
+  a_l[slot] = a_new;
+  if (slot == v.new_slot) pos_l[slot] = v.t;
+  if (compress && pos_i >= P.sink && pos_i <= v.t - P.window) {
+    const float abar = __fdiv_rn(a_new, __int2float_rn(v.t - pos_i + 1));
+    const unsigned long long key = ((unsigned long long)__float_as_uint(abar) << 32) | (uint32_t)pos_i;
+    if (key < best) { best = key; best_slot = slot; }
+  }
+}
+
 // A_t over a range of slots, a = [a,0] + A_t, abar = a/n and the range's pick key (Algorithm 1).
 // e values at lg[g*stride + i] for slot slot0 + i.  Updates the thread's best (key, slot).
 template <typename T, int G, int NT>
@@ -826,7 +920,7 @@ __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<
   const int t = v.t;
   constexpr int U = 4;                          // a, pos and e of U slots are loaded before any of them is used
   for (int i0 = threadIdx.x; i0 < n; i0 += NT * U) {
-    float a_old[U], ev[G][U];
+    float a_old[U], ev[U][G];
     int pos_v[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
@@ -836,51 +930,40 @@ __device__ __forceinline__ void fold_scores(const StepParams& P, const LaneView<
       a_old[u] = (ok && !is_new) ? a_l[slot] : 0.f;
       pos_v[u] = (ok && !is_new) ? pos_l[slot] : t;
 #pragma unroll
-      for (int g = 0; g < G; ++g) ev[g][u] = ok ? lg[(long long)g * stride + i] : 0.f;
+      for (int g = 0; g < G; ++g) ev[u][g] = ok ? lg[(long long)g * stride + i] : 0.f;
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int i = i0 + u * NT;
       if (i >= n) continue;
-      const int slot = slot0 + i;
-      float pg[G];
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        pg[g] = __fdiv_rn(ev[g][u], Z[g]);
-        if (P.probs)
-          P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + slot] = pg[g];
-      }
-      float pbar = pg[0];
-#pragma unroll
-      for (int g = 1; g < G; ++g) pbar = __fadd_rn(pbar, pg[g]);
-      if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
-      const float a_new = __fadd_rn(a_old[u], pbar);
-      const int pos_i = pos_v[u];
-      a_l[slot] = a_new;
-      if (slot == v.new_slot) pos_l[slot] = t;
-      if (compress && pos_i >= P.sink && pos_i <= t - P.window) {
-        const float abar = __fdiv_rn(a_new, __int2float_rn(t - pos_i + 1));
-        const unsigned long long key = ((unsigned long long)__float_as_uint(abar) << 32) | (uint32_t)pos_i;
-        if (key < best) { best = key; best_slot = slot; }
-      }
+      fold_one<T, G>(P, v, a_l, pos_l, slot0 + i, ev[u], Z, a_old[u], pos_v[u], compress, best, best_slot);
     }
   }
 }
 
-// Group-wide minimum of the pick key; returns it in every thread and leaves the owning slot in *slot_out (shared).
+// Group-wide minimum of the pick key and the slot that owns it, in every thread (slot_out: -1 when no slot is
+// evictable).  scratch: NT/32 keys followed by NT/32 slot words (as 64-bit entries); one barrier, after which the
+// caller must not write the scratch before a barrier of its own.
 template <int NT>
 __device__ __forceinline__ unsigned long long group_min_key(unsigned long long best, int best_slot, unsigned long long* scratch,
-                                                            int* slot_out) {
-  const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
+                                                            int& slot_out) {
+  constexpr int NW = NT / 32;
+  const int warp = threadIdx.x >> 5;
   const unsigned long long wmin = warp_min_u64(best);
-  if (lane_id == 0) scratch[warp] = wmin;
-  if (threadIdx.x == 0) *slot_out = -1;
+  // positions are unique, so a key below ~0 has exactly one owner in the warp; ~0 means "no candidate" in every lane
+  if (best == wmin && (best_slot >= 0 || (threadIdx.x & 31) == 0)) {
+    scratch[warp] = wmin;
+    scratch[NW + warp] = (unsigned long long)(long long)best_slot;
+  }
   group_sync<NT>();
   unsigned long long bmin = scratch[0];
+  int bslot = (int)(long long)scratch[NW];
 #pragma unroll
-  for (int w = 1; w < NT / 32; ++w) bmin = scratch[w] < bmin ? scratch[w] : bmin;
-  if (best == bmin && best_slot >= 0) *slot_out = best_slot;       // positions are unique: one owner
-  group_sync<NT>();
+  for (int w = 1; w < NW; ++w) {
+    const unsigned long long k = scratch[w];
+    if (k < bmin) { bmin = k; bslot = (int)(long long)scratch[NW + w]; }
+  }
+  slot_out = bslot;
   return bmin;
 }
 
@@ -961,13 +1044,12 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
   }
 }
 
-// The whole epilogue of a lane from global scratch (all partials and logits of the lane are visible to the caller).
+// Steps (1) and (2) of a lane's epilogue from global scratch: the split weights, the global maximum and normaliser of
+// every query head (left in ep.M / ep.linv / ep.w behind a barrier), and o_t.
 template <typename T, int D, int G, int NT>
-__device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
+__device__ __forceinline__ void combine_partials(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
   const float kLog2e = 1.4426950408889634f;
   const int tid = threadIdx.x;
-  const int L = v.L;
-  float* lg = P.logits + (long long)v.lane_local * G * P.cap;
   const float* part = P.part + (long long)v.lane_local * P.n_splits * G * (D + 2);
   // (1) split weights and the global max / normaliser of every query head
   // (warp g takes head g, a lane takes splits lane and lane + 32: one round of loads instead of a serial loop)
@@ -1005,6 +1087,25 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
       out[idx] = from_f32<T>(o * ep.linv[g]);
     }
   }
+}
+
+// Zeroes of the optional probability output beyond the lane's entries.
+template <int G, int NT>
+__device__ __forceinline__ void clear_probs_tail(const StepParams& P, int b, int hk, int L) {
+  if (P.probs) {
+    for (int i = L + (int)threadIdx.x; i < P.budget + 1; i += NT)
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+        P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = 0.f;
+  }
+}
+
+// The whole epilogue of a lane from global scratch (all partials and logits of the lane are visible to the caller).
+template <typename T, int D, int G, int NT>
+__device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
+  const int L = v.L;
+  float* lg = P.logits + (long long)v.lane_local * G * P.cap;
+  combine_partials<T, D, G, NT>(P, v, ep);
   // (3) Z_g as an exact integer sum
   float Zr[G];
   {
@@ -1015,19 +1116,72 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
     for (int g = 0; g < G; ++g) Zr[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
   }
   // (4) probabilities, score fold, pick
-  const bool compress = L > P.budget;                 // "length of V_t exceeds m"
+  const bool compress = L > P.budget;                 // Algorithm 1's trigger: the list is longer than m
   unsigned long long best = ~0ull;
   int best_slot = -1;
   fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, Zr, compress, best, best_slot);
-  if (P.probs) {
-    for (int i = L + tid; i < P.budget + 1; i += NT)
-#pragma unroll
-      for (int g = 0; g < G; ++g)
-        P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
-  }
-  const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, &ep.i32[1]);   // also publishes a, pos
+  clear_probs_tail<G, NT>(P, v.b, v.hk, L);
+  int j_slot;
+  const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
-  finish_lane<T, D, G, NT>(P, v, ep, compress, bmin, ep.i32[1]);
+  finish_lane<T, D, G, NT>(P, v, ep, compress, bmin, j_slot);
+}
+
+// The same epilogue for a lane of at most E * NT entries, with what a thread needs close at hand: thread tid owns slots
+// tid, tid + NT, ...; their accumulated scores and positions are in shared memory (a_s, pos_s: staged by the caller
+// before the lane's scan was even finished -- the scan writes neither; a thread reads back only what it staged itself)
+// and their parked logits are requested here in one go and stay in registers, so the lane pays one round trip to L2
+// where the loop version pays one per few slots and phase.  Same arithmetic, same results.
+template <typename T, int D, int G, int NT, int E>
+__device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, const LaneView<T>& v, const EpScratch& ep,
+                                                           const float* a_s, const int* pos_s) {
+  const int tid = threadIdx.x, L = v.L;
+  const float* lg = P.logits + (long long)v.lane_local * G * P.cap;
+  float sx[E][G];
+#pragma unroll
+  for (int u = 0; u < E; ++u) {
+    const int i = tid + u * NT;
+#pragma unroll
+    for (int g = 0; g < G; ++g) sx[u][g] = i < L ? __ldcg(lg + (long long)g * P.cap + i) : -INFINITY;
+  }
+  combine_partials<T, D, G, NT>(P, v, ep);
+  // (3) e = exp(s - M) in place, Z_g as an exact integer sum
+  float Zr[G];
+  {
+    unsigned long long zl[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) zl[g] = 0ull;
+#pragma unroll
+    for (int u = 0; u < E; ++u) {
+      if (tid + u * NT < L) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          const float e = repro_exp(__fsub_rn(sx[u][g], ep.M[g]));
+          sx[u][g] = e;
+          zl[g] += __float2ull_rz(__fmul_rn(e, 1099511627776.0f));
+        }
+      }
+    }
+    group_sum_u64<G, NT, false>(zl, ep.u64);
+#pragma unroll
+    for (int g = 0; g < G; ++g) Zr[g] = __fmul_rn(__ull2float_rn(zl[g]), 1.0f / 1099511627776.0f);
+  }
+  // (4) probabilities, score fold, pick
+  const bool compress = L > P.budget;                 // Algorithm 1's trigger: the list is longer than m
+  unsigned long long best = ~0ull;
+  int best_slot = -1;
+  float* a_l = P.a + v.lane * P.cap;
+  int32_t* pos_l = P.pos + v.lane * P.cap;
+#pragma unroll
+  for (int u = 0; u < E; ++u) {
+    const int i = tid + u * NT;
+    if (i < L) fold_one<T, G>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot);
+  }
+  clear_probs_tail<G, NT>(P, v.b, v.hk, L);
+  int j_slot;
+  const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
+  // (5), (6)
+  finish_lane<T, D, G, NT>(P, v, ep, compress, bmin, j_slot);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1052,8 +1206,9 @@ __device__ __forceinline__ void scan_body(const StepParams& P) {
   //      state and put the first K/V tiles in flight, then wait before the first read of a caller input.
   //   0  the caller has handed over all layers of a step at once (wkv_decode_step_layers): the predecessor is the lane
   //      epilogue of the previous layer (other lanes, other scratch set); scan alongside it and wait only at the very
-  //      end, so that the completion of this grid still implies the completion of everything before it and later
-  //      kernels need not reason about more than one predecessor.
+  //      end, before the unit reports to its lane's epilogue, so that the completion of this grid -- and any report of
+  //      it -- still implies the completion of everything before it and later kernels need not reason about more than
+  //      one predecessor.
   if (P.wait_at_start == 2) griddep_wait();
   griddep_launch();
   if (P.wait_at_start == 1 && P.seq_lens != nullptr) griddep_wait();     // seq_lens is a caller input
@@ -1129,6 +1284,11 @@ __device__ __forceinline__ void scan_body(const StepParams& P) {
   }
   __syncthreads();
   combine_warps<D, G, NT>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
+  // Level 0: the wait comes BEFORE the unit reports.  The lane epilogues behind this scan start on the reports alone,
+  // and the scan after them (which reuses the scratch set of the lane epilogues in front of this scan) is released by
+  // those epilogues: with the report behind the wait, "the next scan runs" implies "every unit here has seen the
+  // previous lane epilogues complete", so no two grids ever touch one scratch set at a time.
+  if (!P.wait_at_start) griddep_wait();
   if (P.ticket != nullptr) {
     // tell the lane's epilogue CTA (already resident in the next kernel, or not yet) that this unit is in scratch
     __syncthreads();
@@ -1137,18 +1297,199 @@ __device__ __forceinline__ void scan_body(const StepParams& P) {
       atomicAdd(&P.ticket[lane_local], 1u);
     }
   }
-  if (!P.wait_at_start) griddep_wait();
+}
+
+// ------------------------------------------------------------------------------------------------
+// The scan for four query heads on bf16 rows (Cfg::kMmaPV) in two phases per unit: first every K tile of the unit
+// (logits, parked as always, and the unit's exact maximum per head), then every V tile (probabilities against that
+// maximum, P.V on the tensor cores).  With four heads per cache row the scan is bound by instruction issue, not by
+// bandwidth, and the single-pass form needs the four query rows AND the output accumulators in registers at once
+// (96 per thread, four CTAs per SM).  Apart, each phase fits 64 registers, so six CTAs share an SM, and the online
+// softmax with its per-tile rescaling disappears.  A thread re-reads in phase two exactly the one logit per tile that
+// it parked itself in phase one.  The ring holds single tiles (K or V), twice as many stages in the same bytes; the
+// warp partials are written over the ring once every warp is done with it.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+struct TwoPhase {
+  using C = Cfg<T, D, G>;
+  static constexpr int kStages = WKV_RING_BYTES / C::kTileBytes;
+  static constexpr int kRingBytes = kStages * C::kTileBytes;
+  static_assert(kStages >= 2 && C::kVHalves * C::kVHalfBytes == C::kTileBytes, "a stage holds one tile of either kind");
+  static_assert(C::kWarpPartFloats * 4 <= kRingBytes, "the warp partials reuse the ring");
+  // ring | new token rows | mbarriers | per-warp maxima
+  static constexpr int kSmemBytes = kRingBytes + C::kAuxBytes + 2 * kStages * 8 + kConsumerWarps * G * 4 + 64;
+};
+
+template <typename T, int D, int G>
+__device__ __forceinline__ void scan_body_two_phase(const StepParams& P) {
+  using C = Cfg<T, D, G>;
+  using TP = TwoPhase<T, D, G>;
+  using SC = Scanner<T, D, G>;
+  static_assert(C::kMmaPV && SC::PASSES == 4 && SC::LH == 4 && SC::RPP == 2, "16 threads per row, one logit per thread and tile");
+  constexpr int NS = TP::kStages;
+  constexpr int NT = kThreads;
+  const float kLog2e = 1.4426950408889634f;
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* ring = smem_raw;
+  T* aux = reinterpret_cast<T*>(ring + TP::kRingBytes);                       // [ k: D | v: D ] this step's token
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + TP::kRingBytes + C::kAuxBytes);
+  uint64_t* empty_bar = full_bar + NS;
+  float* wmax = reinterpret_cast<float*>(empty_bar + NS);                     // [warp][G] maxima of phase one
+  float* warp_part = reinterpret_cast<float*>(ring);                          // [warp][G][D+2], after the scan
+  const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
+  const int split = blockIdx.x % P.n_splits;
+  const int lane_local = blockIdx.x / P.n_splits;
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  // ordering against the preceding kernel: as in scan_body
+  if (P.wait_at_start == 2) griddep_wait();
+  griddep_launch();
+  if (P.wait_at_start == 1 && P.seq_lens != nullptr) griddep_wait();
+  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {
+    if (P.wait_at_start != 2) griddep_wait();
+    return;
+  }
+  LaneView<T> v;
+  {
+    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+    fill_view<T, D>(v, P, lane_local, split, st[LS_LEN], st[LS_T], st[LS_FREE]);
+  }
+  v.new_k = aux;
+  v.new_v = aux + D;
+  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
+  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+  if (tid == 32 && v.slot_end > v.slot_begin) {
+    const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);
+    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
+    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
+  }
+  const int n = v.n_tiles;
+  // item x of the unit's stream: K tile x for x < n, then V tile x - n
+  auto issue = [&](int x) {
+    const int s = x % NS;
+    unsigned char* dst = ring + (size_t)s * C::kTileBytes;
+    const int slot0 = (v.tile_begin + (x < n ? x : x - n)) * kTileSlots;
+    if (x < n) {
+      const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
+      mbar_expect_tx(&full_bar[s], bytes);
+      bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &full_bar[s]);
+    } else {
+      // whole 32-row boxes: rows past the lane's entries are other slots' bytes (zero fill past the end of the cache)
+      mbar_expect_tx(&full_bar[s], (uint32_t)C::kTileBytes);
+#pragma unroll
+      for (int h = 0; h < C::kVHalves; ++h)
+        tensor_g2s_2d(dst + h * C::kVHalfBytes, P.vmap, h * 64, (int)(v.lane * P.cap) + slot0, &full_bar[s]);
+    }
+  };
+  if (tid == kConsumerWarps * 32) {
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], kConsumerWarps);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int x = 0; x < min(2 * n, NS); ++x) issue(x);
+  }
+  if (P.wait_at_start == 1) griddep_wait();
+  for (int c = tid; c < D; c += NT) {
+    aux[c] = k_in[c];
+    aux[D + c] = v_in[c];
+  }
+  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
+    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
+    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
+    for (int c = tid; c < D; c += NT) { Kw[c] = k_in[c]; Vw[c] = v_in[c]; }
+  }
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    if (lane_id == 0) {                                   // producer: keeps the ring full
+      for (int x = NS; x < 2 * n; ++x) {
+        mbar_wait(&empty_bar[x % NS], ((x / NS) - 1) & 1, P.status);
+        issue(x);
+      }
+    }
+  } else {
+    const int rg = lane_id / SC::LPR, l = lane_id % SC::LPR;
+    const int my_head = l / SC::LH, li = l % SC::LH;
+    float* lg = P.logits + (long long)lane_local * G * P.cap;
+    // the one (row, head) of every tile whose logit this thread parks in phase one and turns into a probability in two
+    const int my_row = warp * 8 + li * SC::RPP + rg;
+    float* my_lg = lg + (long long)my_head * P.cap;
+    float m_unit;
+    {
+      // ---- phase one: logits of the unit, exact maximum per head ----
+      SC sc;
+      sc.begin(q_in);
+      float m_run = -INFINITY;
+      for (int i = 0; i < n; ++i) {
+        const int s = i % NS;
+        mbar_wait(&full_bar[s], (i / NS) & 1, P.status);
+        T* tK = reinterpret_cast<T*>(ring + (size_t)s * C::kTileBytes);
+        const int slot0 = (v.tile_begin + i) * kTileSlots;
+        SC::patch_new_token(tK, nullptr, slot0, v.new_slot, v.new_k, v.new_v);
+        float sv[SC::PASSES];
+        bool valid[SC::PASSES];
+        sc.logits(tK, slot0, v.L, P.scale, sv, valid);
+        SC::park(sv, slot0, v.L, lg, P.cap, 0);
+#pragma unroll
+        for (int ps = 0; ps < SC::PASSES; ++ps) m_run = fmaxf(m_run, sv[ps]);
+        release_stage(&empty_bar[s]);
+      }
+      m_run = fmaxf(m_run, __shfl_xor_sync(0xffffffffu, m_run, 16));          // the other row group, same head
+      if (rg == 0 && li == 0) wmax[warp * G + my_head] = m_run;
+      group_sync<kConsumerWarps * 32>();
+      m_unit = wmax[my_head];
+#pragma unroll
+      for (int w = 1; w < kConsumerWarps; ++w) m_unit = fmaxf(m_unit, wmax[w * G + my_head]);
+    }
+    // ---- phase two: probabilities against the unit's maximum, P.V ----
+    SC sc;
+    sc.begin_pv();
+    const float m_use = m_unit == -INFINITY ? 0.f : m_unit;
+    float l_mine = 0.f;
+    float s_next = 0.f;
+    {
+      const int slot = v.tile_begin * kTileSlots + my_row;
+      if (n > 0 && slot < v.L) s_next = my_lg[slot];
+    }
+    for (int i = 0; i < n; ++i) {
+      const int x = n + i, s = x % NS;
+      const int slot0 = (v.tile_begin + i) * kTileSlots;
+      const float s_mine = s_next;
+      const bool ok = slot0 + my_row < v.L;
+      if (i + 1 < n && slot0 + kTileSlots + my_row < v.L) s_next = my_lg[slot0 + kTileSlots + my_row];   // next tile's, early
+      const float p = ok ? fast_exp2((s_mine - m_use) * kLog2e) : 0.f;
+      l_mine += p;
+      mbar_wait(&full_bar[s], (x / NS) & 1, P.status);
+      T* tV = reinterpret_cast<T*>(ring + (size_t)s * C::kTileBytes);
+      SC::patch_new_token(nullptr, tV, slot0, v.new_slot, v.new_k, v.new_v);
+      sc.pv_mma(tV, p, slot0, v.L);
+      release_stage(&empty_bar[s]);
+    }
+    // every warp is done with the ring before the partials go over it
+    group_sync<kConsumerWarps * 32>();
+    sc.end_pv(warp_part, m_unit, l_mine);
+  }
+  __syncthreads();
+  combine_warps<D, G, NT>(warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
+  if (!P.wait_at_start) griddep_wait();                   // level 0: wait before reporting (see scan_body)
+  if (P.ticket != nullptr) {
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      atomicAdd(&P.ticket[lane_local], 1u);
+    }
+  }
 }
 
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kThreads) scan_kernel(const __grid_constant__ StepParams P) {
   scan_body<T, D, G>(P);
 }
-// The same scan for the instantiations with the tensor-core P.V half (Cfg::kMmaPV), held to the registers of four CTAs
-// per SM (a second argument to __launch_bounds__ changes the compiler's choices even when it is 1, hence two entries).
+// The scan of the instantiations with the tensor-core P.V half (Cfg::kMmaPV): two phases, six CTAs per SM.
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads, 4) scan_kernel_mma(const __grid_constant__ StepParams P) {
-  scan_body<T, D, G>(P);
+__global__ void __launch_bounds__(kThreads, 6) scan_kernel_mma(const __grid_constant__ StepParams P) {
+  scan_body_two_phase<T, D, G>(P);
 }
 // the entry that a configuration's scan is launched through
 template <typename T, int D, int G>
@@ -1156,9 +1497,21 @@ inline auto scan_entry() -> void (*)(const StepParams) {
   if constexpr (Cfg<T, D, G>::kMmaPV) return scan_kernel_mma<T, D, G>;
   else return scan_kernel<T, D, G>;
 }
+// dynamic shared memory of that entry
+template <typename T, int D, int G>
+constexpr int scan_smem_bytes() {
+  if constexpr (Cfg<T, D, G>::kMmaPV) return TwoPhase<T, D, G>::kSmemBytes;
+  else return Cfg<T, D, G>::kFixedBytes;
+}
 
 constexpr int kEpilogueThreads = 256;
 constexpr int kEpilogueThreadsWide = 512;     // one or two query heads only (registers: two CTAs per SM)
+// Slots per thread that the register version of the lane epilogue is compiled for (0: not compiled); a thread keeps
+// E * G logits in registers.  17 x 256 and 9 x 512 threads cover the 4097 entries of the largest single-head workload,
+// 9 x 384 the 3278 entries of the grouped-query one.
+__host__ __device__ constexpr int epilogue_slots_per_thread(int G, int NT) {
+  return G == 1 ? (NT >= 512 ? 9 : 17) : G == 2 ? (NT >= 512 ? 5 : 9) : (G == 4 && NT >= 384) ? 9 : 0;
+}
 
 // NT threads per lane: kEpilogueThreads, or kEpilogueThreadsWide when a layer has so few lanes that two wide CTAs per
 // SM still hold them all -- the epilogue is a chain of load -> compute rounds, and twice the threads halve the rounds.
@@ -1180,6 +1533,24 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
     v.tail = st[LS_TAIL];
     v.new_k = v.Kl + (long long)v.new_slot * D;          // the scan kernel has stored this step's token in the cache
     v.new_v = v.Vl + (long long)v.new_slot * D;
+  }
+  // A lane of at most E * NT entries is finished by lane_epilogue_in_registers, if the launch gave the CTA room to stage
+  // the lane's scores and positions (P.ep_stage_slots entries each of dynamic shared memory).  They were last written
+  // where its state words were, so they too can be fetched before waiting; the entry of this step's token starts from
+  // a = 0 (Algorithm 1's [a, 0]) at position t.
+  constexpr int E = epilogue_slots_per_thread(G, NT);
+  extern __shared__ __align__(16) unsigned char ep_dyn[];
+  float* a_s = reinterpret_cast<float*>(ep_dyn);
+  int* pos_s = reinterpret_cast<int*>(ep_dyn) + P.ep_stage_slots;
+  const bool in_regs = E > 0 && active && v.L <= E * NT && v.L <= P.ep_stage_slots;
+  if (in_regs) {
+    const float* a_l = P.a + v.lane * P.cap;
+    const int32_t* pos_l = P.pos + v.lane * P.cap;
+    for (int i = threadIdx.x; i < v.L; i += NT) {
+      const bool old_entry = i != v.new_slot;
+      a_s[i] = old_entry ? __ldcg(a_l + i) : 0.f;
+      pos_s[i] = old_entry ? __ldcg(pos_l + i) : v.t;
+    }
   }
   // When is the lane's scan in scratch?  Without tickets: when the whole scan kernel has completed.  With tickets: as
   // soon as the lane's own n_splits units have reported -- this kernel's CTAs become resident only after every CTA of
@@ -1211,7 +1582,11 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
       return;
     }
   }
-  lane_epilogue_from_scratch<T, D, G, NT>(P, v, ep);
+  if (in_regs) {
+    if constexpr (E > 0) lane_epilogue_in_registers<T, D, G, NT, E>(P, v, ep, a_s, pos_s);
+  } else {
+    lane_epilogue_from_scratch<T, D, G, NT>(P, v, ep);
+  }
   if (P.ticket != nullptr) {
     if (threadIdx.x == 0) P.ticket[lane_local] = 0u;     // ready for the next call that uses this scratch set
     griddep_wait();                                      // keeps "this grid complete => the scan complete" literally true
@@ -1360,13 +1735,13 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const __g
     group_sum_u64<G, NT>(zl, sm.ep.u64);
     if (tid == 0) {
 #pragma unroll
-      for (int g = 0; g < G; ++g) sm.ep.u64[80 + g] = zl[g];
+      for (int g = 0; g < G; ++g) sm.ep.u64[96 + g] = zl[g];
     }
   }
   cluster.sync();                                       // #2: Z partials readable (and rank 0 is done with the o partials)
   if (tid < G) {
     unsigned long long z = 0ull;
-    for (int s = 0; s < S; ++s) z += cluster.map_shared_rank(sm.ep.u64, s)[80 + tid];
+    for (int s = 0; s < S; ++s) z += cluster.map_shared_rank(sm.ep.u64, s)[96 + tid];
     sm.ep.Z[tid] = __fmul_rn(__ull2float_rn(z), 1.0f / 1099511627776.0f);
   }
   __syncthreads();
@@ -1381,23 +1756,24 @@ __global__ void __launch_bounds__(kThreads) decode_step_cluster_kernel(const __g
       for (int g = 0; g < G; ++g)
         P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + i] = 0.f;
   }
-  const unsigned long long my_min = group_min_key<NT>(best, best_slot, sm.ep.u64 + 64, &sm.ep.i32[1]);
-  if (tid == 0) sm.ep.u64[88] = my_min;
+  int my_slot;
+  const unsigned long long my_min = group_min_key<NT>(best, best_slot, sm.ep.u64 + 64, my_slot);
+  if (tid == 0) { sm.ep.u64[104] = my_min; sm.ep.i32[1] = my_slot; }
   cluster.sync();                                       // #3: keys readable; a and pos of every slot are written
   // (5) rank 0 gathers the lane's pick
   if (split == 0 && tid == 0) {
     unsigned long long bmin = ~0ull;
     int j = -1;
     for (int s = 0; s < S; ++s) {
-      const unsigned long long k = cluster.map_shared_rank(sm.ep.u64, s)[88];
+      const unsigned long long k = cluster.map_shared_rank(sm.ep.u64, s)[104];
       if (k < bmin) { bmin = k; j = cluster.map_shared_rank(sm.ep.i32, s)[1]; }
     }
     sm.ep.i32[4] = j;
-    sm.ep.u64[89] = bmin;
+    sm.ep.u64[105] = bmin;
   }
   cluster.sync();                                       // #4: nobody's shared memory is needed any more
   if (split != 0) return;
-  finish_lane<T, D, G, NT>(P, v, sm.ep, compress, sm.ep.u64[89], sm.ep.i32[4]);
+  finish_lane<T, D, G, NT>(P, v, sm.ep, compress, sm.ep.u64[105], sm.ep.i32[4]);
 }
 
 // Exercises the give-up path of the bounded wait without any fault: one thread waits on an mbarrier that nothing

@@ -67,14 +67,16 @@ class Parity:
         self.probs = torch.empty(L, B, Hq, wl.budget + 1, device=self.dev) if check_probs else None
 
     # ---- oracle side of one token --------------------------------------------------------------
-    def _oracle_token(self, q, k, v, active, out_gpu, ev_gpu, what, probs_gpu=None):
-        """q [n, G, d], k, v [n, d], out_gpu [n, G, d], ev_gpu [n] already gathered for the sampled lanes (CPU)."""
+    def _oracle_token(self, q, k, v, active, out_gpu, ev_gpu, what, probs_gpu=None, check_out=True):
+        """q [n, G, d], k, v [n, d], out_gpu [n, G, d], ev_gpu [n] already gathered for the sampled lanes (CPU).
+        check_out = False: the removed positions are compared, the attention output is not (and the oracle is not asked
+        for it, which spares it the fp64 pass over the cache)."""
         o_ref, ev_ref, p_ref = self.ref.step(q.float().numpy(), k.float().numpy(), v.float().numpy(), active=active,
-                                             want_probs=probs_gpu is not None)
+                                             want_out=check_out, want_probs=probs_gpu is not None)
         act = np.ones(len(self.lanes), bool) if active is None else np.asarray(active, bool)
         np.testing.assert_array_equal(ev_gpu.numpy()[act], ev_ref[act], err_msg=f"{what}: eviction positions")
         self.n_evictions += int((ev_ref[act] >= 0).sum())
-        if act.any():
+        if act.any() and check_out:
             assert_close(out_gpu.float().numpy()[act], o_ref[act], self.wl.dtype, f"{what}: attention output")
         return p_ref
 
@@ -84,14 +86,18 @@ class Parity:
         return qs.cpu(), k[self.li, self.bi, self.hi].cpu(), v[self.li, self.bi, self.hi].cpu()
 
     # ---- prefill through wkv_prefill, chunked ------------------------------------------------------
-    def prefill(self, n_tokens, chunk=32, compare=True, bulk=False, all_layers=False):
+    def prefill(self, n_tokens, chunk=32, compare=True, bulk=False, all_layers=False, out_every=1):
+        """out_every = k > 1: the attention output is compared on every k-th prompt token only (and on the last token);
+        removed positions are compared on every token either way, and the state afterwards by compare_state."""
         wl = self.wl
         lens_dev = self.lens.to(self.dev)
         t_end = self.t + n_tokens
-        while self.t < t_end:
-            tc = min(chunk, t_end - self.t)
-            Q, K, V = self.stream.tokens(self.t, tc)                      # [L, B, tc, H, d]
-            rel = (lens_dev - self.t).clamp(min=0, max=tc).to(torch.int32)
+
+        def launch(t0):
+            """Issues one chunk on the GPU (asynchronous) and returns what the comparison needs, still on the device."""
+            tc = min(chunk, t_end - t0)
+            Q, K, V = self.stream.tokens(t0, tc)                          # [L, B, tc, H, d]
+            rel = (lens_dev - t0).clamp(min=0, max=tc).to(torch.int32)
             out = torch.empty(wl.n_layers, wl.batch, tc, wl.n_q_heads, wl.head_dim, dtype=wl.torch_dtype, device=self.dev)
             ev = torch.empty(wl.n_layers, wl.batch, tc, wl.n_kv_heads, dtype=torch.int32, device=self.dev)
             if all_layers:
@@ -99,16 +105,25 @@ class Parity:
             for layer in range(0 if all_layers else wl.n_layers):
                 (self.ctx.wkv_prefill_bulk if bulk else self.ctx.wkv_prefill)(layer, Q[layer], K[layer], V[layer], rel,
                                                                               out[layer], ev[layer])
-            Qs = Q.view(wl.n_layers, wl.batch, tc, wl.n_kv_heads, wl.group, wl.head_dim)[self.li, self.bi, :, self.hi].cpu()
-            Ks, Vs = K[self.li, self.bi, :, self.hi].cpu(), V[self.li, self.bi, :, self.hi].cpu()
-            Os = out.view(wl.n_layers, wl.batch, tc, wl.n_kv_heads, wl.group, wl.head_dim)[self.li, self.bi, :, self.hi].cpu()
-            Es = ev[self.li, self.bi, :, self.hi].cpu()
+            Qs = Q.view(wl.n_layers, wl.batch, tc, wl.n_kv_heads, wl.group, wl.head_dim)[self.li, self.bi, :, self.hi]
+            Ks, Vs = K[self.li, self.bi, :, self.hi], V[self.li, self.bi, :, self.hi]
+            Os = out.view(wl.n_layers, wl.batch, tc, wl.n_kv_heads, wl.group, wl.head_dim)[self.li, self.bi, :, self.hi]
+            Es = ev[self.li, self.bi, :, self.hi]
+            return t0, tc, (Qs, Ks, Vs, Os, Es), (Q, K, V, rel, out, ev)     # the last tuple keeps the kernels' buffers alive
+
+        # the GPU works on chunk c + 1 while the oracle checks chunk c
+        pending = launch(self.t) if self.t < t_end else None
+        while pending is not None:
+            t0, tc, dev_parts, _keep = pending
+            Qs, Ks, Vs, Os, Es = (x.cpu() for x in dev_parts)             # waits for chunk c
+            pending = launch(t0 + tc) if t0 + tc < t_end else None
             lens_s = self.lens[self.bi.cpu()].numpy()
             for i in range(tc):
-                active = (self.t + i) < lens_s
+                tok = t0 + i
+                active = tok < lens_s
                 self._oracle_token(Qs[:, i], Ks[:, i], Vs[:, i], active.astype(np.uint8), Os[:, i], Es[:, i],
-                                   f"prefill token {self.t + i}")
-            self.t += tc
+                                   f"prefill token {tok}", check_out=out_every <= 1 or tok % out_every == 0 or tok == t_end - 1)
+            self.t = t0 + tc
 
     # ---- decode through wkv_decode_step --------------------------------------------------------------
     def decode(self, n_steps, host_entry=False, layers_entry=False):

@@ -1,9 +1,8 @@
 """Parity at the full shapes of the large workloads (all layers, full batch, full budget) in the launch
-configuration bench.py times, on sampled lanes the oracle computes one by one.  The streamed prompt is shortened
-to budget + 160 tokens: every cache is then full and has compressed 160 times, which is the state the decode phase
-runs in."""
-import os
-
+configuration bench.py times, on sampled lanes the oracle computes one by one.  Two kinds of test: the configurations'
+stated decode lengths (2048 / 512 / 512 steps) behind a prompt shortened to budget + 160 tokens -- every cache is then
+full and has compressed 160 times, which is the state the decode phase runs in -- and the configurations' stated
+prompt lengths (8192 / 16384 ragged / 32768 tokens) followed by a few decode steps."""
 import numpy as np
 import pytest
 import torch
@@ -15,8 +14,8 @@ from parity_util import Parity
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("name,n_sample,decode,schedule", [("llama7b_b8", 12, 256, 0), ("serving_b16", 12, 96, 0),
-                                                           ("gqa_b32", 10, 64, 0), ("llama7b_b8", 6, 8, 2)])
+@pytest.mark.parametrize("name,n_sample,decode,schedule", [("llama7b_b8", 12, 2048, 0), ("serving_b16", 12, 512, 0),
+                                                           ("gqa_b32", 10, 512, 0), ("llama7b_b8", 6, 8, 2)])
 def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     wl = WORKLOADS[name]
     n_prefill = wl.budget + 160
@@ -68,18 +67,19 @@ def test_llama7b_b8_full_prompt_length():
     torch.cuda.empty_cache()
 
 
-@pytest.mark.skipif(os.environ.get("WKV_LONG_TESTS") != "1", reason="several minutes each: set WKV_LONG_TESTS=1")
-@pytest.mark.parametrize("name,n_sample", [("serving_b16", 6), ("gqa_b32", 4)])
-def test_serving_and_gqa_full_prompt_lengths(name, n_sample):
+@pytest.mark.parametrize("name,n_sample,decode", [("serving_b16", 6, 16), ("gqa_b32", 4, 16)])
+def test_serving_and_gqa_full_prompt_lengths(name, n_sample, decode):
     """The two largest configurations with their whole prompts (16384 tokens with per-sequence lengths drawn from
     8192..16384, and 32768 tokens), in chunks of 256 tokens for all layers at once, then decode; sampled lanes against
-    the oracle.  Tens of thousands of compressions per lane."""
+    the oracle.  Tens of thousands of compressions per lane, every removed position compared; the attention output on
+    every 64th prompt token and on every decode step."""
     wl = WORKLOADS[name]
     p = Parity(wl, sample=n_sample)
     assert int(p.lens.max()) == wl.prefill and int(p.lens.min()) >= wl.prefill_min
-    p.prefill(wl.prefill, chunk=256, all_layers=True)
+    p.prefill(wl.prefill, chunk=256, all_layers=True, out_every=64)
     p.compare_state()
-    p.decode(8)
+    p.decode(decode)
     p.compare_state()
+    assert p.n_evictions >= sum(int(p.lens[b]) - wl.budget for _, b, _ in p.lanes)
     p.close()
     torch.cuda.empty_cache()

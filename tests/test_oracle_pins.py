@@ -642,6 +642,35 @@ def test_merging_loses_less_than_eviction_on_synthetic_streams(rho):
         assert e_merge < 0.97 * e_evict, (rho, m, e_merge, e_evict)
 
 
+@pytest.mark.parametrize("rho", [0.0, 0.5])
+def test_single_step_perturbation_of_the_three_ways_to_compress(rho):
+    """Ideal Merging section: the ideal merged value leaves the output of the step's query unchanged; its two-term
+    convex cut with instantaneous weights is the closest of the practical choices FOR THAT QUERY.  Algorithm 1 swaps the
+    instantaneous weights for historical averages: for the next query, which the instantaneous weights know nothing
+    about, the historical weights are the better of the two.  (Measured and recorded, not predicted by the section:
+    a single eviction perturbs a single output less than either merge; merging wins over many steps, see
+    test_merging_loses_less_than_eviction_on_synthetic_streams.)"""
+    from oracle.diagnostics import merge_perturbation
+    rng = np.random.default_rng(7)
+    T, n, d, r = 256, 6, 32, 8
+    basis = rng.standard_normal((n, d, r))
+    K = np.einsum("ndr,tnr->tnd", basis, rng.standard_normal((T, n, r))) / math.sqrt(r) + 0.05 * rng.standard_normal((T, n, d))
+    Q = rng.standard_normal((T, n, 1, d))
+    noise = rng.standard_normal((T, n, d))
+    V = np.zeros((T, n, d))
+    V[0] = noise[0]
+    for t in range(1, T):
+        V[t] = rho * V[t - 1] + math.sqrt(1 - rho * rho) * noise[t]
+    Q, K, V = (x.astype(np.float32) for x in (Q, K, V))
+    res = merge_perturbation(Q, K, V, 64, 8)
+    assert res["steps"] == n * (T - 64)
+    assert res["ideal_residual"] < 1e-12                                 # the identity, at every compressing step
+    now, nxt = res["now"], res["next"]
+    assert now["instant"] < 0.9 * now["algorithm1"] and now["instant"] < now["evict"]
+    assert nxt["algorithm1"] < nxt["instant"]
+    assert all(0.0 < v < 0.2 for v in list(now.values()) + list(nxt.values()))
+
+
 def test_imported_state_continues_like_the_streamed_one():
     """wkvo_import (set-up for the large-cache tests) must put a lane exactly where streaming left it."""
     rng = np.random.default_rng(0)
