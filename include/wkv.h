@@ -46,7 +46,10 @@ typedef enum {
 typedef enum {
   WKV_SCHEDULE_AUTO = 0,
   WKV_SCHEDULE_SPLIT = 1,  /* two launches: scan every unit, then one CTA per lane finishes it (any n_splits)    */
-  WKV_SCHEDULE_CLUSTER = 2 /* one launch: a lane's units form a thread-block cluster (n_splits in {1,2,4,8,16})  */
+  WKV_SCHEDULE_CLUSTER = 2,/* one launch: a lane's units form a thread-block cluster (n_splits in {1,2,4,8,16})  */
+  WKV_SCHEDULE_FLAT = 3    /* two launches as in SPLIT, but the scan's CTAs take equal runs of the 32-entry tiles of
+                              ALL lanes, across lane boundaries (n_splits = CTAs per lane on average, 0 = one wave
+                              that fills the GPU); same results                                                  */
 } wkv_schedule;
 
 /* Device memory provider.  alloc returns a device address aligned to at least 256 bytes, or NULL. */

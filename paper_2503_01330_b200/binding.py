@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwkv.so")
 
 WKV_F32, WKV_BF16 = 0, 1
-WKV_SCHEDULE_AUTO, WKV_SCHEDULE_SPLIT, WKV_SCHEDULE_CLUSTER = 0, 1, 2
+WKV_SCHEDULE_AUTO, WKV_SCHEDULE_SPLIT, WKV_SCHEDULE_CLUSTER, WKV_SCHEDULE_FLAT = 0, 1, 2, 3
 WKV_OK, WKV_ERR_INVALID, WKV_ERR_ALLOC, WKV_ERR_CUDA, WKV_ERR_STATE, WKV_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 ALLOC_FN = C.CFUNCTYPE(C.c_void_p, C.c_size_t, C.c_void_p)

@@ -15,6 +15,7 @@
 #include "../../include/wkv.h"
 #include "wkv_kernels.cuh"
 #include "wkv_prefill.cuh"
+#include "wkv_block.cuh"
 
 struct wkv_ctx {
   wkv_config cfg;
@@ -23,12 +24,13 @@ struct wkv_ctx {
   long long lanes_total = 0;
   int cap = 0;            // slots per lane
   int group = 1;
-  int n_splits = 1;
+  int n_splits = 1;       // units per lane; with the flat deal the most pieces a lane can have (stride of the partials)
+  int flat_chunk = 0;     // tiles per CTA under the flat deal of the two-kernel schedule, 0 = even deal
   int chunk_cap = 0;      // cluster kernel: logits per CTA and query head
   bool use_cluster = false;
   // all layers of a step in one launch (wkv_decode_step_layers), when the scratch for every lane at once is small
   bool fused_ok = false, fused_cluster = false;
-  int fused_splits = 1, fused_chunk_cap = 0;
+  int fused_splits = 1, fused_chunk_cap = 0, fused_flat_chunk = 0;
   float* fused_logits = nullptr;
   float* fused_part = nullptr;
   int sm_count = 148;
@@ -69,6 +71,15 @@ struct wkv_ctx {
   long long bulk_lanes = 0;     // lanes the scratch has rows for
   // per layer: an upper bound on the tokens any lane of the layer has consumed since creation / reset; while it is
   // below the budget no lane has compressed and token i of every lane sits in slot i (kCompressed: unknown / beyond)
+  // blocked prompt tail (wkv_block.cuh): scratch for `blk_lanes` lanes, taken on first use
+  float* blk_logits = nullptr;
+  float* blk_lgx = nullptr;
+  float* blk_ptab = nullptr;
+  float* blk_opart = nullptr;
+  float* blk_rec_rows = nullptr;
+  int32_t* blk_rec_slot = nullptr;
+  long long blk_lanes = 0;
+  int blk_units = 1;
   std::vector<long long> tokens_hi;
   std::vector<void*> owned;
   long long device_bytes = 0;
@@ -157,38 +168,38 @@ const char* check_config(const wkv_config* c) {
   if (c->merge != 0 && c->merge != 1) return "merge must be 0 or 1";
   if (c->n_splits < 0 || c->n_splits > wkv::kMaxSplits) return "n_splits must be in [0, 64]";
   if (!(c->scale >= 0.f) || std::isinf(c->scale)) return "scale must be finite and >= 0";
-  if (c->schedule < WKV_SCHEDULE_AUTO || c->schedule > WKV_SCHEDULE_CLUSTER) return "schedule must be 0 (auto), 1 (two kernels) or 2 (clusters)";
+  if (c->schedule < WKV_SCHEDULE_AUTO || c->schedule > WKV_SCHEDULE_FLAT) return "schedule must be 0 (auto), 1 (two kernels), 2 (clusters) or 3 (two kernels, flat deal)";
   if ((c->alloc == nullptr) != (c->release == nullptr)) return "alloc and release must both be set or both be NULL";
   if ((long long)c->batch * c->n_kv_heads * wkv::kMaxSplits > 0x7fffffffLL) return "batch * n_kv_heads too large";
   return nullptr;
 }
 
-// Scan CTAs that fit on one SM together (registers and shared memory of the instantiation this configuration runs).
+// Scan CTAs that fit on one SM together (registers and shared memory of the instantiation this configuration runs;
+// flat: the entry of the flat deal).
 template <typename T, int D, int G>
-int scan_ctas_per_sm_of() {
-  using C = wkv::Cfg<T, D, G>;
+int scan_ctas_per_sm_of(bool flat) {
   int n = 0;
   constexpr int smem = wkv::scan_smem_bytes<T, D, G>();
-  if (cudaFuncSetAttribute(wkv::scan_entry<T, D, G>(), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, wkv::scan_entry<T, D, G>(), wkv::kThreads, smem) != cudaSuccess) {
+  if (cudaFuncSetAttribute(wkv::scan_entry<T, D, G>(flat), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, wkv::scan_entry<T, D, G>(flat), wkv::kThreads, smem) != cudaSuccess) {
     cudaGetLastError();
     return 4;
   }
   return n < 1 ? 1 : n;
 }
 template <typename T, int D>
-int scan_ctas_per_sm_by_group(int G) {
+int scan_ctas_per_sm_by_group(int G, bool flat) {
   switch (G) {
-    case 1: return scan_ctas_per_sm_of<T, D, 1>();
-    case 2: return scan_ctas_per_sm_of<T, D, 2>();
-    case 4: return scan_ctas_per_sm_of<T, D, 4>();
-    default: return scan_ctas_per_sm_of<T, D, 8>();
+    case 1: return scan_ctas_per_sm_of<T, D, 1>(flat);
+    case 2: return scan_ctas_per_sm_of<T, D, 2>(flat);
+    case 4: return scan_ctas_per_sm_of<T, D, 4>(flat);
+    default: return scan_ctas_per_sm_of<T, D, 8>(flat);
   }
 }
-int scan_ctas_per_sm(const wkv_config& c) {
+int scan_ctas_per_sm(const wkv_config& c, bool flat) {
   const int G = c.n_q_heads / c.n_kv_heads;
-  if (c.dtype == WKV_BF16) return c.head_dim == 128 ? scan_ctas_per_sm_by_group<__nv_bfloat16, 128>(G) : scan_ctas_per_sm_by_group<__nv_bfloat16, 64>(G);
-  return c.head_dim == 128 ? scan_ctas_per_sm_by_group<float, 128>(G) : scan_ctas_per_sm_by_group<float, 64>(G);
+  if (c.dtype == WKV_BF16) return c.head_dim == 128 ? scan_ctas_per_sm_by_group<__nv_bfloat16, 128>(G, flat) : scan_ctas_per_sm_by_group<__nv_bfloat16, 64>(G, flat);
+  return c.head_dim == 128 ? scan_ctas_per_sm_by_group<float, 128>(G, flat) : scan_ctas_per_sm_by_group<float, 64>(G, flat);
 }
 
 // Splits per lane when the caller leaves the choice to the library: a power of two (so the lane's CTAs can form a
@@ -216,7 +227,80 @@ int auto_splits(const wkv_config& c, long long lanes, long long slots) {
 
 bool is_cluster_size(int s) { return s == 1 || s == 2 || s == 4 || s == 8 || s == 16; }
 
+// The flat deal of the two-kernel schedule (see lane_pieces in wkv_kernels.cuh): tiles per CTA, or 0 to keep whole units
+// per lane.  `units` = the even deal's split count.  Chosen when the even deal would put all its CTAs on the GPU in one
+// wave that fills the SMs unequally -- then the slowest SM sets the time -- or when the caller asks for it; on request
+// n_splits > 0 means that many CTAs per lane on average.  slots / flat_slots: scan CTAs the GPU holds at once under either
+// deal.  `stride` receives the most pieces a lane can have.
+int flat_deal(const wkv_config& c, long long lanes, long long slots, long long flat_slots, int sms, int units, int* stride) {
+  const int tiles = (c.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+  const long long total = lanes * tiles;
+  long long n_ctas;
+  if (c.schedule == WKV_SCHEDULE_FLAT) {
+    n_ctas = c.n_splits > 0 ? lanes * c.n_splits : flat_slots;
+  } else {
+    if (c.schedule != WKV_SCHEDULE_AUTO || c.n_splits > 0) return 0;
+    // Only where the scan is bound by instruction issue, i.e. per SM: four or more query heads per cache row.  A
+    // bandwidth-bound scan shares HBM among all SMs, so an SM holding fewer CTAs simply finishes each of them sooner,
+    // and whole units keep the start-up cost lower (measured: one head per row, 256 lanes x 52 tiles, 44.3 us per layer
+    // call with whole units against 45.2 us flat; four heads per row, 256 lanes x 103 tiles, 99.2 against 96.6 us).
+    if (c.n_q_heads / c.n_kv_heads < 4) return 0;
+    const long long even = lanes * units;
+    if (even > slots || even <= sms || even % sms == 0) return 0;        // several waves, or already level
+    // whole CTAs per SM, at least 8 tiles each
+    const long long per_sm = std::min<long long>(flat_slots / sms, total / (8LL * sms));
+    if (per_sm < 1) return 0;
+    n_ctas = per_sm * sms;
+  }
+  if (n_ctas < 1) n_ctas = 1;
+  long long chunk = (total + n_ctas - 1) / n_ctas;
+  chunk = std::max<long long>(chunk, (tiles + wkv::kMaxSplits - 3) / (wkv::kMaxSplits - 2));   // at most kMaxSplits pieces per lane
+  if (chunk < 1) chunk = 1;
+  if (chunk > 0x3fffffff) return 0;
+  *stride = (int)((tiles + chunk - 1) / chunk) + 1;
+  if (*stride > wkv::kMaxSplits) return 0;
+  return (int)chunk;
+}
+
 constexpr int kMaxDynSmem = 200 * 1024;
+
+// Threads per lane of the lane-epilogue kernel for a launch of `lanes` lanes: 512 (one or two query heads) or 384 (four)
+// when two such CTAs per SM hold every lane at once, else 256.
+inline int epilogue_threads(int G, int lanes, int sms) {
+  if (G <= 2 && lanes <= 2 * sms) return wkv::kEpilogueThreadsWide;
+  if (G == 4 && lanes <= 2 * sms) return wkv::kEpilogueThreadsMid;
+  return wkv::kEpilogueThreads;
+}
+
+// The lane-epilogue kernel: one CTA per lane, launched with programmatic stream serialization (it orders itself
+// against its predecessor on the device).
+template <typename T, int D, int G>
+cudaError_t launch_epilogue(const wkv::StepParams& P, int lanes, int dev, cudaStream_t stream) {
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t k2 = {};
+  k2.gridDim = dim3((unsigned)lanes);
+  int sms = 148;
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int nt = epilogue_threads(G, lanes, sms);
+  k2.blockDim = dim3(nt);
+  k2.stream = stream;
+  k2.attrs = pdl;
+  k2.numAttrs = 1;
+  // room to stage a lane's scores and positions in shared memory, when the lane can be finished out of registers
+  wkv::StepParams P2 = P;
+  const int e_slots = wkv::epilogue_slots_per_thread(G, nt) * nt;
+  P2.ep_stage_slots = (e_slots > 0 && P.budget + 1 <= e_slots) ? P.cap : 0;
+  k2.dynamicSmemBytes = (size_t)P2.ep_stage_slots * 8;
+  if constexpr (G <= 2) {
+    if (nt == wkv::kEpilogueThreadsWide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P2);
+  }
+  if constexpr (G == 4) {
+    if (nt == wkv::kEpilogueThreadsMid) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel_mid<T, D, G>, P2);
+  }
+  return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P2);
+}
 
 // cluster = true: one launch, the n_splits CTAs of a lane form a thread-block cluster;
 // otherwise two launches: the scan over all units, then one CTA per lane on the finished scratch.
@@ -225,24 +309,26 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
   using C = wkv::Cfg<T, D, G>;
   // largest dynamic shared memory size configured per device and kernel (contexts may be driven from several host
   // threads: two of them setting the same attribute twice is harmless, a torn read is not)
-  static std::atomic<int> attr_done[64][2];
+  static std::atomic<int> attr_done[64][3];
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   const int smem = cluster ? C::kFixedBytes + G * P.chunk_cap * 4 : wkv::scan_smem_bytes<T, D, G>();
   if (smem > kMaxDynSmem) return cudaErrorInvalidValue;
-  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_entry<T, D, G>();
-  if (attr_done[dev][cluster].load(std::memory_order_acquire) < smem) {
+  const bool flat = !cluster && P.flat_chunk > 0;
+  const int which = cluster ? 1 : (flat ? 2 : 0);
+  const void* fn = cluster ? (const void*)wkv::decode_step_cluster_kernel<T, D, G> : (const void*)wkv::scan_entry<T, D, G>(flat);
+  if (attr_done[dev][which].load(std::memory_order_acquire) < smem) {
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     if (cluster) {
       e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
       if (e != cudaSuccess) return e;
     }
-    attr_done[dev][cluster].store(smem, std::memory_order_release);
+    attr_done[dev][which].store(smem, std::memory_order_release);
   }
-  const int n_ctas = lanes * P.n_splits;
+  const int n_ctas = P.flat_chunk > 0 ? (int)(((long long)lanes * P.tiles_cap + P.flat_chunk - 1) / P.flat_chunk) : lanes * P.n_splits;
   if (!cluster) {
     // Both kernels are launched with programmatic stream serialization: each may be set up while its predecessor
     // drains and orders itself against it on the device (griddep_wait in the kernels).
@@ -256,31 +342,9 @@ cudaError_t launch_step(const wkv::StepParams& P, int lanes, bool cluster, cudaS
     k1.stream = stream;
     k1.attrs = pdl;
     k1.numAttrs = 1;
-    e = cudaLaunchKernelEx(&k1, wkv::scan_entry<T, D, G>(), P);
+    e = cudaLaunchKernelEx(&k1, wkv::scan_entry<T, D, G>(flat), P);
     if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t k2 = {};
-    k2.gridDim = dim3((unsigned)lanes);
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const bool wide = G <= 2 && lanes <= 2 * sms;        // two wide CTAs per SM hold every lane at once
-    const bool mid = G == 4 && lanes <= 2 * sms;
-    const int nt = wide ? wkv::kEpilogueThreadsWide : (mid ? wkv::kEpilogueThreadsMid : wkv::kEpilogueThreads);
-    k2.blockDim = dim3(nt);
-    k2.stream = stream;
-    k2.attrs = pdl;
-    k2.numAttrs = 1;
-    // room to stage a lane's scores and positions in shared memory, when the lane can be finished out of registers
-    wkv::StepParams P2 = P;
-    const int e_slots = wkv::epilogue_slots_per_thread(G, nt) * nt;
-    P2.ep_stage_slots = (e_slots > 0 && P.budget + 1 <= e_slots) ? P.cap : 0;
-    k2.dynamicSmemBytes = (size_t)P2.ep_stage_slots * 8;
-    if constexpr (G <= 2) {
-      if (wide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P2);
-    }
-    if constexpr (G == 4) {
-      if (mid) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel_mid<T, D, G>, P2);
-    }
-    return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreads>, P2);
+    return launch_epilogue<T, D, G>(P, lanes, dev, stream);
   }
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3((unsigned)n_ctas);
@@ -311,8 +375,11 @@ cudaError_t launch_by_group(int G, const wkv::StepParams& P, int lanes, bool clu
 }
 
 // cluster = false forces the two-kernel schedule (global scratch), which the static-scratch entry point needs.
-cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P, bool cluster, int lanes = 0) {
+cudaError_t launch_any(const wkv_ctx* c, const wkv::StepParams& P_in, bool cluster, int lanes = 0) {
   const int n = lanes > 0 ? lanes : c->lanes_per_layer;
+  wkv::StepParams P = P_in;
+  P.n_lanes = n;
+  if (cluster) P.flat_chunk = 0;
   if (c->cfg.dtype == WKV_BF16) {
     return c->cfg.head_dim == 128 ? launch_by_group<__nv_bfloat16, 128>(c->group, P, n, cluster, c->stream)
                                   : launch_by_group<__nv_bfloat16, 64>(c->group, P, n, cluster, c->stream);
@@ -331,9 +398,14 @@ wkv::StepParams base_params(const wkv_ctx* c, int layer) {
   P.cap = c->cap;
   P.budget = c->cfg.budget; P.window = c->cfg.window; P.sink = c->cfg.sink;
   P.n_splits = c->n_splits;
+  P.flat_chunk = c->flat_chunk;
+  P.tiles_cap = (c->cfg.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
   P.chunk_cap = c->chunk_cap;
   P.merge = c->cfg.merge;
   P.scale = c->scale;
+  P.logit_rows = c->group;
+  P.probs_rows = c->group;
+  P.probs_stride = c->cfg.budget + 1;
   std::memcpy(P.vmap, c->vmap, sizeof(P.vmap));
   return P;
 }
@@ -454,7 +526,8 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   c->lanes_per_layer = cfg->batch * cfg->n_kv_heads;
   c->lanes_total = (long long)cfg->n_layers * c->lanes_per_layer;
   c->cap = (cfg->budget + 1 + 3) & ~3;
-  const long long slots = (long long)c->sm_count * scan_ctas_per_sm(*cfg);
+  const long long slots = (long long)c->sm_count * scan_ctas_per_sm(*cfg, false);
+  const long long flat_slots = (long long)c->sm_count * scan_ctas_per_sm(*cfg, true);
   c->n_splits = cfg->n_splits > 0 ? cfg->n_splits : auto_splits(*cfg, c->lanes_per_layer, slots);
   {
     const int tiles = (cfg->budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
@@ -470,6 +543,11 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     // lanes in a second launch (17.4 vs 18.4 us on 32 lanes x 65 tiles, and far ahead on large shapes)
     c->use_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ||
                      (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_per_layer * tiles < 148 * 4);
+    if (!c->use_cluster) {
+      int stride = 0;
+      const int chunk = flat_deal(*cfg, c->lanes_per_layer, slots, flat_slots, c->sm_count, c->n_splits, &stride);
+      if (chunk > 0) { c->flat_chunk = chunk; c->n_splits = stride; }
+    }
   }
   if (cfg->n_layers > 1 && c->lanes_total * wkv::kMaxSplits < 0x7fffffffLL) {
     // One launch for all layers: the lanes of all layers are just more lanes.  Worth it when a layer alone cannot
@@ -480,6 +558,11 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
     const bool can_cluster = is_cluster_size(c->fused_splits) && c->group * c->fused_chunk_cap * 4 <= 64 * 1024;
     c->fused_cluster = cfg->schedule == WKV_SCHEDULE_CLUSTER ? can_cluster
                        : (cfg->schedule == WKV_SCHEDULE_AUTO && can_cluster && c->lanes_total * tiles < 148 * 4);
+    if (!c->fused_cluster) {
+      int stride = 0;
+      const int chunk = flat_deal(*cfg, c->lanes_total, slots, flat_slots, c->sm_count, c->fused_splits, &stride);
+      if (chunk > 0) { c->fused_flat_chunk = chunk; c->fused_splits = stride; }
+    }
     const size_t bytes = (size_t)c->lanes_total * c->group * ((size_t)c->cap * 4 + (size_t)c->fused_splits * (cfg->head_dim + 2) * 4);
     c->fused_ok = bytes <= ((size_t)64 << 20) && (cfg->schedule != WKV_SCHEDULE_CLUSTER || can_cluster);
   }
@@ -598,6 +681,7 @@ int wkv_decode_step_layers(wkv_ctx* c, const void* q, const void* k, const void*
     // the lanes of all layers in one launch (pair): [n_layers, batch, ...] is [n_layers*batch, ...] to the kernels
     wkv::StepParams P = base_params(c, 0);
     P.n_splits = c->fused_splits;
+    P.flat_chunk = c->fused_flat_chunk;
     P.chunk_cap = c->fused_chunk_cap;
     P.logits = c->fused_logits;
     P.part = c->fused_part;
@@ -727,6 +811,155 @@ static int stream_tokens(wkv_ctx* c, int32_t layer, const void* Q, const void* K
   return WKV_OK;
 }
 
+}  // extern "C"
+
+// ---- blocked prompt tail (wkv_block.cuh) --------------------------------------------------------------------------
+// Tokens per block for this context, or 0 where the tail is streamed token by token: the block's query rows (tokens x
+// query heads per key) must be 8 at most, the window must be longer than the block (an entry removed inside the block and
+// its right neighbour are then never tokens of the block), and the lane epilogue must be the register version.
+static int block_tokens_of(const wkv_ctx* c, int lanes) {
+  if (c->use_cluster || c->group > 4) return 0;
+  const int B = 8 / c->group;
+  if (c->cfg.window <= B) return 0;
+  const int nt = epilogue_threads(c->group, lanes, c->sm_count);
+  if (c->cfg.budget + 1 > wkv::epilogue_slots_per_thread(c->group, nt) * nt) return 0;
+  return B;
+}
+
+template <typename T, int D>
+static cudaError_t launch_block_kernels(int which, const wkv::BlockParams& BP, int lanes, cudaStream_t s) {
+  using namespace wkv;
+  constexpr int R = 8;
+  if (which == 0) {
+    constexpr int smem = BlockCfg<T, D, R>::kLogitsSmem;
+    cudaError_t e = cudaFuncSetAttribute(block_logits_kernel<T, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    block_logits_kernel<T, D, R><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
+  } else if (which == 1) {
+    constexpr int smem = BlockCfg<T, D, R>::kPvSmem;
+    cudaError_t e = cudaFuncSetAttribute(block_pv_kernel<T, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    block_pv_kernel<T, D, R><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
+  } else {
+    block_out_kernel<T, D><<<lanes, D, 0, s>>>(BP);
+  }
+  return cudaGetLastError();
+}
+static cudaError_t launch_block(const wkv_ctx* c, int which, const wkv::BlockParams& BP, int lanes) {
+  if (c->cfg.dtype == WKV_BF16)
+    return c->cfg.head_dim == 128 ? launch_block_kernels<__nv_bfloat16, 128>(which, BP, lanes, c->stream)
+                                  : launch_block_kernels<__nv_bfloat16, 64>(which, BP, lanes, c->stream);
+  return c->cfg.head_dim == 128 ? launch_block_kernels<float, 128>(which, BP, lanes, c->stream)
+                                : launch_block_kernels<float, 64>(which, BP, lanes, c->stream);
+}
+template <typename T, int D>
+static cudaError_t launch_epilogue_by_group(int G, const wkv::StepParams& P, int lanes, int dev, cudaStream_t s) {
+  switch (G) {
+    case 1: return launch_epilogue<T, D, 1>(P, lanes, dev, s);
+    case 2: return launch_epilogue<T, D, 2>(P, lanes, dev, s);
+    case 4: return launch_epilogue<T, D, 4>(P, lanes, dev, s);
+  }
+  return cudaErrorInvalidValue;
+}
+static cudaError_t launch_epilogue_any(const wkv_ctx* c, const wkv::StepParams& P, int lanes) {
+  if (c->cfg.dtype == WKV_BF16)
+    return c->cfg.head_dim == 128 ? launch_epilogue_by_group<__nv_bfloat16, 128>(c->group, P, lanes, c->device, c->stream)
+                                  : launch_epilogue_by_group<__nv_bfloat16, 64>(c->group, P, lanes, c->device, c->stream);
+  return c->cfg.head_dim == 128 ? launch_epilogue_by_group<float, 128>(c->group, P, lanes, c->device, c->stream)
+                                : launch_epilogue_by_group<float, 64>(c->group, P, lanes, c->device, c->stream);
+}
+
+// Tokens [t_begin, T_max) of a prompt for `lanes` consecutive lanes starting at lane0 (one layer, or all layers: to the
+// kernels the sequences of several layers are just more sequences), B tokens per pair of cache sweeps.
+// q_bs / kv_bs: batch strides of Q and K, V in elements; seq_lens indexed by lane / n_kv_heads.
+static int blocked_tokens(wkv_ctx* c, long long lane0, int lanes, int B, const void* Q, const void* K, const void* V,
+                          const int32_t* seq_lens, int32_t t_begin, int32_t T_max, void* out, int32_t* evicted_pos) {
+  const long long D = c->cfg.head_dim, Hq = c->cfg.n_q_heads, Hk = c->cfg.n_kv_heads;
+  const int R = 8, G = c->group;
+  const size_t cap = c->cap;
+  if (c->blk_logits == nullptr || c->blk_lanes < lanes) {
+    const int tiles = (c->cfg.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+    int units = (int)((6LL * c->sm_count + lanes - 1) / lanes);
+    units = std::max(1, std::min({units, 16, std::max(1, tiles / 8)}));
+    int rc = WKV_OK;
+    if (rc == WKV_OK) rc = take(c, &c->blk_logits, (size_t)lanes * R * cap * 4);
+    if (rc == WKV_OK) rc = take(c, &c->blk_lgx, (size_t)lanes * R * B * 4 + 256);
+    if (rc == WKV_OK) rc = take(c, &c->blk_ptab, (size_t)lanes * R * cap * 4 + 256);   // the last tile of the last row is read whole
+    if (rc == WKV_OK) rc = take(c, &c->blk_opart, (size_t)lanes * units * R * D * 4);
+    if (rc == WKV_OK) rc = take(c, &c->blk_rec_rows, (size_t)lanes * 2 * B * D * 4);
+    if (rc == WKV_OK) rc = take(c, &c->blk_rec_slot, (size_t)lanes * 2 * B * 4);
+    if (rc != WKV_OK) { c->blk_logits = nullptr; c->blk_lanes = 0; return rc; }
+    c->blk_lanes = lanes;
+    c->blk_units = units;
+  }
+  wkv::BlockParams BP;
+  std::memset(&BP, 0, sizeof(BP));
+  BP.Kc = c->Kc; BP.Vc = c->Vc; BP.lane_state = c->lane_state;
+  BP.Q = Q; BP.K = K; BP.out = out; BP.seq_lens = seq_lens;
+  BP.logits = c->blk_logits; BP.lgx = c->blk_lgx; BP.ptab = c->blk_ptab; BP.opart = c->blk_opart;
+  BP.rec_rows = c->blk_rec_rows; BP.rec_slot = c->blk_rec_slot; BP.status = c->status;
+  BP.q_bs = (long long)T_max * Hq * D; BP.kv_bs = (long long)T_max * Hk * D; BP.out_bs = BP.q_bs;
+  BP.q_ts = Hq * D; BP.kv_ts = Hk * D; BP.out_ts = Hq * D;
+  BP.lane0 = (int)lane0; BP.n_kv_heads = c->cfg.n_kv_heads; BP.cap = c->cap; BP.budget = c->cfg.budget;
+  BP.block_tokens = B; BP.group = G; BP.n_units = c->blk_units; BP.scale = c->scale;
+
+  wkv::StepParams P = base_params(c, 0);
+  P.lane0 = (int)lane0;
+  P.n_lanes = lanes;
+  P.flat_chunk = 0;
+  P.n_splits = 1;
+  P.part = nullptr;
+  P.ticket = nullptr;
+  P.wait_at_start = 2;
+  P.logits = c->blk_logits;
+  P.lgx = c->blk_lgx;
+  P.rec_rows = c->blk_rec_rows;
+  P.rec_slot = c->blk_rec_slot;
+  P.logit_rows = R;
+  P.block_tokens = B;
+  P.probs = out ? c->blk_ptab : nullptr;
+  P.probs_rows = R;
+  P.probs_stride = (int)cap;
+  P.seq_lens = seq_lens;
+  P.q_bs = BP.q_bs; P.kv_bs = BP.kv_bs;
+  P.out = nullptr; P.out_bs = 0;
+  P.ev_bs = evicted_pos ? (long long)T_max * Hk : Hk;
+  for (int t0 = t_begin; t0 < T_max; t0 += B) {
+    const int n_tok = std::min<int>(B, T_max - t0);
+    BP.tok0 = t0;
+    BP.n_tok = n_tok;
+    cudaError_t e = launch_block(c, 0, BP, lanes);
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "block logits launch");
+    for (int i = 0; i < n_tok; ++i) {
+      const int t = t0 + i;
+      P.tok_idx = t;
+      P.block_step = i;
+      P.logit_row0 = i * G;
+      P.probs_row0 = i * G;
+      P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
+      P.k = (const char*)K + (size_t)t * Hk * D * c->elem;
+      P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
+      P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
+      e = launch_epilogue_any(c, P, lanes);
+      c->launches += 1;
+      if (e != cudaSuccess) return cuda_fail(c, e, "lane epilogue launch (blocked prompt tail)");
+    }
+    if (out) {
+      e = launch_block(c, 1, BP, lanes);
+      if (e == cudaSuccess) e = launch_block(c, 2, BP, lanes);
+      c->launches += 2;
+      if (e != cudaSuccess) return cuda_fail(c, e, "block output launch");
+    }
+  }
+  c->last_layer = -1;
+  g_last_launcher.store(nullptr);
+  note_outputs(c, nullptr, 0, nullptr, 0, nullptr, 0);
+  return WKV_OK;
+}
+
+extern "C" {
+
 static int check_prefill_args(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const void* V, int32_t T_max) {
   if (!c) return WKV_ERR_INVALID;
   if (!Q || !K || !V) return fail(c, WKV_ERR_INVALID, "Q, K and V must not be NULL");
@@ -808,6 +1041,13 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     if (rc != WKV_OK) return rc;
     c->tokens_hi[layer] += n0;
   }
+  // the rest: in blocks of tokens that share two sweeps of the cache where the configuration allows, else token by token
+  const int B = block_tokens_of(c, c->lanes_per_layer);
+  if (B > 0 && T_max - n0 >= 2) {
+    c->tokens_hi[layer] += T_max - n0;
+    return blocked_tokens(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, B, Q, K, V, seq_lens, n0, T_max, out,
+                          evicted_pos);
+  }
   return stream_tokens(c, layer, Q, K, V, seq_lens, n0, T_max, out, evicted_pos);
 }
 
@@ -851,6 +1091,28 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
   // layer's lane epilogues.
   for (auto& th : c->tokens_hi) th += T_max - n0;
   c->last_layer = -1;
+  if (T_max - n0 >= 2) {
+    // the rest in blocks of tokens (wkv_block.cuh) where the configuration allows: over the lanes of all layers at once
+    // when a layer alone is small, else layer after layer (the layers' prompts are independent)
+    const int B_all = c->fused_ok ? block_tokens_of(c, (int)c->lanes_total) : 0;
+    const int B_one = block_tokens_of(c, c->lanes_per_layer);
+    if (B_all > 0) {
+      if (seq_lens != nullptr)
+        for (int l = 0; l < L; ++l)
+          WKV_CUDA(c, cudaMemcpyAsync(c->fused_seq_lens + (size_t)l * B, seq_lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, c->stream));
+      return blocked_tokens(c, 0, (int)c->lanes_total, B_all, Q, K, V, seq_lens != nullptr ? c->fused_seq_lens : nullptr, n0, T_max,
+                            out, evicted_pos);
+    }
+    if (B_one > 0) {
+      for (int l = 0; l < L; ++l) {
+        rc = blocked_tokens(c, (long long)l * c->lanes_per_layer, c->lanes_per_layer, B_one, (const char*)Q + l * q_layer,
+                            (const char*)K + l * kv_layer, (const char*)V + l * kv_layer, seq_lens, n0, T_max,
+                            out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr);
+        if (rc != WKV_OK) return rc;
+      }
+      return WKV_OK;
+    }
+  }
   if (c->fused_ok && n0 < T_max) {
     // a layer alone cannot fill the GPU: one launch (pair) per token over the lanes of all layers, as in
     // wkv_decode_step_layers; [n_layers, batch, ...] is [n_layers * batch, ...] to the kernels
@@ -859,6 +1121,7 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
         WKV_CUDA(c, cudaMemcpyAsync(c->fused_seq_lens + (size_t)l * B, seq_lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, c->stream));
     wkv::StepParams P = base_params(c, 0);
     P.n_splits = c->fused_splits;
+    P.flat_chunk = c->fused_flat_chunk;
     P.chunk_cap = c->fused_chunk_cap;
     P.logits = c->fused_logits;
     P.part = c->fused_part;

@@ -64,7 +64,7 @@ struct StepParams {
   int32_t* prev;         // [lanes_total][cap]
   int32_t* lane_state;   // [lanes_total][LS_STRIDE]
   float* logits;         // scratch [lanes_per_layer*G][cap]
-  float* part;           // scratch [lanes_per_layer][n_splits][G][D+2] : m, l, o[D]
+  float* part;           // scratch [lanes_per_layer][n_splits][G][D+2] : m, l, o[D] per unit / piece of a lane
   uint32_t* ticket;      // scratch [lanes_per_layer] or nullptr: units of the lane whose scan is finished (zero between calls)
   uint32_t* status;      // device status word
   const void* q;         // [B][..][Hq][D]   batch stride q_bs elements
@@ -80,11 +80,24 @@ struct StepParams {
   int n_kv_heads;
   int cap;               // slots per lane (>= budget+1, multiple of 4)
   int budget, window, sink;
-  int n_splits;
+  int n_splits;          // units per lane (even deal); with the flat deal: the most pieces a lane can have
+  int flat_chunk;        // 0: even deal, CTA = (lane, unit).  c > 0: flat deal, CTA i takes tiles [i*c, (i+1)*c) of all lanes' tiles
+  int tiles_cap;         // flat deal: tiles per lane in that sequence = ceil((budget + 1) / 32)
+  int n_lanes;           // lanes of this launch
   int chunk_cap;         // cluster kernel: logits one CTA can hold per query head (its tiles * 32)
   int merge;
   int wait_at_start;     // scan kernel: how it orders itself against the preceding kernel, 0 / 1 / 2 (see scan_kernel)
   int ep_stage_slots;    // lane epilogue kernel: entries of a and pos its dynamic shared memory can stage (0: none)
+  // Where the lane epilogue finds its logits and puts the optional probabilities: logits of query head g of lane x at
+  // logits[(x * logit_rows + logit_row0 + g) * cap + slot], probabilities at probs[(x * probs_rows + probs_row0 + g) *
+  // probs_stride + slot].  A decode step has logit_rows = probs_rows = G, row0 = 0, probs_stride = budget + 1.
+  int logit_rows, logit_row0, probs_rows, probs_row0, probs_stride;
+  // Blocked prompt tail (wkv_block.cuh): this launch finishes token number block_step of a block of block_tokens tokens
+  // (0: not a blocked tail) whose logits against the cache as it was before the block were parked by one sweep.
+  int block_tokens, block_step;
+  const float* lgx;      // [lanes][logit_rows][block_tokens]: logits against the block's own keys (entries that joined inside the block)
+  float* rec_rows;       // [lanes][2 * block_tokens][D] fp32: value rows as they were before a step of the block changed them
+  int32_t* rec_slot;     // [lanes][2 * block_tokens]: their slots (entry 2*step: the removed entry, 2*step + 1: its right neighbour), -1 = none
   float scale;
   // Tensor map over the value cache as a [lanes_total * cap][D] matrix: boxes of 64 elements x 32 rows, 128-byte
   // swizzle.  Encoded by the host for configurations whose scan takes its V tiles that way (Cfg::kMmaPV), else unused.
@@ -347,7 +360,9 @@ struct Cfg {
   static constexpr int kAuxBytes = 2 * kRowBytes;           // k row and v row of the new token
   static constexpr int kWarpPartFloats = kConsumerWarps * G * (D + 2);
   static constexpr int kCtaPartFloats = G * (D + 2);
-  // ring | new token rows | warp partials | CTA partial | mbarriers | epilogue scalars | (cluster: chunk logits)
+  // ring | new token rows | warp partials | mbarriers: all that a scan kernel uses
+  static constexpr int kScanBytes = kRingBytes + kAuxBytes + kWarpPartFloats * 4 + 2 * kStages * 8 + 128;
+  // ring | new token rows | warp partials | mbarriers | CTA partial | epilogue scalars | (cluster: chunk logits)
   static constexpr int kFixedBytes = kRingBytes + kAuxBytes + (kWarpPartFloats + kCtaPartFloats) * 4 + 2 * kStages * 8 +
                                      EpScratch::bytes(G) + 128;
 };
@@ -367,11 +382,11 @@ struct Smem {
     ring = raw;
     aux = reinterpret_cast<T*>(ring + C::kRingBytes);
     warp_part = reinterpret_cast<float*>(ring + C::kRingBytes + C::kAuxBytes);
-    cta_part = warp_part + C::kWarpPartFloats;
-    full_bar = reinterpret_cast<uint64_t*>(cta_part + C::kCtaPartFloats);
+    full_bar = reinterpret_cast<uint64_t*>(warp_part + C::kWarpPartFloats);
     empty_bar = full_bar + C::kStages;
-    ep.carve(reinterpret_cast<unsigned char*>(empty_bar + C::kStages), G);
-    chunk_logits = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(empty_bar + C::kStages) + EpScratch::bytes(G));
+    cta_part = reinterpret_cast<float*>(empty_bar + C::kStages);
+    ep.carve(reinterpret_cast<unsigned char*>(cta_part + C::kCtaPartFloats), G);
+    chunk_logits = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(cta_part + C::kCtaPartFloats) + EpScratch::bytes(G));
   }
   __device__ __forceinline__ T* aux_k(int) const { return aux; }
   __device__ __forceinline__ T* aux_v(int) const { return aux + D; }
@@ -415,6 +430,39 @@ __device__ __forceinline__ void fill_view(LaneView<T>& v, const StepParams& P, i
   v.n_tiles = base + (split < extra ? 1 : 0);
   v.slot_begin = min(v.L, v.tile_begin * kTileSlots);
   v.slot_end = min(v.L, (v.tile_begin + v.n_tiles) * kTileSlots);
+}
+
+// The flat deal of the two-kernel schedule.  The tiles of all lanes of a launch, P.tiles_cap per lane, form one
+// sequence, lane after lane, and CTA i scans tiles [i*c, (i+1)*c) of it, c = P.flat_chunk: every CTA gets the same
+// number of tiles whatever the number of lanes, so one wave of CTAs fills every SM equally -- with whole units per lane
+// the CTA count is a multiple of the lane count and the SMs hold unequal numbers of them.  A CTA's range may end one
+// lane and begin the next: per lane it holds a "piece", which it treats as the even deal treats a unit (own partial,
+// own report to the lane's epilogue).  The pieces of a lane belong to consecutive CTAs.
+// first CTA and number of pieces (units) of a lane, under either deal
+__device__ __forceinline__ void lane_pieces(const StepParams& P, int lane_local, int& first_cta, int& n_pieces) {
+  if (P.flat_chunk == 0) {
+    first_cta = lane_local * P.n_splits;
+    n_pieces = P.n_splits;
+  } else {
+    const long long g0 = (long long)lane_local * P.tiles_cap;
+    first_cta = (int)(g0 / P.flat_chunk);
+    n_pieces = (int)((g0 + P.tiles_cap - 1) / P.flat_chunk) - first_cta + 1;
+  }
+}
+// The piece of lane `lane_local` that CTA `cta` holds under the flat deal: tiles [tb, te) of the lane, clipped to the
+// tiles the lane really has; sets the view's share and returns the piece's index among the lane's pieces.
+template <typename T>
+__device__ __forceinline__ int flat_piece(LaneView<T>& v, const StepParams& P, int lane_local, int cta) {
+  const long long lane_g0 = (long long)lane_local * P.tiles_cap;
+  const long long g0 = (long long)cta * P.flat_chunk, g1 = g0 + P.flat_chunk;
+  const int tb = (int)max(g0 - lane_g0, 0ll), te = (int)min(g1 - lane_g0, (long long)P.tiles_cap);
+  const int tiles_total = (v.L + kTileSlots - 1) / kTileSlots;
+  v.tile_begin = min(tb, tiles_total);
+  v.n_tiles = max(0, min(te, tiles_total) - tb);
+  v.slot_begin = min(v.L, tb * kTileSlots);
+  v.slot_end = min(v.L, te * kTileSlots);
+  v.split = cta - (int)(lane_g0 / P.flat_chunk);
+  return v.split;
 }
 
 // Producer side of one ring stage (one thread): `rows` cache rows of K in one bulk copy and the same rows of V in one
@@ -487,6 +535,19 @@ struct Scanner {
     if constexpr (MMA) {
 #pragma unroll
       for (int j = 0; j < NB; ++j) oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.f;
+    }
+  }
+  // The same start for query rows that are not contiguous: row r is head r % group of token min(r / group, n_tok - 1),
+  // tokens tok_stride elements apart (the blocked prompt tail scans for several tokens of a prompt at once).
+  __device__ __forceinline__ void begin_rows(const T* q, long long tok_stride, int group, int n_tok) {
+    const int l = (threadIdx.x & 31) % LPR;
+    m_run = -INFINITY;
+    l_run = 0.f;
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      const T* row = q + (long long)min(g / group, n_tok - 1) * tok_stride + (long long)(g % group) * D;
+#pragma unroll
+      for (int j = 0; j < NP; ++j) load_pairs<CP>(row + (l + LPR * j) * CH, qf[g][j]);
     }
   }
   // 32-bit word w of row `row` of a stage's V tile: plain rows, or (MMA) the swizzled halves that the tensor-map copies
@@ -689,44 +750,6 @@ struct Scanner {
     }  // !MMA
   }
 
-  // Two-phase scan (MMA configurations): the value phase starts from zero accumulators and ends with the warp's partial
-  // (m = the unit's maximum of the head, l = sum of the warp's probabilities, o[D]) in shared memory.  l_mine is the sum
-  // over the tiles of this thread's own (row, head) probabilities.
-  __device__ __forceinline__ void begin_pv() {
-#pragma unroll
-    for (int j = 0; j < NB; ++j) oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.f;
-  }
-  __device__ __forceinline__ void end_pv(float* warp_part, float m_unit, float l_mine) {
-    const int warp = threadIdx.x >> 5, lane_id = threadIdx.x & 31;
-    const int rg = lane_id / LPR, l = lane_id % LPR;
-    const int my_head = l / LH, li = l % LH;
-    // the head's eight rows of every tile: four threads (li) in each of the two row groups
-    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 1);
-    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 2);
-    l_mine += __shfl_xor_sync(0xffffffffu, l_mine, 16);
-    const int c = lane_id >> 2, q = lane_id & 3;
-#pragma unroll
-    for (int j = 0; j < NB; ++j)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) oc[j][i] += __shfl_xor_sync(0xffffffffu, oc[j][i], 2);   // high-part + low-part columns
-    if (q < 2) {
-      float* wa = warp_part + (warp * G + 2 * q) * (D + 2) + 2;
-      float* wb = wa + (D + 2);
-#pragma unroll
-      for (int j = 0; j < NB; ++j) {
-        wa[16 * j + c] = oc[j][0];
-        wb[16 * j + c] = oc[j][1];
-        wa[16 * j + 8 + c] = oc[j][2];
-        wb[16 * j + 8 + c] = oc[j][3];
-      }
-    }
-    if (rg == 0 && li == 0) {
-      float* wp = warp_part + (warp * G + my_head) * (D + 2);
-      wp[0] = m_unit;
-      wp[1] = l_mine;
-    }
-  }
-
   // Fold the warp's row groups and leave the warp's partial (m, l, o[D]) per query head in shared memory.
   __device__ __forceinline__ void end(float* warp_part) {
     const float kLog2e = 1.4426950408889634f;
@@ -892,8 +915,7 @@ __device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>&
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     pg[g] = __fdiv_rn(e[g], Z[g]);
-    if (P.probs)
-      P.probs[((long long)v.b * P.n_kv_heads * G + (long long)v.hk * G + g) * (P.budget + 1) + slot] = pg[g];
+    if (P.probs) P.probs[((long long)v.lane_local * P.probs_rows + P.probs_row0 + g) * P.probs_stride + slot] = pg[g];
   }
   float pbar = pg[0];
 #pragma unroll
@@ -984,7 +1006,9 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
   // (the row of this step's token may have been written to the cache by other threads: v.new_v is the safe copy)
   float vj = 0.f;
   const bool merging = compress && P.merge && j_slot >= 0;
-  if (merging && tid < D) vj = to_f32(j_slot == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)j_slot * D + tid));
+  const bool blocked = P.block_tokens > 0;               // blocked prompt tail: rows that this step changes are recorded
+  if ((merging || (blocked && compress && j_slot >= 0)) && tid < D)
+    vj = to_f32(j_slot == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)j_slot * D + tid));
   // ... and so can the right neighbour's row, without waiting for thread 0's walk: r = next[j], which this step
   // changes only if j is the old tail (then r is the new entry).  One round trip less on the lane's critical path.
   int r_early = -1;
@@ -1033,6 +1057,11 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     v.st[LS_TAIL] = tail;
     v.st[LS_FREE] = new_free;
     if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = ev_pos;
+    if (blocked) {
+      int32_t* rs = P.rec_slot + ((long long)v.lane_local * P.block_tokens + P.block_step) * 2;
+      rs[0] = ep.i32[2];                                   // the removed entry's slot (-1: nothing removed)
+      rs[1] = (ep.i32[2] >= 0 && P.merge) ? ep.i32[3] : -1;
+    }
   }
   group_sync<NT>();
   // V[r] <- (abar_j V[j] + abar_r V[r]) / (abar_j + abar_r), stored in T
@@ -1041,7 +1070,10 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     const float wj = ep.misc[0], wr = ep.misc[1];
     const float vr = r == r_early ? vr_early : to_f32(r == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r * D + tid));
     Vw[(long long)r * D + tid] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
+    if (blocked) P.rec_rows[(((long long)v.lane_local * P.block_tokens + P.block_step) * 2 + 1) * D + tid] = vr;
   }
+  if (blocked && compress && ep.i32[2] >= 0 && tid < D)
+    P.rec_rows[(((long long)v.lane_local * P.block_tokens + P.block_step) * 2) * D + tid] = vj;
 }
 
 // Steps (1) and (2) of a lane's epilogue from global scratch: the split weights, the global maximum and normaliser of
@@ -1051,6 +1083,8 @@ __device__ __forceinline__ void combine_partials(const StepParams& P, const Lane
   const float kLog2e = 1.4426950408889634f;
   const int tid = threadIdx.x;
   const float* part = P.part + (long long)v.lane_local * P.n_splits * G * (D + 2);
+  int first_cta, n_pieces;
+  lane_pieces(P, v.lane_local, first_cta, n_pieces);
   // (1) split weights and the global max / normaliser of every query head
   // (warp g takes head g, a lane takes splits lane and lane + 32: one round of loads instead of a serial loop)
   static_assert(NT / 32 >= G && kMaxSplits <= 64, "one warp per query head, two splits per lane");
@@ -1058,7 +1092,7 @@ __device__ __forceinline__ void combine_partials(const StepParams& P, const Lane
     const int g = tid >> 5, lq = tid & 31;
     const float* pg = part + g * (D + 2);
     const long long st = (long long)G * (D + 2);
-    const bool has0 = lq < P.n_splits, has1 = lq + 32 < P.n_splits;
+    const bool has0 = lq < n_pieces, has1 = lq + 32 < n_pieces;
     const float m0 = has0 ? __ldcg(pg + lq * st) : -INFINITY, l0 = has0 ? __ldcg(pg + lq * st + 1) : 0.f;
     const float m1 = has1 ? __ldcg(pg + (lq + 32) * st) : -INFINITY, l1 = has1 ? __ldcg(pg + (lq + 32) * st + 1) : 0.f;
     float M = fmaxf(m0, m1);
@@ -1083,7 +1117,7 @@ __device__ __forceinline__ void combine_partials(const StepParams& P, const Lane
       const int g = idx / D, c = idx % D;
       const float* pg = part + g * (D + 2) + 2 + c;
       float o = 0.f;
-      for (int s = 0; s < P.n_splits; ++s) o += ep.w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
+      for (int s = 0; s < n_pieces; ++s) o += ep.w[g * kMaxSplits + s] * __ldcg(pg + (long long)s * G * (D + 2));
       out[idx] = from_f32<T>(o * ep.linv[g]);
     }
   }
@@ -1091,12 +1125,11 @@ __device__ __forceinline__ void combine_partials(const StepParams& P, const Lane
 
 // Zeroes of the optional probability output beyond the lane's entries.
 template <int G, int NT>
-__device__ __forceinline__ void clear_probs_tail(const StepParams& P, int b, int hk, int L) {
+__device__ __forceinline__ void clear_probs_tail(const StepParams& P, int lane_local, int L) {
   if (P.probs) {
     for (int i = L + (int)threadIdx.x; i < P.budget + 1; i += NT)
 #pragma unroll
-      for (int g = 0; g < G; ++g)
-        P.probs[((long long)b * P.n_kv_heads * G + (long long)hk * G + g) * (P.budget + 1) + i] = 0.f;
+      for (int g = 0; g < G; ++g) P.probs[((long long)lane_local * P.probs_rows + P.probs_row0 + g) * P.probs_stride + i] = 0.f;
   }
 }
 
@@ -1104,7 +1137,7 @@ __device__ __forceinline__ void clear_probs_tail(const StepParams& P, int b, int
 template <typename T, int D, int G, int NT>
 __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
   const int L = v.L;
-  float* lg = P.logits + (long long)v.lane_local * G * P.cap;
+  float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.cap;
   combine_partials<T, D, G, NT>(P, v, ep);
   // (3) Z_g as an exact integer sum
   float Zr[G];
@@ -1120,7 +1153,7 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
   unsigned long long best = ~0ull;
   int best_slot = -1;
   fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, Zr, compress, best, best_slot);
-  clear_probs_tail<G, NT>(P, v.b, v.hk, L);
+  clear_probs_tail<G, NT>(P, v.lane_local, L);
   int j_slot;
   const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
@@ -1136,7 +1169,7 @@ template <typename T, int D, int G, int NT, int E>
 __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, const LaneView<T>& v, const EpScratch& ep,
                                                            const float* a_s, const int* pos_s) {
   const int tid = threadIdx.x, L = v.L;
-  const float* lg = P.logits + (long long)v.lane_local * G * P.cap;
+  const float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.cap;
   float sx[E][G];
 #pragma unroll
   for (int u = 0; u < E; ++u) {
@@ -1144,7 +1177,40 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
 #pragma unroll
     for (int g = 0; g < G; ++g) sx[u][g] = i < L ? __ldcg(lg + (long long)g * P.cap + i) : -INFINITY;
   }
-  combine_partials<T, D, G, NT>(P, v, ep);
+  if (P.block_tokens > 0) {
+    // Blocked prompt tail: the parked logits were taken against the cache as it was before the block.  An entry that
+    // joined inside the block (its position says so) has its logit in the small table of the block's own keys.
+    const int t0 = v.t - P.block_step;
+    const float* lx = P.lgx + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.block_tokens;
+#pragma unroll
+    for (int u = 0; u < E; ++u) {
+      const int i = tid + u * NT;
+      if (i < L && pos_s[i] >= t0) {
+#pragma unroll
+        for (int g = 0; g < G; ++g) sx[u][g] = __ldcg(lx + g * P.block_tokens + (pos_s[i] - t0));
+      }
+    }
+    // no split partials here: the maximum of every head comes from the logits themselves (exact, order-free)
+    float mx[G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      mx[g] = -INFINITY;
+#pragma unroll
+      for (int u = 0; u < E; ++u) mx[g] = fmaxf(mx[g], sx[u][g]);
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) mx[g] = fmaxf(mx[g], __shfl_xor_sync(0xffffffffu, mx[g], off));
+      if ((tid & 31) == 0) ep.w[g * kMaxSplits + (tid >> 5)] = mx[g];
+    }
+    group_sync<NT>();
+    if (tid < G) {
+      float m = ep.w[tid * kMaxSplits];
+      for (int w = 1; w < NT / 32; ++w) m = fmaxf(m, ep.w[tid * kMaxSplits + w]);
+      ep.M[tid] = m;
+    }
+    group_sync<NT>();
+  } else {
+    combine_partials<T, D, G, NT>(P, v, ep);
+  }
   // (3) e = exp(s - M) in place, Z_g as an exact integer sum
   float Zr[G];
   {
@@ -1177,7 +1243,7 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
     const int i = tid + u * NT;
     if (i < L) fold_one<T, G>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot);
   }
-  clear_probs_tail<G, NT>(P, v.b, v.hk, L);
+  clear_probs_tail<G, NT>(P, v.lane_local, L);
   int j_slot;
   const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
@@ -1189,8 +1255,9 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
 // scratch, nothing else -- its CTAs are short-lived and all alike, which keeps HBM busy.  A2 runs one CTA per lane
 // on the finished scratch: o_t, probabilities, score fold, pick, merge, relink.
 // ------------------------------------------------------------------------------------------------
+// The scan under the even deal: CTA = (lane, unit).
 template <typename T, int D, int G>
-__device__ __forceinline__ void scan_body(const StepParams& P) {
+__device__ __forceinline__ void scan_body_even(const StepParams& P) {
   using C = Cfg<T, D, G>;
   constexpr int kStages = C::kStages;
   constexpr int NT = kThreads;
@@ -1299,210 +1366,164 @@ __device__ __forceinline__ void scan_body(const StepParams& P) {
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// The scan for four query heads on bf16 rows (Cfg::kMmaPV) in two phases per unit: first every K tile of the unit
-// (logits, parked as always, and the unit's exact maximum per head), then every V tile (probabilities against that
-// maximum, P.V on the tensor cores).  With four heads per cache row the scan is bound by instruction issue, not by
-// bandwidth, and the single-pass form needs the four query rows AND the output accumulators in registers at once
-// (96 per thread, four CTAs per SM).  Apart, each phase fits 64 registers, so six CTAs share an SM, and the online
-// softmax with its per-tile rescaling disappears.  A thread re-reads in phase two exactly the one logit per tile that
-// it parked itself in phase one.  The ring holds single tiles (K or V), twice as many stages in the same bytes; the
-// warp partials are written over the ring once every warp is done with it.
-// ------------------------------------------------------------------------------------------------
-template <typename T, int D, int G>
-struct TwoPhase {
+// The scan under either deal as a loop over the CTA's pieces; compiled for the flat deal (kFlat, P.flat_chunk > 0): the
+// even deal's single pass above carries no loop state and starts a little faster, which 2560 short CTAs per launch feel.
+template <typename T, int D, int G, bool kFlat>
+__device__ __forceinline__ void scan_body(const StepParams& P) {
   using C = Cfg<T, D, G>;
-  static constexpr int kStages = WKV_RING_BYTES / C::kTileBytes;
-  static constexpr int kRingBytes = kStages * C::kTileBytes;
-  static_assert(kStages >= 2 && C::kVHalves * C::kVHalfBytes == C::kTileBytes, "a stage holds one tile of either kind");
-  static_assert(C::kWarpPartFloats * 4 <= kRingBytes, "the warp partials reuse the ring");
-  // ring | new token rows | mbarriers | per-warp maxima
-  static constexpr int kSmemBytes = kRingBytes + C::kAuxBytes + 2 * kStages * 8 + kConsumerWarps * G * 4 + 64;
-};
-
-template <typename T, int D, int G>
-__device__ __forceinline__ void scan_body_two_phase(const StepParams& P) {
-  using C = Cfg<T, D, G>;
-  using TP = TwoPhase<T, D, G>;
-  using SC = Scanner<T, D, G>;
-  static_assert(C::kMmaPV && SC::PASSES == 4 && SC::LH == 4 && SC::RPP == 2, "16 threads per row, one logit per thread and tile");
-  constexpr int NS = TP::kStages;
-  constexpr int NT = kThreads;
-  const float kLog2e = 1.4426950408889634f;
+  constexpr int kStages = C::kStages;
+  constexpr int NC = kConsumerWarps * 32;               // consumer threads: 0 .. NC-1; thread NC is the producer
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  unsigned char* ring = smem_raw;
-  T* aux = reinterpret_cast<T*>(ring + TP::kRingBytes);                       // [ k: D | v: D ] this step's token
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(ring + TP::kRingBytes + C::kAuxBytes);
-  uint64_t* empty_bar = full_bar + NS;
-  float* wmax = reinterpret_cast<float*>(empty_bar + NS);                     // [warp][G] maxima of phase one
-  float* warp_part = reinterpret_cast<float*>(ring);                          // [warp][G][D+2], after the scan
+  const Smem<T, D, G> sm(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane_id = tid & 31;
-  const int split = blockIdx.x % P.n_splits;
-  const int lane_local = blockIdx.x / P.n_splits;
-  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
-  // ordering against the preceding kernel: as in scan_body
+  // Ordering against the kernel launched just before this one (P.wait_at_start, chosen by the host):
+  //   2  wait right here: the predecessor may touch this layer's lanes (same layer twice in a row, reset, ...).
+  //   1  the predecessor works on other memory, but the caller's q, k, v may come from it: set up, read the lanes'
+  //      state and put the first K/V tiles in flight, then wait before the first read of a caller input.
+  //   0  the caller has handed over all layers of a step at once (wkv_decode_step_layers): the predecessor is the lane
+  //      epilogue of the previous layer (other lanes, other scratch set); scan alongside it and wait only at the very
+  //      end, before the unit reports to its lane's epilogue, so that the completion of this grid -- and any report of
+  //      it -- still implies the completion of everything before it and later kernels need not reason about more than
+  //      one predecessor.
   if (P.wait_at_start == 2) griddep_wait();
   griddep_launch();
-  if (P.wait_at_start == 1 && P.seq_lens != nullptr) griddep_wait();
-  if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) {
-    if (P.wait_at_start != 2) griddep_wait();
-    return;
+  if (P.wait_at_start == 1 && P.seq_lens != nullptr) griddep_wait();     // seq_lens is a caller input
+  // the lanes this CTA works on: one under the even deal, one or more (a piece of each) under the flat deal
+  int lane_lo, lane_hi;
+  if constexpr (!kFlat) {
+    lane_lo = lane_hi = blockIdx.x / P.n_splits;
+  } else {
+    const long long g0 = (long long)blockIdx.x * P.flat_chunk;
+    const long long g1 = min(g0 + P.flat_chunk, (long long)P.n_lanes * P.tiles_cap);
+    lane_lo = (int)(g0 / P.tiles_cap);
+    lane_hi = g1 > g0 ? (int)((g1 - 1) / P.tiles_cap) : lane_lo - 1;
   }
-  LaneView<T> v;
-  {
+  // the view of one of those lanes and this CTA's share of it; false: the lane's sequence is already consumed (ragged prefill)
+  auto view_of = [&](int lane_local, LaneView<T>& v) -> bool {
+    const int b = lane_local / P.n_kv_heads;
+    if (P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]) return false;
     const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
-    fill_view<T, D>(v, P, lane_local, split, st[LS_LEN], st[LS_T], st[LS_FREE]);
-  }
-  v.new_k = aux;
-  v.new_v = aux + D;
-  const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
-  const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
-  const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
-  if (tid == 32 && v.slot_end > v.slot_begin) {
-    const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);
-    l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
-    l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
-  }
-  const int n = v.n_tiles;
-  // item x of the unit's stream: K tile x for x < n, then V tile x - n
-  auto issue = [&](int x) {
-    const int s = x % NS;
-    unsigned char* dst = ring + (size_t)s * C::kTileBytes;
-    const int slot0 = (v.tile_begin + (x < n ? x : x - n)) * kTileSlots;
-    if (x < n) {
-      const uint32_t bytes = (uint32_t)min(kTileSlots, v.L - slot0) * C::kRowBytes;
-      mbar_expect_tx(&full_bar[s], bytes);
-      bulk_g2s(dst, v.Kl + (long long)slot0 * D, bytes, &full_bar[s]);
-    } else {
-      // whole 32-row boxes: rows past the lane's entries are other slots' bytes (zero fill past the end of the cache)
-      mbar_expect_tx(&full_bar[s], (uint32_t)C::kTileBytes);
-#pragma unroll
-      for (int h = 0; h < C::kVHalves; ++h)
-        tensor_g2s_2d(dst + h * C::kVHalfBytes, P.vmap, h * 64, (int)(v.lane * P.cap) + slot0, &full_bar[s]);
-    }
+    fill_view<T, D>(v, P, lane_local, kFlat ? 0 : (int)(blockIdx.x % P.n_splits), st[LS_LEN], st[LS_T], st[LS_FREE]);
+    if constexpr (kFlat) flat_piece(v, P, lane_local, (int)blockIdx.x);
+    v.new_k = sm.aux_k(0);
+    v.new_v = sm.aux_v(0);
+    return true;
   };
-  if (tid == kConsumerWarps * 32) {
-    for (int s = 0; s < NS; ++s) {
-      mbar_init(&full_bar[s], 1);
-      mbar_init(&empty_bar[s], kConsumerWarps);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    for (int x = 0; x < min(2 * n, NS); ++x) issue(x);
-  }
-  if (P.wait_at_start == 1) griddep_wait();
-  for (int c = tid; c < D; c += NT) {
-    aux[c] = k_in[c];
-    aux[D + c] = v_in[c];
-  }
-  if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
-    T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
-    T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
-    for (int c = tid; c < D; c += NT) { Kw[c] = k_in[c]; Vw[c] = v_in[c]; }
-  }
-  __syncthreads();
-
+  // The producer warp sets the ring's barriers up, says so on a named barrier without waiting there, and starts filling
+  // the ring at once; the consumer warps wait on that named barrier before their first look at the ring.
   if (warp == kConsumerWarps) {
-    if (lane_id == 0) {                                   // producer: keeps the ring full
-      for (int x = NS; x < 2 * n; ++x) {
-        mbar_wait(&empty_bar[x % NS], ((x / NS) - 1) & 1, P.status);
-        issue(x);
+    if (lane_id == 0) {
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(&sm.full_bar[s], 1);
+        mbar_init(&sm.empty_bar[s], kConsumerWarps);
       }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    asm volatile("bar.arrive 2, %0;" ::"n"(kThreads) : "memory");
+    if (lane_id == 0) {
+      // Producer: keeps the ring full across the CTA's pieces.  It reads lane state and cache rows only, none of which
+      // the kernel in front of this one writes, so it does not wait for that kernel (levels 0 and 1).
+      int it = 0;                                           // tiles issued so far, over all pieces
+      int lane_local = lane_lo;
+      if (lane_lo <= lane_hi) do {
+        LaneView<T> v;
+        if (!view_of(lane_local, v)) continue;
+        if (v.slot_end > v.slot_begin) {
+          // The epilogue kernel reads a and pos of these slots: pull their lines into L2 now.
+          const uint32_t bytes = (uint32_t)(((v.slot_end - v.slot_begin) * 4 + 15) & ~15);   // cap is a multiple of 4 slots
+          l2_prefetch(P.a + v.lane * P.cap + v.slot_begin, bytes);
+          l2_prefetch(P.pos + v.lane * P.cap + v.slot_begin, bytes);
+        }
+        for (int i = 0; i < v.n_tiles; ++i, ++it) {
+          const int s = it % kStages;
+          if (it >= kStages) mbar_wait(&sm.empty_bar[s], ((it / kStages) - 1) & 1, P.status);
+          const int slot0 = (v.tile_begin + i) * kTileSlots;
+          fill_stage<T, D, G>(sm.ring + (size_t)s * C::kStageBytes, v.Kl + (long long)slot0 * D, v.Vl + (long long)slot0 * D,
+                              min(kTileSlots, v.L - slot0), &sm.full_bar[s], P.vmap, (int)(v.lane * P.cap) + slot0);
+        }
+      } while (kFlat && ++lane_local <= lane_hi);
     }
   } else {
-    const int rg = lane_id / SC::LPR, l = lane_id % SC::LPR;
-    const int my_head = l / SC::LH, li = l % SC::LH;
-    float* lg = P.logits + (long long)lane_local * G * P.cap;
-    // the one (row, head) of every tile whose logit this thread parks in phase one and turns into a probability in two
-    const int my_row = warp * 8 + li * SC::RPP + rg;
-    float* my_lg = lg + (long long)my_head * P.cap;
-    float m_unit;
-    {
-      // ---- phase one: logits of the unit, exact maximum per head ----
-      SC sc;
-      sc.begin(q_in);
-      float m_run = -INFINITY;
-      for (int i = 0; i < n; ++i) {
-        const int s = i % NS;
-        mbar_wait(&full_bar[s], (i / NS) & 1, P.status);
-        T* tK = reinterpret_cast<T*>(ring + (size_t)s * C::kTileBytes);
-        const int slot0 = (v.tile_begin + i) * kTileSlots;
-        SC::patch_new_token(tK, nullptr, slot0, v.new_slot, v.new_k, v.new_v);
-        float sv[SC::PASSES];
-        bool valid[SC::PASSES];
-        sc.logits(tK, slot0, v.L, P.scale, sv, valid);
-        SC::park(sv, slot0, v.L, lg, P.cap, 0);
-#pragma unroll
-        for (int ps = 0; ps < SC::PASSES; ++ps) m_run = fmaxf(m_run, sv[ps]);
-        release_stage(&empty_bar[s]);
+    if (P.wait_at_start == 1) griddep_wait();             // before the first read of q, k, v
+    asm volatile("bar.sync 2, %0;" ::"n"(kThreads) : "memory");   // the ring's barriers exist
+    int it = 0;                                           // tiles consumed so far, over all pieces
+    int lane_local = lane_lo;
+    if (lane_lo <= lane_hi) do {
+      LaneView<T> v;
+      if (!view_of(lane_local, v)) continue;
+      const int b = v.b, hk = v.hk;
+      const T* q_in = reinterpret_cast<const T*>(P.q) + b * P.q_bs + (long long)hk * G * D;
+      const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+      const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+      // The new token's rows are kept in shared memory for the scan (the cache copy of that slot may still be in
+      // flight) and written to the cache by the CTA whose share owns the slot.  (The barrier at the end of the previous
+      // piece has every consumer warp done with the previous lane's rows.)
+      for (int c = tid; c < D; c += NC) {
+        sm.aux_k(0)[c] = k_in[c];
+        sm.aux_v(0)[c] = v_in[c];
       }
-      m_run = fmaxf(m_run, __shfl_xor_sync(0xffffffffu, m_run, 16));          // the other row group, same head
-      if (rg == 0 && li == 0) wmax[warp * G + my_head] = m_run;
-      group_sync<kConsumerWarps * 32>();
-      m_unit = wmax[my_head];
-#pragma unroll
-      for (int w = 1; w < kConsumerWarps; ++w) m_unit = fmaxf(m_unit, wmax[w * G + my_head]);
-    }
-    // ---- phase two: probabilities against the unit's maximum, P.V ----
-    SC sc;
-    sc.begin_pv();
-    const float m_use = m_unit == -INFINITY ? 0.f : m_unit;
-    float l_mine = 0.f;
-    float s_next = 0.f;
-    {
-      const int slot = v.tile_begin * kTileSlots + my_row;
-      if (n > 0 && slot < v.L) s_next = my_lg[slot];
-    }
-    for (int i = 0; i < n; ++i) {
-      const int x = n + i, s = x % NS;
-      const int slot0 = (v.tile_begin + i) * kTileSlots;
-      const float s_mine = s_next;
-      const bool ok = slot0 + my_row < v.L;
-      if (i + 1 < n && slot0 + kTileSlots + my_row < v.L) s_next = my_lg[slot0 + kTileSlots + my_row];   // next tile's, early
-      const float p = ok ? fast_exp2((s_mine - m_use) * kLog2e) : 0.f;
-      l_mine += p;
-      mbar_wait(&full_bar[s], (x / NS) & 1, P.status);
-      T* tV = reinterpret_cast<T*>(ring + (size_t)s * C::kTileBytes);
-      SC::patch_new_token(nullptr, tV, slot0, v.new_slot, v.new_k, v.new_v);
-      sc.pv_mma(tV, p, slot0, v.L);
-      release_stage(&empty_bar[s]);
-    }
-    // every warp is done with the ring before the partials go over it
-    group_sync<kConsumerWarps * 32>();
-    sc.end_pv(warp_part, m_unit, l_mine);
+      if (v.new_slot >= v.slot_begin && v.new_slot < v.slot_end) {
+        T* Kw = const_cast<T*>(v.Kl) + (long long)v.new_slot * D;
+        T* Vw = const_cast<T*>(v.Vl) + (long long)v.new_slot * D;
+        for (int c = tid; c < D; c += NC) { Kw[c] = k_in[c]; Vw[c] = v_in[c]; }
+      }
+      group_sync<NC>();
+      Scanner<T, D, G> sc;
+      sc.begin(q_in);
+      float* lg = P.logits + (long long)lane_local * G * P.cap;
+      for (int i = 0; i < v.n_tiles; ++i, ++it) {
+        const int s = it % kStages;
+        mbar_wait(&sm.full_bar[s], (it / kStages) & 1, P.status);
+        T* tK = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes);
+        T* tV = reinterpret_cast<T*>(sm.ring + (size_t)s * C::kStageBytes + C::kTileBytes);
+        sc.tile(tK, tV, (v.tile_begin + i) * kTileSlots, v.L, v.new_slot, v.new_k, v.new_v, P.scale, lg, P.cap, 0);
+        release_stage(&sm.empty_bar[s]);
+      }
+      sc.end(sm.warp_part);
+      group_sync<NC>();
+      combine_warps<D, G, NC>(sm.warp_part, P.part + ((long long)lane_local * P.n_splits + v.split) * G * (D + 2));
+      // Level 0: the wait comes BEFORE the unit reports.  The lane epilogues behind this scan start on the reports
+      // alone, and the scan after them (which reuses the scratch set of the lane epilogues in front of this scan) is
+      // released by those epilogues: with the report behind the wait, "the next scan runs" implies "every unit here has
+      // seen the previous lane epilogues complete", so no two grids ever touch one scratch set at a time.
+      if (!P.wait_at_start) griddep_wait();
+      // the barrier orders every consumer's stores (partial, logits, cache row) before the report, and ends the piece:
+      // the next piece may overwrite the token rows and the warp partials
+      group_sync<NC>();
+      if (P.ticket != nullptr && tid == 0) {
+        // tell the lane's epilogue CTA (already resident in the next kernel, or not yet) that this unit is in scratch
+        __threadfence();                                 // release
+        atomicAdd(&P.ticket[lane_local], 1u);
+      }
+    } while (kFlat && ++lane_local <= lane_hi);
   }
-  __syncthreads();
-  combine_warps<D, G, NT>(warp_part, P.part + ((long long)lane_local * P.n_splits + split) * G * (D + 2));
-  if (!P.wait_at_start) griddep_wait();                   // level 0: wait before reporting (see scan_body)
-  if (P.ticket != nullptr) {
-    __syncthreads();
-    if (tid == 0) {
-      __threadfence();
-      atomicAdd(&P.ticket[lane_local], 1u);
-    }
-  }
+  // every CTA, with work or without, ends behind the kernel in front of it: the completion of this grid implies that
+  // kernel's completion
+  if (P.wait_at_start != 2) griddep_wait();
 }
 
-template <typename T, int D, int G>
+template <typename T, int D, int G, bool kFlat>
 __global__ void __launch_bounds__(kThreads) scan_kernel(const __grid_constant__ StepParams P) {
-  scan_body<T, D, G>(P);
+  if constexpr (kFlat) scan_body<T, D, G, true>(P);
+  else scan_body_even<T, D, G>(P);
 }
-// The scan of the instantiations with the tensor-core P.V half (Cfg::kMmaPV): two phases, six CTAs per SM.
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kThreads, 6) scan_kernel_mma(const __grid_constant__ StepParams P) {
-  scan_body_two_phase<T, D, G>(P);
+// The same scan for the instantiations with the tensor-core P.V half (Cfg::kMmaPV), held to the registers of four CTAs
+// per SM (a second argument to __launch_bounds__ changes the compiler's choices even when it is 1, hence two entries).
+template <typename T, int D, int G, bool kFlat>
+__global__ void __launch_bounds__(kThreads, 4) scan_kernel_mma(const __grid_constant__ StepParams P) {
+  if constexpr (kFlat) scan_body<T, D, G, true>(P);
+  else scan_body_even<T, D, G>(P);
 }
 // the entry that a configuration's scan is launched through
 template <typename T, int D, int G>
-inline auto scan_entry() -> void (*)(const StepParams) {
-  if constexpr (Cfg<T, D, G>::kMmaPV) return scan_kernel_mma<T, D, G>;
-  else return scan_kernel<T, D, G>;
+inline auto scan_entry(bool flat) -> void (*)(const StepParams) {
+  if constexpr (Cfg<T, D, G>::kMmaPV) return flat ? scan_kernel_mma<T, D, G, true> : scan_kernel_mma<T, D, G, false>;
+  else return flat ? scan_kernel<T, D, G, true> : scan_kernel<T, D, G, false>;
 }
 // dynamic shared memory of that entry
 template <typename T, int D, int G>
-constexpr int scan_smem_bytes() {
-  if constexpr (Cfg<T, D, G>::kMmaPV) return TwoPhase<T, D, G>::kSmemBytes;
-  else return Cfg<T, D, G>::kFixedBytes;
-}
+constexpr int scan_smem_bytes() { return Cfg<T, D, G>::kScanBytes; }
 
 constexpr int kEpilogueThreads = 256;
 constexpr int kEpilogueThreadsWide = 512;     // one or two query heads only (registers: two CTAs per SM)
@@ -1525,6 +1546,8 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
   const bool active = !(P.seq_lens != nullptr && P.tok_idx >= P.seq_lens[b]);   // else: sequence already consumed
   // The lane's state words were last written by an earlier lane epilogue of the same layer, which is complete (the
   // scan in front of this kernel did not finish before everything older had finished): read them before waiting.
+  // (A step of a blocked prompt tail follows the previous step of the same lanes: nothing is read before that one is done.)
+  if (P.block_tokens > 0) griddep_wait();
   LaneView<T> v;
   const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
   if (active) {
@@ -1533,6 +1556,16 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
     v.tail = st[LS_TAIL];
     v.new_k = v.Kl + (long long)v.new_slot * D;          // the scan kernel has stored this step's token in the cache
     v.new_v = v.Vl + (long long)v.new_slot * D;
+    if (P.block_tokens > 0) {
+      // ... in a blocked tail no scan runs per token: the token's rows go into its slot here.  (Thread c writes channel c
+      // and is the only one to read it back from the cache in this kernel.)
+      const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)hk * D;
+      const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)hk * D;
+      for (int c = threadIdx.x; c < D; c += NT) {
+        const_cast<T*>(v.new_k)[c] = k_in[c];
+        const_cast<T*>(v.new_v)[c] = v_in[c];
+      }
+    }
   }
   // A lane of at most E * NT entries is finished by lane_epilogue_in_registers, if the launch gave the CTA room to stage
   // the lane's scores and positions (P.ep_stage_slots entries each of dynamic shared memory).  They were last written
@@ -1566,9 +1599,11 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
   } else {
     if (threadIdx.x == 0) {
       volatile uint32_t* tk = P.ticket + lane_local;
+      int first_cta, n_pieces;
+      lane_pieces(P, lane_local, first_cta, n_pieces);
       int ok = 0;
       for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (*tk >= (uint32_t)P.n_splits) { ok = 1; break; }
+        if (*tk >= (uint32_t)n_pieces) { ok = 1; break; }
         __nanosleep(100);
       }
       if (!ok) atomicOr(P.status, kStatusWaitTimeout);
@@ -1584,6 +1619,8 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
   }
   if (in_regs) {
     if constexpr (E > 0) lane_epilogue_in_registers<T, D, G, NT, E>(P, v, ep, a_s, pos_s);
+  } else if (P.block_tokens > 0) {
+    if (threadIdx.x == 0) atomicOr(P.status, kStatusBadLink);   // the host sends blocked tails only where the lane fits
   } else {
     lane_epilogue_from_scratch<T, D, G, NT>(P, v, ep);
   }
@@ -1593,8 +1630,11 @@ __device__ __forceinline__ void lane_epilogue_body(const StepParams& P) {
   }
 }
 
+// One query head: held to 64 registers, i.e. 1024 threads per SM, so that a layer of up to 4 x 148 lanes is one wave of
+// CTAs -- the kernel behind this one can only be set up once every CTA here has started, and a second wave would start
+// only when the first has finished.
 template <typename T, int D, int G, int NT>
-__global__ void __launch_bounds__(NT) lane_epilogue_kernel(const StepParams P) {
+__global__ void __launch_bounds__(NT, G == 1 ? 1024 / NT : 1) lane_epilogue_kernel(const StepParams P) {
   lane_epilogue_body<T, D, G, NT>(P);
 }
 // Four query heads, a layer of at most two lanes per SM: 384 threads per lane, held to the registers of two CTAs per SM.

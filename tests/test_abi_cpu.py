@@ -58,7 +58,7 @@ GOOD = dict(n_layers=1, batch=1, n_q_heads=4, n_kv_heads=4, head_dim=64, budget=
     ({"n_splits": 65}, "n_splits"),
     ({"scale": -1.0}, "scale"),
     ({"n_layers": 0}, "n_layers"),
-    ({"schedule": 3}, "schedule"),
+    ({"schedule": 4}, "schedule"),
 ])
 def test_config_validation(lib, change, fragment):
     cfg = binding.make_config(**{**GOOD, **change})

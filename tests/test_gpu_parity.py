@@ -44,7 +44,7 @@ def test_tiny_config_every_step():
     ("bf16", 128, 2, 2, 8, 8, 0, 0, 40),       # window == budget: a single candidate
     ("bf16", 128, 2, 2, 200, 32, 0, 64, 260),  # maximum split count
 ])
-@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER])
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_SPLIT, binding.WKV_SCHEDULE_CLUSTER, binding.WKV_SCHEDULE_FLAT])
 def test_shapes_every_step(dtype, d, hq, hkv, m, W, S, splits, steps, schedule):
     if schedule == binding.WKV_SCHEDULE_CLUSTER and splits not in (0, 1, 2, 4, 8, 16):
         pytest.skip("a cluster needs a power-of-two split count")
@@ -56,13 +56,39 @@ def test_shapes_every_step(dtype, d, hq, hkv, m, W, S, splits, steps, schedule):
     p.close()
 
 
+@pytest.mark.parametrize("dtype,hq,hkv,m,splits", [("bf16", 32, 32, 70, 0), ("bf16", 32, 8, 100, 0), ("f32", 16, 16, 40, 0),
+                                                    ("bf16", 8, 8, 300, 3)])
+def test_flat_deal_runs_of_tiles_across_lanes(dtype, hq, hkv, m, splits):
+    """The flat deal with runs that do not line up with the lanes: with splits = 0 the scan takes one wave of CTAs, so
+    with far more lanes than CTAs a CTA holds a piece of several lanes (the end of one, whole lanes, the start of the
+    next), and with few lanes a lane is cut into pieces of unequal size; ragged prompts leave some lanes shorter than
+    their tile count.  Compared with the oracle every step, and with the even deal at the end."""
+    batch = 40 if splits == 0 else 3
+    wl = small(batch=batch, hq=hq, hkv=hkv, d=128 if dtype == "bf16" else 64, dtype=dtype, m=m, W=6, S=1,
+               rank=16 if dtype == "bf16" else 0)
+    lens = [m + 30 - (7 * b) % 50 for b in range(batch)]
+    p = Parity(wl, seed=23, sample=24, n_splits=splits, schedule=binding.WKV_SCHEDULE_FLAT, ragged=lens)
+    q = Parity(wl, seed=23, sample=24, schedule=binding.WKV_SCHEDULE_SPLIT, ragged=lens)
+    p.prefill(m + 30, chunk=40)
+    q.prefill(m + 30, chunk=40, compare=False)
+    p.decode(12)
+    p.decode(4, layers_entry=True)
+    q.decode(16)
+    p.compare_state()
+    for ln in p.lanes:
+        s0, s1 = p.ctx.wkv_export_state(*ln), q.ctx.wkv_export_state(*ln)
+        assert torch.equal(s0["pos"], s1["pos"]) and torch.equal(s0["a"], s1["a"]) and torch.equal(s0["V"], s1["V"])
+    p.close()
+    q.close()
+
+
 def test_split_count_does_not_change_results():
     """The same stream under 1, 2, 5 and 16 CTAs per lane: identical eviction sequences and bit-identical a."""
     wl = small(batch=2, d=128, dtype="bf16", m=150, W=8, rank=16)
     states = []
-    for splits, schedule in ((1, 1), (2, 2), (5, 1), (16, 2), (8, 1), (4, 0)):
+    for splits, schedule in ((1, 1), (2, 2), (5, 1), (16, 2), (8, 1), (4, 0), (3, 3), (0, 3)):
         p = Parity(wl, seed=5, n_splits=splits, schedule=schedule)
-        assert p.ctx.wkv_splits() == splits
+        assert schedule == 3 or p.ctx.wkv_splits() == splits
         p.decode(230)
         states.append([p.ctx.wkv_export_state(*ln) for ln in p.lanes])
         p.close()
