@@ -841,7 +841,7 @@ static cudaError_t launch_block_kernels(int which, const wkv::BlockParams& BP, i
     if (e != cudaSuccess) return e;
     block_pv_kernel<T, D, R><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
   } else {
-    block_out_kernel<T, D><<<lanes, D, 0, s>>>(BP);
+    block_out_kernel<T, D><<<lanes * BP.block_tokens * BP.group, D, 0, s>>>(BP);
   }
   return cudaGetLastError();
 }

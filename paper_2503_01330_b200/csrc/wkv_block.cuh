@@ -14,9 +14,9 @@
 //                         in streaming.  It writes the token's rows into the freed slot, leaves the token's probabilities
 //                         in a table (slot order) and records every value row that it changes as it was before.
 //   block_pv_kernel       one sweep over the V rows as they are after the block: sum_s P[token][s] * V[s] for all B tokens.
-//   block_out_kernel      per lane: adds the units' partial sums and, for every recorded change, P[token][s] * (row as it
-//                         was when the token attended - row as it is now) for the tokens in front of the change: the
-//                         attention output uses V before the step's own merge, as in Algorithm 1.
+//   block_out_kernel      per query row of the block: adds the units' partial sums and, for every recorded change,
+//                         P[token][s] * (row as it was when the token attended - row as it is now) for the tokens in
+//                         front of the change: the attention output uses V before the step's own merge, as in Algorithm 1.
 //
 // Everything that decides a removal (logits, probabilities, accumulated scores, pick, merged values) is computed by the
 // same code as in the streamed step, in the same order, so the state after the block is bit-identical; the outputs
@@ -275,37 +275,33 @@ __global__ void __launch_bounds__(kThreads) block_pv_kernel(const BlockParams P)
 // ------------------------------------------------------------------------------------------------
 template <typename T, int D>
 __global__ void __launch_bounds__(D) block_out_kernel(const BlockParams P) {
+  // one CTA per (lane, query row of the block), one thread per channel
   const int c = threadIdx.x;
-  const int lane_local = blockIdx.x;
+  const int R = P.block_tokens * P.group;
+  const int lane_local = blockIdx.x / R, row = blockIdx.x % R;
+  const int tok = row / P.group, g = row % P.group;
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
   const int n_act = block_active_tokens(P, b);
-  if (n_act == 0 || P.out == nullptr) return;
+  if (tok >= n_act || P.out == nullptr) return;
   const long long lane = (long long)P.lane0 + lane_local;
-  const int R = P.block_tokens * P.group;
   const T* Vl = reinterpret_cast<const T*>(P.Vc) + lane * (long long)P.cap * D;
-  const float* pt = P.ptab + (long long)lane_local * R * P.cap;
+  const float* pt = P.ptab + ((long long)lane_local * R + row) * P.cap;
   const int32_t* rs = P.rec_slot + (long long)lane_local * P.block_tokens * 2;
   const float* rr = P.rec_rows + (long long)lane_local * P.block_tokens * 2 * D;
-  for (int tok = 0; tok < n_act; ++tok) {
-    for (int g = 0; g < P.group; ++g) {
-      const int row = tok * P.group + g;
-      float o = 0.f;
-      for (int u = 0; u < P.n_units; ++u) o += P.opart[(((long long)lane_local * P.n_units + u) * R + row) * D + c];
-      // A record made at step k (k >= tok) holds the row of its slot as token tok attended it, unless an earlier record
-      // (tok <= k' < k) of the same slot does: the first record of a slot at or after the token's own step counts.
-      for (int k = 2 * tok; k < 2 * n_act; ++k) {
-        const int slot = rs[k];
-        if (slot < 0) continue;
-        bool first = true;
-        for (int k2 = 2 * tok; k2 < k; ++k2) first = first && rs[k2] != slot;
-        if (!first) continue;
-        const float p = pt[(long long)row * P.cap + slot];
-        o += p * (rr[(long long)k * D + c] - to_f32(Vl[(long long)slot * D + c]));
-      }
-      T* dst = reinterpret_cast<T*>(P.out) + b * P.out_bs + (long long)(P.tok0 + tok) * P.out_ts + ((long long)hk * P.group + g) * D;
-      dst[c] = from_f32<T>(o);
-    }
+  float o = 0.f;
+  for (int u = 0; u < P.n_units; ++u) o += P.opart[(((long long)lane_local * P.n_units + u) * R + row) * D + c];
+  // A record made at step k (k >= tok) holds the row of its slot as token tok attended it, unless an earlier record
+  // (tok <= k' < k) of the same slot does: the first record of a slot at or after the token's own step counts.
+  for (int k = 2 * tok; k < 2 * n_act; ++k) {
+    const int slot = rs[k];
+    if (slot < 0) continue;
+    bool first = true;
+    for (int k2 = 2 * tok; k2 < k; ++k2) first = first && rs[k2] != slot;
+    if (!first) continue;
+    o += pt[slot] * (rr[(long long)k * D + c] - to_f32(Vl[(long long)slot * D + c]));
   }
+  T* dst = reinterpret_cast<T*>(P.out) + b * P.out_bs + (long long)(P.tok0 + tok) * P.out_ts + ((long long)hk * P.group + g) * D;
+  dst[c] = from_f32<T>(o);
 }
 
 }  // namespace wkv
