@@ -271,3 +271,62 @@ def test_bulk_prefill_eviction_ablation_and_stream_switch():
     p.decode(5)
     p.compare_state()
     p.close()
+
+
+@pytest.mark.parametrize("dtype,d,hq,hkv,m,W,S,T,chunk", [
+    ("bf16", 128, 4, 4, 70, 9, 0, 150, 150),     # one head per key: blocks of 8 tokens, the smallest window that allows them; last block of 8 full
+    ("bf16", 128, 4, 4, 70, 12, 2, 149, 149),    # ... last block of 7 tokens, sinks
+    ("f32", 64, 2, 2, 33, 10, 0, 100, 29),       # fp32 rows; the prompt in chunks that end inside blocks (blocks restart per call)
+    ("bf16", 64, 8, 4, 100, 16, 1, 171, 171),    # two heads per key: blocks of 4
+    ("bf16", 128, 8, 2, 95, 16, 0, 170, 60),     # four heads per key: blocks of 2, chunked
+    ("f32", 128, 4, 1, 40, 6, 0, 90, 90),        # four heads per key on fp32 rows
+])
+def test_blocked_prompt_tail_every_token(dtype, d, hq, hkv, m, W, S, T, chunk):
+    """The tokens of a prompt beyond the budget, in blocks that share two sweeps of the cache (two-kernel schedule forced,
+    so that small shapes take that path): removed positions bit for bit and outputs within tolerance for every token,
+    state afterwards, then decode.  Ragged lengths end sequences inside a block and leave one sequence below the budget."""
+    wl = small(batch=4, hq=hq, hkv=hkv, d=d, dtype=dtype, m=m, W=W, S=S, rank=16 if dtype == "bf16" else 0)
+    lens = [T, T - 3, m - 5, m + 11]
+    p = Parity(wl, seed=70 + m, ragged=lens, schedule=binding.WKV_SCHEDULE_SPLIT)
+    before = p.ctx.wkv_launch_count()
+    p.prefill(T, chunk=chunk, bulk=True)
+    launches = p.ctx.wkv_launch_count() - before
+    # what the blocked path launches: per call the dense kernel (if the layer is still below the budget), then per block
+    # one logit sweep, one lane epilogue per token, the value sweep and the output kernel
+    B, expected, consumed = 8 // (hq // hkv), 0, 0
+    for t0 in range(0, T, chunk):
+        tc = min(chunk, T - t0)
+        n0 = min(tc, max(0, m - consumed))
+        tail = tc - n0
+        expected += (1 if n0 > 0 else 0) + (2 * tail if tail < 2 else 3 * ((tail + B - 1) // B) + tail)
+        consumed += tc
+    assert launches == expected, "the tail did not go through the blocked path"
+    p.compare_state()
+    p.decode(m // 2 + 3)
+    p.compare_state()
+    p.close()
+
+
+def test_blocked_prompt_tail_without_outputs_and_all_layers():
+    """Outputs not requested (the value sweep is skipped) and the all-layers call: same state as the streamed prompt."""
+    wl = small(layers=3, batch=2, hq=4, hkv=4, d=128, dtype="bf16", m=60, W=10, S=1, rank=16)
+    st = TokenStream(wl, 33, "cuda:0")
+    Q, K, V = st.tokens(0, 140)
+    lens = torch.tensor([140, 97], dtype=torch.int32, device="cuda:0")
+    states = []
+    for mode in ("streamed", "blocked", "blocked_layers"):
+        ctx = binding.Context(wl.n_layers, wl.batch, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.budget, wl.window,
+                              wl.sink, binding.WKV_BF16, schedule=binding.WKV_SCHEDULE_SPLIT)
+        if mode == "blocked_layers":
+            ctx.wkv_prefill_bulk_layers(Q, K, V, lens)
+        else:
+            for layer in range(wl.n_layers):
+                (ctx.wkv_prefill if mode == "streamed" else ctx.wkv_prefill_bulk)(layer, Q[layer], K[layer], V[layer], lens)
+        assert ctx.wkv_status() == 0
+        states.append([ctx.wkv_export_state(l, b, h) for l in range(wl.n_layers) for b in range(wl.batch) for h in range(wl.n_kv_heads)])
+        ctx.close()
+    for other in states[1:]:
+        for s0, s1 in zip(states[0], other):
+            assert s0["len"] == s1["len"] and s0["tokens"] == s1["tokens"]
+            assert torch.equal(s0["pos"], s1["pos"]) and torch.equal(s0["a"], s1["a"])
+            assert torch.equal(s0["K"], s1["K"]) and torch.equal(s0["V"], s1["V"])
