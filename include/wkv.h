@@ -172,18 +172,22 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
                 int32_t T_max, void* out, int32_t* evicted_pos);
 
 /* The same prompt, same arguments and same results as wkv_prefill, with the uncompressed part of the prompt done as
- * one dense problem per lane.  Algorithm 1 compresses only once a lane holds more than `budget` entries; until then
+ * one dense problem per lane and the rest in blocks of tokens that share two sweeps of the cache.  Algorithm 1 compresses only once a lane holds more than `budget` entries; until then
  * its iterations are causal attention (Background section) plus the running sums of the attention columns.  The
  * library keeps, per layer, an upper bound on the tokens any lane has consumed since wkv_create / wkv_reset (calls of
  * every kind count; an imported lane counts as its token count if nothing of it was removed, as full otherwise).
  * While that bound is below the budget, the first min(T_max, budget - bound) tokens of the call go through one kernel
  * for all lanes of the layer -- on top of what each lane already holds, whose keys and values it reads from the cache
  * -- with every logit, probability and accumulated score computed by the arithmetic of the streamed step and the
- * scores added in the order of the tokens; the remaining tokens are streamed as in wkv_prefill.  So a prompt may come
- * in one call or in chunks.  K, positions, accumulated scores and removed positions are bit-identical to
+ * scores added in the order of the tokens.  The remaining tokens are taken 8 / group at a time where window > 8 / group
+ * and a lane's entries fit the register form of the per-lane kernel (budget + 1 <= 4352 for one query head per key):
+ * one sweep over the key rows gives the logits of the whole block, the per-token step of Algorithm 1 (probabilities,
+ * score fold, pick, merge) then runs on them token after token exactly as when streaming, and one sweep over the value
+ * rows gives all outputs; elsewhere they are streamed as in wkv_prefill.  So a prompt may come in one call or in chunks.  K, positions, accumulated scores and removed positions are bit-identical to
  * wkv_prefill's; outputs and merged values agree within rounding.
- * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider and
- * keeps them until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
+ * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider, the first
+ * blocked tail about 64 * lanes_per_layer * (budget + 1) bytes more (if the provider refuses those, the tail is streamed);
+ * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos);
 
@@ -238,7 +242,8 @@ int wkv_selftest_wait_timeout(wkv_ctx* ctx);
 /* Number of kernels this context has launched so far, and bytes it obtained from the provider. */
 int64_t wkv_launch_count(const wkv_ctx* ctx);
 int64_t wkv_device_bytes(const wkv_ctx* ctx);
-/* The number of CTAs per lane the context uses (after resolving n_splits = 0). */
+/* The number of CTAs per lane the context uses (after resolving n_splits = 0); under the flat deal, where runs of tiles
+ * cross lane boundaries, the largest number of CTAs that can share one lane. */
 int32_t wkv_splits(const wkv_ctx* ctx);
 
 const char* wkv_strerror(int code);

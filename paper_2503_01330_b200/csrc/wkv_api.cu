@@ -826,6 +826,27 @@ static int block_tokens_of(const wkv_ctx* c, int lanes) {
   return B;
 }
 
+// Scratch of the blocked tail for `lanes` lanes, taken from the provider on first use (or when more lanes are needed).
+// false: the provider refused; the caller then streams the tokens instead -- nothing has been launched for them yet.
+static bool block_scratch(wkv_ctx* c, int lanes, int B) {
+  if (c->blk_logits != nullptr && c->blk_lanes >= lanes) return true;
+  const size_t cap = c->cap, D = c->cfg.head_dim;
+  const int R = 8;
+  const int tiles = (c->cfg.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
+  int units = (int)((6LL * c->sm_count + lanes - 1) / lanes);
+  units = std::max(1, std::min({units, 16, std::max(1, tiles / 8)}));
+  int rc = take(c, &c->blk_logits, (size_t)lanes * R * cap * 4);
+  if (rc == WKV_OK) rc = take(c, &c->blk_lgx, (size_t)lanes * R * B * 4 + 256);
+  if (rc == WKV_OK) rc = take(c, &c->blk_ptab, (size_t)lanes * R * cap * 4 + 256);   // the last tile of the last row is read whole
+  if (rc == WKV_OK) rc = take(c, &c->blk_opart, (size_t)lanes * units * R * D * 4);
+  if (rc == WKV_OK) rc = take(c, &c->blk_rec_rows, (size_t)lanes * 2 * B * D * 4);
+  if (rc == WKV_OK) rc = take(c, &c->blk_rec_slot, (size_t)lanes * 2 * B * 4);
+  if (rc != WKV_OK) { c->blk_logits = nullptr; c->blk_lanes = 0; return false; }
+  c->blk_lanes = lanes;
+  c->blk_units = units;
+  return true;
+}
+
 template <typename T, int D>
 static cudaError_t launch_block_kernels(int which, const wkv::BlockParams& BP, int lanes, cudaStream_t s) {
   using namespace wkv;
@@ -877,21 +898,7 @@ static int blocked_tokens(wkv_ctx* c, long long lane0, int lanes, int B, const v
   const long long D = c->cfg.head_dim, Hq = c->cfg.n_q_heads, Hk = c->cfg.n_kv_heads;
   const int R = 8, G = c->group;
   const size_t cap = c->cap;
-  if (c->blk_logits == nullptr || c->blk_lanes < lanes) {
-    const int tiles = (c->cfg.budget + 1 + wkv::kTileSlots - 1) / wkv::kTileSlots;
-    int units = (int)((6LL * c->sm_count + lanes - 1) / lanes);
-    units = std::max(1, std::min({units, 16, std::max(1, tiles / 8)}));
-    int rc = WKV_OK;
-    if (rc == WKV_OK) rc = take(c, &c->blk_logits, (size_t)lanes * R * cap * 4);
-    if (rc == WKV_OK) rc = take(c, &c->blk_lgx, (size_t)lanes * R * B * 4 + 256);
-    if (rc == WKV_OK) rc = take(c, &c->blk_ptab, (size_t)lanes * R * cap * 4 + 256);   // the last tile of the last row is read whole
-    if (rc == WKV_OK) rc = take(c, &c->blk_opart, (size_t)lanes * units * R * D * 4);
-    if (rc == WKV_OK) rc = take(c, &c->blk_rec_rows, (size_t)lanes * 2 * B * D * 4);
-    if (rc == WKV_OK) rc = take(c, &c->blk_rec_slot, (size_t)lanes * 2 * B * 4);
-    if (rc != WKV_OK) { c->blk_logits = nullptr; c->blk_lanes = 0; return rc; }
-    c->blk_lanes = lanes;
-    c->blk_units = units;
-  }
+  if (!block_scratch(c, lanes, B)) return WKV_ERR_ALLOC;
   wkv::BlockParams BP;
   std::memset(&BP, 0, sizeof(BP));
   BP.Kc = c->Kc; BP.Vc = c->Vc; BP.lane_state = c->lane_state;
@@ -1043,7 +1050,7 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
   }
   // the rest: in blocks of tokens that share two sweeps of the cache where the configuration allows, else token by token
   const int B = block_tokens_of(c, c->lanes_per_layer);
-  if (B > 0 && T_max - n0 >= 2) {
+  if (B > 0 && T_max - n0 >= 2 && block_scratch(c, c->lanes_per_layer, B)) {
     c->tokens_hi[layer] += T_max - n0;
     return blocked_tokens(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, B, Q, K, V, seq_lens, n0, T_max, out,
                           evicted_pos);
@@ -1096,14 +1103,14 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
     // when a layer alone is small, else layer after layer (the layers' prompts are independent)
     const int B_all = c->fused_ok ? block_tokens_of(c, (int)c->lanes_total) : 0;
     const int B_one = block_tokens_of(c, c->lanes_per_layer);
-    if (B_all > 0) {
+    if (B_all > 0 && block_scratch(c, (int)c->lanes_total, B_all)) {
       if (seq_lens != nullptr)
         for (int l = 0; l < L; ++l)
           WKV_CUDA(c, cudaMemcpyAsync(c->fused_seq_lens + (size_t)l * B, seq_lens, (size_t)B * 4, cudaMemcpyDeviceToDevice, c->stream));
       return blocked_tokens(c, 0, (int)c->lanes_total, B_all, Q, K, V, seq_lens != nullptr ? c->fused_seq_lens : nullptr, n0, T_max,
                             out, evicted_pos);
     }
-    if (B_one > 0) {
+    if (B_one > 0 && block_scratch(c, c->lanes_per_layer, B_one)) {
       for (int l = 0; l < L; ++l) {
         rc = blocked_tokens(c, (long long)l * c->lanes_per_layer, c->lanes_per_layer, B_one, (const char*)Q + l * q_layer,
                             (const char*)K + l * kv_layer, (const char*)V + l * kv_layer, seq_lens, n0, T_max,

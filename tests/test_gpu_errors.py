@@ -135,3 +135,40 @@ def test_inconsistent_bookkeeping_is_reported_as_state_error():
     assert L.wkv_strerror(binding.WKV_ERR_STATE).decode().startswith("inconsistent")
     L.wkv_destroy(h)                                         # no further step runs on the damaged lanes
     assert not p.live
+
+
+def test_provider_refusing_the_blocked_tail_scratch_falls_back_to_streaming():
+    """The blocked prompt tail takes its scratch on first use, after the dense part of the prompt has been launched.  A
+    refusal there must not lose the prompt: the tail is streamed token by token instead, with the same results."""
+    L = binding.lib()
+    g = torch.Generator(device="cuda:0").manual_seed(11)
+    Q, K, V = (torch.randn(2, 120, 4, 64, generator=g, device="cuda:0").to(torch.bfloat16) for _ in range(3))
+    dp = lambda t: C.c_void_p(t.data_ptr())
+    states = []
+    for refuse in (False, True):
+        p = Provider()
+        cfg = p.config(n_layers=1, budget=64, window=12, schedule=binding.WKV_SCHEDULE_SPLIT)
+        h = C.c_void_p()
+        assert L.wkv_create(C.byref(cfg), C.byref(h)) == binding.WKV_OK
+        n_create = p.calls
+        if refuse:
+            p.fail_at = {n_create + 1}                      # request n_create is the dense phase's scratch, the next one the tail's
+        launches = L.wkv_launch_count(h)
+        assert L.wkv_prefill_bulk(h, 0, dp(Q), dp(K), dp(V), None, 120, None, None) == binding.WKV_OK
+        launches = L.wkv_launch_count(h) - launches
+        # 64 tokens dense, 56 in blocks of 8 (one sweep + 8 lane epilogues each) -- or streamed, two launches per token
+        assert launches == (1 + 56 * 2 if refuse else 1 + 7 * 9) and p.calls == (n_create + 2 if refuse else n_create + 7)
+        assert L.wkv_status(h) == binding.WKV_OK
+        pos = torch.empty(64, dtype=torch.int32)
+        a = torch.empty(64)
+        n = C.c_int32()
+        lane_states = []
+        for b in range(2):
+            for hd in range(4):
+                assert L.wkv_export_state(h, 0, b, hd, C.byref(n), None, dp(pos), dp(a), None, None) == binding.WKV_OK
+                lane_states.append((n.value, pos.clone(), a.clone()))
+        states.append(lane_states)
+        L.wkv_destroy(h)
+        assert not p.live
+    for (n0, p0, a0), (n1, p1, a1) in zip(*states):
+        assert n0 == n1 == 64 and torch.equal(p0, p1) and torch.equal(a0, a1)
