@@ -67,7 +67,7 @@ def test_llama7b_b8_full_prompt_length():
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("name,n_sample,decode", [("serving_b16", 6, 16), ("gqa_b32", 4, 16)])
+@pytest.mark.parametrize("name,n_sample,decode", [("serving_b16", 12, 16), ("gqa_b32", 8, 16)])
 def test_serving_and_gqa_full_prompt_lengths(name, n_sample, decode):
     """The two largest configurations with their whole prompts (16384 tokens with per-sequence lengths drawn from
     8192..16384, and 32768 tokens), in chunks of 256 tokens for all layers at once, then decode; sampled lanes against
