@@ -192,3 +192,61 @@ class Parity:
     def close(self):
         self.ctx.close()
         self.ref.close()
+
+
+def check_all_lanes(ctx, wl, tokens_per_seq, evicted=None):
+    """Properties of Algorithm 1's bookkeeping that hold at any size, checked on EVERY lane of the context at once, on the
+    device arrays themselves (the context's memory comes from this process's provider, in the order the library asks for
+    it: K, V, a, pos, next, prev, lane state).  tokens_per_seq [batch]: tokens each sequence has consumed.
+    evicted [n_layers, batch, n_kv_heads] (optional): the removed positions of the last step."""
+    bufs = list(ctx._bufs.values())
+    lanes, m, W, S = wl.lanes, wl.budget, wl.window, wl.sink
+    cap = (m + 1 + 3) // 4 * 4
+    a = bufs[2].view(torch.float32)[:lanes * cap].view(lanes, cap)
+    pos, nxt, prv = (bufs[i].view(torch.int32)[:lanes * cap].view(lanes, cap) for i in (3, 4, 5))
+    st = bufs[6].view(torch.int32)[:lanes * 8].view(lanes, 8)
+    dev = a.device
+    t = torch.as_tensor(tokens_per_seq, dtype=torch.int32, device=dev).repeat_interleave(wl.n_kv_heads).repeat(wl.n_layers)  # [lanes]
+    length, tok, head, tail, free = (st[:, i] for i in range(5))
+    assert torch.equal(tok, t), "tokens consumed"
+    assert torch.equal(length, torch.minimum(t, torch.full_like(t, m))), "entries held = min(tokens, budget)"
+    used = pos[:, :m + 1] >= 0
+    assert torch.equal(used.sum(1).to(torch.int32), length), "occupied slots = entries held"
+    p64 = pos[:, :m + 1].to(torch.int64)
+    # positions are distinct and below the token count
+    srt = torch.where(used, p64, torch.full_like(p64, -1)).sort(dim=1).values
+    dup = (srt[:, 1:] == srt[:, :-1]) & (srt[:, 1:] >= 0)
+    assert not dup.any() and (p64.max(dim=1).values < t.to(torch.int64)).all(), "distinct positions below the token count"
+    # the protected regions are whole: the newest `window` tokens and the first `sink` tokens are all still there
+    newest = torch.minimum(t, torch.full_like(t, W)).to(torch.int64)
+    kept_recent = (used & (p64 >= (t.to(torch.int64) - newest)[:, None])).sum(1)
+    assert torch.equal(kept_recent, newest), "recent window retained"
+    if S > 0:
+        assert torch.equal((used & (p64 < S)).sum(1), torch.minimum(t, torch.full_like(t, S)).to(torch.int64)), "initial tokens retained"
+    # the chain: next and prev are inverse on occupied slots, positions increase along it, one head and one tail
+    idx = torch.arange(m + 1, device=dev)[None, :].expand(lanes, -1)
+    n64, q64 = nxt[:, :m + 1].to(torch.int64), prv[:, :m + 1].to(torch.int64)
+    has_next, has_prev = used & (n64 >= 0), used & (q64 >= 0)
+    assert torch.equal(has_next.sum(1), (length - 1).clamp(min=0).to(torch.int64)), "every entry but the tail has a right neighbour"
+    assert torch.equal(has_prev.sum(1), (length - 1).clamp(min=0).to(torch.int64)), "every entry but the head has a left neighbour"
+    back = torch.gather(q64, 1, n64.clamp(min=0))
+    pos_next = torch.gather(p64, 1, n64.clamp(min=0))
+    assert (back[has_next] == idx[has_next]).all(), "prev[next[s]] = s"
+    assert (pos_next[has_next] > p64[has_next]).all(), "positions increase along the chain"
+    nonempty = length > 0
+    hs, ts = head[nonempty].to(torch.int64), tail[nonempty].to(torch.int64)
+    rows = torch.nonzero(nonempty)[:, 0]
+    assert (q64[rows, hs] == -1).all() and (n64[rows, ts] == -1).all() and used[rows, hs].all() and used[rows, ts].all(), "head and tail"
+    assert (p64[rows, ts] == t[nonempty].to(torch.int64) - 1).all(), "the tail is the newest token"
+    full = t > m
+    assert (~used[full, :][torch.arange(int(full.sum()), device=dev), free[full].to(torch.int64)]).all(), "the free slot is free"
+    # accumulated scores: non-negative, each at most the steps its entry has been attended, all of a lane at most the steps
+    n_att = (t.to(torch.int64)[:, None] - p64).clamp(min=0)
+    av = torch.where(used, a[:, :m + 1], torch.zeros_like(a[:, :m + 1]))
+    assert (av >= 0).all() and (av <= n_att.to(torch.float32) * (1 + 1e-5) + 1e-6).all(), "0 <= a <= n"
+    assert (av.sum(1, dtype=torch.float64) <= t.to(torch.float64) * (1 + 1e-5)).all(), "sum of a <= steps"
+    if evicted is not None:
+        ev = evicted.reshape(-1).to(torch.int64)
+        comp = full
+        assert (ev[~comp] == -1).all() and (ev[comp] >= S).all() and (ev[comp] <= t[comp].to(torch.int64) - 1 - W).all(), "removed position in range"
+        assert not (used & (p64 == ev[:, None]) & comp[:, None]).any(), "the removed position is gone"

@@ -9,7 +9,7 @@ import torch
 
 from paper_2503_01330_b200.synth import WORKLOADS
 
-from parity_util import Parity
+from parity_util import Parity, check_all_lanes
 
 pytestmark = pytest.mark.gpu
 
@@ -31,6 +31,8 @@ def test_full_shape_sampled_lanes(name, n_sample, decode, schedule):
     p.decode(4, layers_entry=True)
     p.compare_state()
     assert p.n_evictions >= len(p.lanes) * (100 + decode)
+    # ... and what holds at any size, on every lane of the context (not only the sampled ones)
+    check_all_lanes(p.ctx, wl, (p.lens + decode + 4).tolist(), p.ev)
     p.close()
     torch.cuda.empty_cache()
 
@@ -81,5 +83,6 @@ def test_serving_and_gqa_full_prompt_lengths(name, n_sample, decode):
     p.decode(decode)
     p.compare_state()
     assert p.n_evictions >= sum(int(p.lens[b]) - wl.budget for _, b, _ in p.lanes)
+    check_all_lanes(p.ctx, wl, (p.lens + decode).tolist(), p.ev)
     p.close()
     torch.cuda.empty_cache()
