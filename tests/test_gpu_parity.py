@@ -183,10 +183,12 @@ def test_large_budget_is_full_attention():
     p.close()
 
 
-def test_bounded_wait_reports_timeout_and_context_survives():
-    """A wait that nothing completes runs out of polls: the status word says so, once, and decoding goes on."""
+@pytest.mark.parametrize("schedule", [binding.WKV_SCHEDULE_AUTO, binding.WKV_SCHEDULE_SPLIT])
+def test_bounded_wait_reports_timeout_and_context_survives(schedule):
+    """A wait that nothing completes runs out of polls: the status word says so, once, and decoding goes on (with the
+    two-kernel schedule the status call also clears the lanes' arrival counters, which must leave the next step intact)."""
     wl = small(batch=1, hq=2, hkv=2, d=64, dtype="f32", m=12, W=2)
-    p = Parity(wl, seed=2)
+    p = Parity(wl, seed=2, schedule=schedule, n_splits=2 if schedule else 0)
     p.decode(20)
     p.ctx.wkv_selftest_wait_timeout()
     assert p.ctx.wkv_status() == binding.WKV_ERR_TIMEOUT
