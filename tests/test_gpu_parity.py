@@ -351,6 +351,47 @@ def test_large_imported_caches_grouped_heads(dtype, d, hq, hkv, m, schedule):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("hq,hkv,batch,m", [
+    (20, 20, 16, 4351),     # 320 lanes x 4352 entries: exactly what 256 threads x 17 slots hold (the register epilogue's limit)
+    (20, 20, 16, 4352),     # one entry more: the loop version of the epilogue, and a streamed prompt tail
+    (4, 4, 4, 4607),        # 16 lanes x 4608 entries: the limit of the 512-thread epilogue (9 slots per thread)
+    (4, 4, 4, 4608),        # ... and one more
+    (8, 2, 8, 3455),        # four heads per key, 16 lanes x 3456 entries: the limit of the 384-thread epilogue
+    (8, 2, 8, 3456),
+])
+def test_lane_lengths_at_the_register_epilogue_limits(hq, hkv, batch, m):
+    """Lanes exactly as long as the register version of the lane epilogue takes, and one entry longer (the loop version
+    through global scratch): imported full caches, a prompt chunk through wkv_prefill_bulk (blocked tail on one side of
+    the limit, streamed on the other), decode steps through both entry points; sampled lanes against the oracle."""
+    wl = small(batch=batch, hq=hq, hkv=hkv, d=128, dtype="bf16", m=m, W=40, S=2, rank=16)
+    p = Parity(wl, seed=m, sample=8, ragged=[m + 500] * batch)
+    rng = np.random.default_rng(m)
+    tokens = m + 300
+    lane_set = {ln: i for i, ln in enumerate(p.lanes)}
+    K1 = torch.from_numpy((rng.standard_normal((m, 128)) * 0.3).astype(np.float32)).to(torch.bfloat16)
+    V1 = torch.from_numpy(rng.standard_normal((m, 128)).astype(np.float32)).to(torch.bfloat16)
+    for b in range(batch):
+        for h in range(hkv):
+            pos = np.sort(np.concatenate([np.arange(2), 2 + rng.choice(tokens - 2, size=m - 2, replace=False)])).astype(np.int32)
+            pos[-40:] = np.arange(tokens - 40, tokens)                       # the recent window is always whole
+            pos = np.unique(pos)
+            while len(pos) < m:                                              # (the window may have swallowed a drawn position)
+                pos = np.unique(np.concatenate([pos, 2 + rng.choice(tokens - 42, size=m - len(pos))])).astype(np.int32)
+            a = (rng.random(m) * (tokens - pos) * 1e-4 + 1e-8).astype(np.float32)
+            p.ctx.wkv_import_state(0, b, h, tokens=tokens, pos=torch.from_numpy(pos), a=torch.from_numpy(a), K=K1, V=V1)
+            if (0, b, h) in lane_set:
+                p.ref.import_state(lane_set[(0, b, h)], tokens, pos, a.astype(np.float64), K1.float().numpy(), V1.float().numpy())
+    p.t = tokens
+    p.lens = torch.full((batch,), tokens + 100, dtype=torch.int32)
+    p.prefill(19, chunk=19, bulk=True)       # two blocks of 8 and a block of 3 where the tail is blocked
+    p.decode(4)
+    p.decode(2, layers_entry=True)
+    p.compare_state()
+    assert p.n_evictions == 25 * len(p.lanes)
+    p.close()
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("dtype,schedule", [("f32", binding.WKV_SCHEDULE_SPLIT), ("bf16", binding.WKV_SCHEDULE_CLUSTER)])
 def test_structural_ties_and_saturated_softmax(dtype, schedule):
     """Degenerate score distributions.  (1) zero queries: every probability is exactly 1/(m+1) (m+1 a power of two), so
