@@ -818,7 +818,7 @@ static int stream_tokens(wkv_ctx* c, int32_t layer, const void* Q, const void* K
 // query heads per key) must be 8 at most, the window must be longer than the block (an entry removed inside the block and
 // its right neighbour are then never tokens of the block), and the lane epilogue must be the register version.
 static int block_tokens_of(const wkv_ctx* c, int lanes) {
-  if (c->use_cluster || c->group > 4) return 0;
+  if (c->group > 4) return 0;
   const int B = 8 / c->group;
   if (c->cfg.window <= B) return 0;
   const int nt = epilogue_threads(c->group, lanes, c->sm_count);
