@@ -275,7 +275,7 @@ inline int epilogue_threads(int G, int lanes, int sms) {
 // The lane-epilogue kernel: one CTA per lane, launched with programmatic stream serialization (it orders itself
 // against its predecessor on the device).
 template <typename T, int D, int G>
-cudaError_t launch_epilogue(const wkv::StepParams& P, int lanes, int dev, cudaStream_t stream) {
+cudaError_t launch_epilogue(const wkv::StepParams& P, int lanes, int dev, cudaStream_t stream, bool whole_block = false) {
   cudaLaunchAttribute pdl[1];
   pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   pdl[0].val.programmaticStreamSerializationAllowed = 1;
@@ -293,6 +293,17 @@ cudaError_t launch_epilogue(const wkv::StepParams& P, int lanes, int dev, cudaSt
   const int e_slots = wkv::epilogue_slots_per_thread(G, nt) * nt;
   P2.ep_stage_slots = (e_slots > 0 && P.budget + 1 <= e_slots) ? P.cap : 0;
   k2.dynamicSmemBytes = (size_t)P2.ep_stage_slots * 8;
+  if (whole_block) {
+    // every token of a block of a blocked prompt tail in one launch (lane_epilogue_block_kernel)
+    if constexpr (G <= 2) {
+      if (nt == wkv::kEpilogueThreadsWide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_block_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P2);
+    }
+    if constexpr (G == 4) {
+      if (nt == wkv::kEpilogueThreadsMid) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_block_kernel_mid<T, D, G>, P2);
+    }
+    if constexpr (G <= 4) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_block_kernel<T, D, G, wkv::kEpilogueThreads>, P2);
+    return cudaErrorInvalidValue;
+  }
   if constexpr (G <= 2) {
     if (nt == wkv::kEpilogueThreadsWide) return cudaLaunchKernelEx(&k2, wkv::lane_epilogue_kernel<T, D, G, wkv::kEpilogueThreadsWide>, P2);
   }
@@ -876,9 +887,9 @@ static cudaError_t launch_block(const wkv_ctx* c, int which, const wkv::BlockPar
 template <typename T, int D>
 static cudaError_t launch_epilogue_by_group(int G, const wkv::StepParams& P, int lanes, int dev, cudaStream_t s) {
   switch (G) {
-    case 1: return launch_epilogue<T, D, 1>(P, lanes, dev, s);
-    case 2: return launch_epilogue<T, D, 2>(P, lanes, dev, s);
-    case 4: return launch_epilogue<T, D, 4>(P, lanes, dev, s);
+    case 1: return launch_epilogue<T, D, 1>(P, lanes, dev, s, true);
+    case 2: return launch_epilogue<T, D, 2>(P, lanes, dev, s, true);
+    case 4: return launch_epilogue<T, D, 4>(P, lanes, dev, s, true);
   }
   return cudaErrorInvalidValue;
 }
@@ -938,20 +949,17 @@ static int blocked_tokens(wkv_ctx* c, long long lane0, int lanes, int B, const v
     cudaError_t e = launch_block(c, 0, BP, lanes);
     c->launches += 1;
     if (e != cudaSuccess) return cuda_fail(c, e, "block logits launch");
-    for (int i = 0; i < n_tok; ++i) {
-      const int t = t0 + i;
-      P.tok_idx = t;
-      P.block_step = i;
-      P.logit_row0 = i * G;
-      P.probs_row0 = i * G;
-      P.q = (const char*)Q + (size_t)t * Hq * D * c->elem;
-      P.k = (const char*)K + (size_t)t * Hk * D * c->elem;
-      P.v = (const char*)V + (size_t)t * Hk * D * c->elem;
-      P.evicted = evicted_pos ? evicted_pos + (size_t)t * Hk : c->stage_ev;
-      e = launch_epilogue_any(c, P, lanes);
-      c->launches += 1;
-      if (e != cudaSuccess) return cuda_fail(c, e, "lane epilogue launch (blocked prompt tail)");
-    }
+    // the block's tokens, one after the other inside one launch
+    P.tok_idx = t0;
+    P.block_n = n_tok;
+    P.k = (const char*)K + (size_t)t0 * Hk * D * c->elem;
+    P.v = (const char*)V + (size_t)t0 * Hk * D * c->elem;
+    P.kv_ts = Hk * D;
+    P.evicted = evicted_pos ? evicted_pos + (size_t)t0 * Hk : c->stage_ev;
+    P.ev_ts = evicted_pos ? Hk : 0;
+    e = launch_epilogue_any(c, P, lanes);
+    c->launches += 1;
+    if (e != cudaSuccess) return cuda_fail(c, e, "lane epilogue launch (blocked prompt tail)");
     if (out) {
       e = launch_block(c, 1, BP, lanes);
       if (e == cudaSuccess) e = launch_block(c, 2, BP, lanes);

@@ -7,12 +7,13 @@
 //   block_logits_kernel   one sweep over the K rows as they are before the block: the logits of all B tokens' queries
 //                         against every slot (reproducible dot, parked per token), plus the B x B logits of the block's
 //                         tokens against the block's own keys.
-//   lane_epilogue_kernel  B launches, one per token, in order (wkv_kernels.cuh, StepParams::block_tokens > 0): exactly
-//                         the per-token epilogue of the streamed step -- probabilities, score fold, pick, merge, relink --
-//                         on the parked logits of its token.  An entry that joined inside the block is recognised by its
-//                         position and takes its logit from the B x B table; removed entries are gone from the chain as
-//                         in streaming.  It writes the token's rows into the freed slot, leaves the token's probabilities
-//                         in a table (slot order) and records every value row that it changes as it was before.
+//   lane_epilogue_block_kernel  one launch (wkv_kernels.cuh, StepParams::block_tokens > 0): per lane, token after token,
+//                         exactly the per-token epilogue of the streamed step -- probabilities, score fold, pick, merge,
+//                         relink -- on the parked logits of each token.  An entry that joined inside the block is
+//                         recognised by its position and takes its logit from the B x B table; removed entries are gone
+//                         from the chain as in streaming.  Each step writes its token's rows into the freed slot, leaves
+//                         the token's probabilities in a table (slot order) and records every value row that it changes
+//                         as it was before.  (lane_epilogue_kernel does one such step per launch when given block_step.)
 //   block_pv_kernel       one sweep over the V rows as they are after the block: sum_s P[token][s] * V[s] for all B tokens.
 //   block_out_kernel      per query row of the block: adds the units' partial sums and, for every recorded change,
 //                         P[token][s] * (row as it was when the token attended - row as it is now) for the tokens in

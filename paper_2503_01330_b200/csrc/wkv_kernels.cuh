@@ -95,6 +95,9 @@ struct StepParams {
   // Blocked prompt tail (wkv_block.cuh): this launch finishes token number block_step of a block of block_tokens tokens
   // (0: not a blocked tail) whose logits against the cache as it was before the block were parked by one sweep.
   int block_tokens, block_step;
+  int block_n;           // lane_epilogue_block_kernel: tokens of the block that this one launch finishes, one after the other
+  long long kv_ts;       // ... elements between consecutive tokens' k (and v) rows of one sequence
+  long long ev_ts;       // ... int32 entries between consecutive tokens' removed positions (0: one shared entry)
   const float* lgx;      // [lanes][logit_rows][block_tokens]: logits against the block's own keys (entries that joined inside the block)
   float* rec_rows;       // [lanes][2 * block_tokens][D] fp32: value rows as they were before a step of the block changed them
   int32_t* rec_slot;     // [lanes][2 * block_tokens]: their slots (entry 2*step: the removed entry, 2*step + 1: its right neighbour), -1 = none
@@ -404,7 +407,15 @@ struct LaneView {
   const T *new_k, *new_v;    // this step's token (shared memory)
   int* st;                   // the lane's state words
   int head, tail;            // chain ends before this step (only the code that finishes the lane reads them)
+  int step;                  // set and used only by the kernel that finishes a whole block of a blocked prompt tail (kLoop):
+  int row0;                  // the token's index inside its block, and the first row of its logits / probabilities
 };
+// Index of the step's token inside its block, and first row of its logits / probabilities among the lane's rows: launch
+// parameters, except in the kernel that loops over a block's tokens (kLoop), where they change from step to step.
+template <bool kLoop, typename T>
+__device__ __forceinline__ int step_of(const StepParams& P, const LaneView<T>& v) { return kLoop ? v.step : P.block_step; }
+template <bool kLoop, typename T>
+__device__ __forceinline__ int row0_of(const StepParams& P, const LaneView<T>& v) { return kLoop ? v.row0 : P.logit_row0; }
 
 // Lane-level part of a view: addresses and the even deal of tiles (the first tiles_total % n_splits units get one more).
 template <typename T, int D>
@@ -907,7 +918,7 @@ __device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsign
 
 // One slot's share of a step: p = e / Z per query head (written to the optional probability output), the group mean
 // folded into the slot's accumulated score (Algorithm 1: a = [a,0] + A_t), abar = a / n and the pick key.
-template <typename T, int G>
+template <typename T, int G, bool kLoop = false>
 __device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>& v, float* a_l, int32_t* pos_l, int slot,
                                          const float (&e)[G], const float* Z, float a_old, int pos_i, bool compress,
                                          unsigned long long& best, int& best_slot) {
@@ -915,7 +926,7 @@ __device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>&
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     pg[g] = __fdiv_rn(e[g], Z[g]);
-    if (P.probs) P.probs[((long long)v.lane_local * P.probs_rows + P.probs_row0 + g) * P.probs_stride + slot] = pg[g];
+    if (P.probs) P.probs[((long long)v.lane_local * P.probs_rows + row0_of<kLoop>(P, v) + g) * P.probs_stride + slot] = pg[g];
   }
   float pbar = pg[0];
 #pragma unroll
@@ -991,7 +1002,7 @@ __device__ __forceinline__ unsigned long long group_min_key(unsigned long long b
 
 // Link the new entry as the chain's tail, unlink the victim j (Algorithm 1: remove K[j], a[j], n[j]; the right
 // neighbour keeps its own key, a and n), merge V[j] into V[next[j]], update the lane state.  One group per lane runs it.
-template <typename T, int D, int G, int NT>
+template <typename T, int D, int G, int NT, bool kLoop = false>
 __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const EpScratch& ep, bool compress,
                                             unsigned long long bmin, int j_slot) {
   static_assert(NT >= D, "one thread per channel of the merged row");
@@ -1056,9 +1067,9 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     v.st[LS_HEAD] = head;
     v.st[LS_TAIL] = tail;
     v.st[LS_FREE] = new_free;
-    if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk] = ev_pos;
+    if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk + (kLoop ? (long long)v.step * P.ev_ts : 0ll)] = ev_pos;
     if (blocked) {
-      int32_t* rs = P.rec_slot + ((long long)v.lane_local * P.block_tokens + P.block_step) * 2;
+      int32_t* rs = P.rec_slot + ((long long)v.lane_local * P.block_tokens + step_of<kLoop>(P, v)) * 2;
       rs[0] = ep.i32[2];                                   // the removed entry's slot (-1: nothing removed)
       rs[1] = (ep.i32[2] >= 0 && P.merge) ? ep.i32[3] : -1;
     }
@@ -1070,10 +1081,10 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     const float wj = ep.misc[0], wr = ep.misc[1];
     const float vr = r == r_early ? vr_early : to_f32(r == new_slot ? v.new_v[tid] : __ldcg(Vw + (long long)r * D + tid));
     Vw[(long long)r * D + tid] = from_f32<T>(__fmaf_rn(wj, vj, __fmul_rn(wr, vr)));
-    if (blocked) P.rec_rows[(((long long)v.lane_local * P.block_tokens + P.block_step) * 2 + 1) * D + tid] = vr;
+    if (blocked) P.rec_rows[(((long long)v.lane_local * P.block_tokens + step_of<kLoop>(P, v)) * 2 + 1) * D + tid] = vr;
   }
   if (blocked && compress && ep.i32[2] >= 0 && tid < D)
-    P.rec_rows[(((long long)v.lane_local * P.block_tokens + P.block_step) * 2) * D + tid] = vj;
+    P.rec_rows[(((long long)v.lane_local * P.block_tokens + step_of<kLoop>(P, v)) * 2) * D + tid] = vj;
 }
 
 // Steps (1) and (2) of a lane's epilogue from global scratch: the split weights, the global maximum and normaliser of
@@ -1125,11 +1136,11 @@ __device__ __forceinline__ void combine_partials(const StepParams& P, const Lane
 
 // Zeroes of the optional probability output beyond the lane's entries.
 template <int G, int NT>
-__device__ __forceinline__ void clear_probs_tail(const StepParams& P, int lane_local, int L) {
+__device__ __forceinline__ void clear_probs_tail(const StepParams& P, int lane_local, int row0, int L) {
   if (P.probs) {
     for (int i = L + (int)threadIdx.x; i < P.budget + 1; i += NT)
 #pragma unroll
-      for (int g = 0; g < G; ++g) P.probs[((long long)lane_local * P.probs_rows + P.probs_row0 + g) * P.probs_stride + i] = 0.f;
+      for (int g = 0; g < G; ++g) P.probs[((long long)lane_local * P.probs_rows + row0 + g) * P.probs_stride + i] = 0.f;
   }
 }
 
@@ -1137,6 +1148,7 @@ __device__ __forceinline__ void clear_probs_tail(const StepParams& P, int lane_l
 template <typename T, int D, int G, int NT>
 __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, const LaneView<T>& v, const EpScratch& ep) {
   const int L = v.L;
+  constexpr bool kLoop = false;
   float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.cap;
   combine_partials<T, D, G, NT>(P, v, ep);
   // (3) Z_g as an exact integer sum
@@ -1153,7 +1165,7 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
   unsigned long long best = ~0ull;
   int best_slot = -1;
   fold_scores<T, G, NT>(P, v, lg, P.cap, 0, L, Zr, compress, best, best_slot);
-  clear_probs_tail<G, NT>(P, v.lane_local, L);
+  clear_probs_tail<G, NT>(P, v.lane_local, row0_of<kLoop>(P, v), L);
   int j_slot;
   const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
@@ -1165,11 +1177,11 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
 // before the lane's scan was even finished -- the scan writes neither; a thread reads back only what it staged itself)
 // and their parked logits are requested here in one go and stay in registers, so the lane pays one round trip to L2
 // where the loop version pays one per few slots and phase.  Same arithmetic, same results.
-template <typename T, int D, int G, int NT, int E>
+template <typename T, int D, int G, int NT, int E, bool kLoop = false>
 __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, const LaneView<T>& v, const EpScratch& ep,
                                                            const float* a_s, const int* pos_s) {
   const int tid = threadIdx.x, L = v.L;
-  const float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.cap;
+  const float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + row0_of<kLoop>(P, v)) * P.cap;
   float sx[E][G];
 #pragma unroll
   for (int u = 0; u < E; ++u) {
@@ -1180,8 +1192,8 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
   if (P.block_tokens > 0) {
     // Blocked prompt tail: the parked logits were taken against the cache as it was before the block.  An entry that
     // joined inside the block (its position says so) has its logit in the small table of the block's own keys.
-    const int t0 = v.t - P.block_step;
-    const float* lx = P.lgx + ((long long)v.lane_local * P.logit_rows + P.logit_row0) * P.block_tokens;
+    const int t0 = v.t - step_of<kLoop>(P, v);
+    const float* lx = P.lgx + ((long long)v.lane_local * P.logit_rows + row0_of<kLoop>(P, v)) * P.block_tokens;
 #pragma unroll
     for (int u = 0; u < E; ++u) {
       const int i = tid + u * NT;
@@ -1241,13 +1253,13 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
 #pragma unroll
   for (int u = 0; u < E; ++u) {
     const int i = tid + u * NT;
-    if (i < L) fold_one<T, G>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot);
+    if (i < L) fold_one<T, G, kLoop>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot);
   }
-  clear_probs_tail<G, NT>(P, v.lane_local, L);
+  clear_probs_tail<G, NT>(P, v.lane_local, row0_of<kLoop>(P, v), L);
   int j_slot;
   const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
-  finish_lane<T, D, G, NT>(P, v, ep, compress, bmin, j_slot);
+  finish_lane<T, D, G, NT, kLoop>(P, v, ep, compress, bmin, j_slot);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1526,6 +1538,7 @@ template <typename T, int D, int G>
 constexpr int scan_smem_bytes() { return Cfg<T, D, G>::kScanBytes; }
 
 constexpr int kEpilogueThreads = 256;
+constexpr int kEpilogueThreadsMid = 384;      // four query heads, a layer of at most two lanes per SM
 constexpr int kEpilogueThreadsWide = 512;     // one or two query heads only (registers: two CTAs per SM)
 // Slots per thread that the register version of the lane epilogue is compiled for (0: not compiled); a thread keeps
 // E * G logits in registers.  17 x 256 and 9 x 512 threads cover the 4097 entries of the largest single-head workload,
@@ -1637,8 +1650,71 @@ template <typename T, int D, int G, int NT>
 __global__ void __launch_bounds__(NT, G == 1 ? 1024 / NT : 1) lane_epilogue_kernel(const StepParams P) {
   lane_epilogue_body<T, D, G, NT>(P);
 }
+// The per-token lane epilogue for a whole block of a blocked prompt tail in ONE launch: a lane's tokens follow one another
+// inside the lane's CTA (lanes are independent, so nothing is ordered across CTAs), which spares the launch gap and the
+// grid-wide wait between tokens that one launch per token costs.  Same steps, same order, same results as B launches of
+// lane_epilogue_kernel with block_step = 0 .. B-1.
+template <typename T, int D, int G, int NT>
+__device__ __forceinline__ void lane_epilogue_block_body(const StepParams& P) {
+  __shared__ __align__(16) unsigned char ep_raw[EpScratch::bytes(G)];
+  EpScratch ep;
+  ep.carve(ep_raw, G);
+  constexpr int E = epilogue_slots_per_thread(G, NT);
+  extern __shared__ __align__(16) unsigned char ep_dyn[];
+  float* a_s = reinterpret_cast<float*>(ep_dyn);
+  int* pos_s = reinterpret_cast<int*>(ep_dyn) + P.ep_stage_slots;
+  const int lane_local = blockIdx.x;
+  const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
+  griddep_wait();                                        // the block's logit sweep (and everything before it) is done
+  griddep_launch();
+  for (int step = 0; step < P.block_n; ++step) {
+    if (P.seq_lens != nullptr && P.tok_idx + step >= P.seq_lens[b]) {          // the sequence has ended (same for the whole CTA)
+      if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk + (long long)step * P.ev_ts] = -1;
+      continue;
+    }
+    LaneView<T> v;
+    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;   // written by thread 0 in the step before
+    fill_view<T, D>(v, P, lane_local, 0, __ldcg(st + LS_LEN), __ldcg(st + LS_T), __ldcg(st + LS_FREE));
+    v.head = __ldcg(st + LS_HEAD);
+    v.tail = __ldcg(st + LS_TAIL);
+    v.step = step;
+    v.row0 = step * G;
+    v.new_k = v.Kl + (long long)v.new_slot * D;
+    v.new_v = v.Vl + (long long)v.new_slot * D;
+    {
+      // the token's rows go into its slot (thread c writes channel c and is the only one to read it back in this step)
+      const T* k_in = reinterpret_cast<const T*>(P.k) + b * P.kv_bs + (long long)step * P.kv_ts + (long long)hk * D;
+      const T* v_in = reinterpret_cast<const T*>(P.v) + b * P.kv_bs + (long long)step * P.kv_ts + (long long)hk * D;
+      for (int c = threadIdx.x; c < D; c += NT) {
+        const_cast<T*>(v.new_k)[c] = k_in[c];
+        const_cast<T*>(v.new_v)[c] = v_in[c];
+      }
+    }
+    if (E > 0 && v.L <= E * NT && v.L <= P.ep_stage_slots) {
+      const float* a_l = P.a + v.lane * P.cap;
+      const int32_t* pos_l = P.pos + v.lane * P.cap;
+      for (int i = threadIdx.x; i < v.L; i += NT) {
+        const bool old_entry = i != v.new_slot;
+        a_s[i] = old_entry ? __ldcg(a_l + i) : 0.f;
+        pos_s[i] = old_entry ? __ldcg(pos_l + i) : v.t;
+      }
+      if constexpr (E > 0) lane_epilogue_in_registers<T, D, G, NT, E, true>(P, v, ep, a_s, pos_s);
+    } else if (threadIdx.x == 0) {
+      atomicOr(P.status, kStatusBadLink);                 // the host sends blocked tails only where the lane fits
+    }
+    __syncthreads();                                     // the step's writes before the next step reads them; scratch reuse
+  }
+}
+template <typename T, int D, int G, int NT>
+__global__ void __launch_bounds__(NT, G == 1 ? 1024 / NT : 1) lane_epilogue_block_kernel(const StepParams P) {
+  lane_epilogue_block_body<T, D, G, NT>(P);
+}
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kEpilogueThreadsMid, 2) lane_epilogue_block_kernel_mid(const StepParams P) {
+  lane_epilogue_block_body<T, D, G, kEpilogueThreadsMid>(P);
+}
+
 // Four query heads, a layer of at most two lanes per SM: 384 threads per lane, held to the registers of two CTAs per SM.
-constexpr int kEpilogueThreadsMid = 384;
 template <typename T, int D, int G>
 __global__ void __launch_bounds__(kEpilogueThreadsMid, 2) lane_epilogue_kernel_mid(const StepParams P) {
   lane_epilogue_body<T, D, G, kEpilogueThreadsMid>(P);

@@ -156,8 +156,8 @@ def test_provider_refusing_the_blocked_tail_scratch_falls_back_to_streaming():
         launches = L.wkv_launch_count(h)
         assert L.wkv_prefill_bulk(h, 0, dp(Q), dp(K), dp(V), None, 120, None, None) == binding.WKV_OK
         launches = L.wkv_launch_count(h) - launches
-        # 64 tokens dense, 56 in blocks of 8 (one sweep + 8 lane epilogues each) -- or streamed, two launches per token
-        assert launches == (1 + 56 * 2 if refuse else 1 + 7 * 9) and p.calls == (n_create + 2 if refuse else n_create + 7)
+        # 64 tokens dense, 56 in blocks of 8 (one sweep + one lane-epilogue launch each) -- or streamed, two launches per token
+        assert launches == (1 + 56 * 2 if refuse else 1 + 7 * 2) and p.calls == (n_create + 2 if refuse else n_create + 7)
         assert L.wkv_status(h) == binding.WKV_OK
         pos = torch.empty(64, dtype=torch.int32)
         a = torch.empty(64)

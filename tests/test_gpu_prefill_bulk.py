@@ -292,13 +292,13 @@ def test_blocked_prompt_tail_every_token(dtype, d, hq, hkv, m, W, S, T, chunk):
     p.prefill(T, chunk=chunk, bulk=True)
     launches = p.ctx.wkv_launch_count() - before
     # what the blocked path launches: per call the dense kernel (if the layer is still below the budget), then per block
-    # one logit sweep, one lane epilogue per token, the value sweep and the output kernel
+    # one logit sweep, one lane-epilogue launch for the block's tokens, the value sweep and the output kernel
     B, expected, consumed = 8 // (hq // hkv), 0, 0
     for t0 in range(0, T, chunk):
         tc = min(chunk, T - t0)
         n0 = min(tc, max(0, m - consumed))
         tail = tc - n0
-        expected += (1 if n0 > 0 else 0) + (2 * tail if tail < 2 else 3 * ((tail + B - 1) // B) + tail)
+        expected += (1 if n0 > 0 else 0) + (2 * tail if tail < 2 else 4 * ((tail + B - 1) // B))
         consumed += tc
     assert launches == expected, "the tail did not go through the blocked path"
     p.compare_state()
