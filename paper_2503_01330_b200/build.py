@@ -8,7 +8,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libwkv.so")
 SOURCES = ["wkv_api.cu"]
-DEPS = SOURCES + ["wkv_kernels.cuh", "wkv_prefill.cuh", os.path.join("..", "..", "include", "wkv.h")]
+DEPS = SOURCES + ["wkv_kernels.cuh", "wkv_prefill.cuh", "wkv_block.cuh", os.path.join("..", "..", "include", "wkv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC"]
 
