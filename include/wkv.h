@@ -85,8 +85,8 @@ const char* wkv_config_error(const wkv_config* cfg);
 /* Validates cfg, allocates the cache and bookkeeping for n_layers*batch*n_kv_heads lanes on the current
  * CUDA device through the provider and clears them (Algorithm 1 starts from empty score and count lists).  *out is
  * NULL on failure; when the provider returns NULL for one of the blocks the call returns WKV_ERR_ALLOC after handing
- * every block it had obtained back to `release`.  With four query heads per key on bf16 rows the cache scan takes its value tiles through a
- * tensor map, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
+ * every block it had obtained back to `release`.  On bf16 rows the cache scan with four query heads per key and the value sweep of a blocked prompt tail take
+ * their value tiles through a tensor map, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
  * the driver lacks it, WKV_ERR_INVALID if the value cache would have 2^31 rows or more. */
 int wkv_create(const wkv_config* cfg, wkv_ctx** out);
 

@@ -139,7 +139,7 @@ int encode_value_map(wkv_ctx* c, void* base, unsigned long long rows, int head_d
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
   if (qr != cudaDriverEntryPointSuccess || !sym) return fail(c, WKV_ERR_CUDA, "the driver has no cuTensorMapEncodeTiled");
-  if (rows >= 0x7fffffffULL) return fail(c, WKV_ERR_INVALID, "n_layers * batch * n_kv_heads * (budget + 1) must stay below 2^31 rows with four query heads per key");
+  if (rows >= 0x7fffffffULL) return fail(c, WKV_ERR_INVALID, "n_layers * batch * n_kv_heads * (budget + 1) must stay below 2^31 rows with bf16 storage");
   const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
   const cuuint32_t box[2] = {64u, (cuuint32_t)wkv::kTileSlots};
@@ -612,7 +612,8 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   WKV_TAKE(&c->stage_out, (size_t)cfg->n_layers * cfg->batch * cfg->n_q_heads * row);
   WKV_TAKE(&c->stage_ev, (size_t)c->lanes_total * 4);
 #undef WKV_TAKE
-  if (rc == WKV_OK && c->group == 4 && cfg->dtype == WKV_BF16)
+  // bf16 rows: the scan with four query heads per key and the value sweep of a blocked prompt tail take V tiles through it
+  if (rc == WKV_OK && cfg->dtype == WKV_BF16)
     rc = encode_value_map(c, c->Vc, (unsigned long long)c->lanes_total * cap, cfg->head_dim);
   if (rc == WKV_OK) rc = run_reset(c);
   if (rc != WKV_OK) {
@@ -869,9 +870,10 @@ static cudaError_t launch_block_kernels(int which, const wkv::BlockParams& BP, i
     block_logits_kernel<T, D, R><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
   } else if (which == 1) {
     constexpr int smem = BlockCfg<T, D, R>::kPvSmem;
-    cudaError_t e = cudaFuncSetAttribute(block_pv_kernel<T, D, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    constexpr bool mma = BlockCfg<T, D, R>::kPvMma;      // bf16 rows: on the tensor cores
+    cudaError_t e = cudaFuncSetAttribute(block_pv_kernel<T, D, R, mma>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    block_pv_kernel<T, D, R><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
+    block_pv_kernel<T, D, R, mma><<<lanes * BP.n_units, kThreads, smem, s>>>(BP);
   } else {
     block_out_kernel<T, D><<<lanes * BP.block_tokens * BP.group, D, 0, s>>>(BP);
   }
@@ -920,6 +922,7 @@ static int blocked_tokens(wkv_ctx* c, long long lane0, int lanes, int B, const v
   BP.q_ts = Hq * D; BP.kv_ts = Hk * D; BP.out_ts = Hq * D;
   BP.lane0 = (int)lane0; BP.n_kv_heads = c->cfg.n_kv_heads; BP.cap = c->cap; BP.budget = c->cfg.budget;
   BP.block_tokens = B; BP.group = G; BP.n_units = c->blk_units; BP.scale = c->scale;
+  std::memcpy(BP.vmap, c->vmap, sizeof(BP.vmap));
 
   wkv::StepParams P = base_params(c, 0);
   P.lane0 = (int)lane0;

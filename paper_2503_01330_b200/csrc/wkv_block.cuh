@@ -52,6 +52,8 @@ struct BlockParams {
   int group;                 // query heads per kv head
   int n_units;               // CTAs per lane in the two sweeps
   float scale;
+  // Tensor map over the value cache (as in StepParams), for the value sweep on the tensor cores.
+  alignas(64) unsigned char vmap[128];
 };
 
 // tokens of the block that sequence b still has (ragged prompts end inside a block)
@@ -69,6 +71,11 @@ struct BlockCfg {
   static constexpr int kStages = 4;
   static constexpr int kProbBytes = R * kTileSlots * 4;                      // [R][32] fp32 per stage (value sweep)
   static constexpr int kLogitsSmem = kStages * kTileBytes + kTileBytes + 2 * kStages * 8 + 64;
+  // Value sweep on the tensor cores: bf16 rows, R = 8 tokens (the n dimension of mma.m16n8k8), and a tensor map for
+  // the swizzled V tiles (a stage must then start on a 1024-byte boundary, which kTileBytes + kProbBytes keeps).
+  static constexpr bool kPvMma = sizeof(T) == 2 && R == 8 && D % 64 == 0;
+  static constexpr int kVHalves = kRowBytes / 128;
+  static constexpr int kVHalfBytes = kTileSlots * 128;
   static constexpr int kPvSmem = kStages * (kTileBytes + kProbBytes) + kConsumerWarps * R * D * 4 + 2 * kStages * 8 + 64;
 };
 
@@ -162,9 +169,10 @@ __global__ void __launch_bounds__(kThreads) block_logits_kernel(const BlockParam
 // ------------------------------------------------------------------------------------------------
 // sweep 2: sum_s P[row][s] * V[s] over the unit's slots, all R rows at once
 // ------------------------------------------------------------------------------------------------
-template <typename T, int D, int R>
-__global__ void __launch_bounds__(kThreads) block_pv_kernel(const BlockParams P) {
+template <typename T, int D, int R, bool kMma>
+__global__ void __launch_bounds__(kThreads) block_pv_kernel(const __grid_constant__ BlockParams P) {
   using BC = BlockCfg<T, D, R>;
+  static_assert(!kMma || BC::kPvMma, "the tensor-core sweep needs bf16 rows and blocks of 8 query rows");
   constexpr int NS = BC::kStages;
   constexpr int NC = kConsumerWarps * 32;
   constexpr int LPR = 16, CH = D / 16, CP = CH / 2, RPP = 32 / LPR, PASSES = 8 / RPP;
@@ -205,11 +213,76 @@ __global__ void __launch_bounds__(kThreads) block_pv_kernel(const BlockParams P)
         const int slot0 = (tile_begin + i) * kTileSlots;
         const uint32_t bytes = (uint32_t)min(kTileSlots, L - slot0) * BC::kRowBytes;
         unsigned char* dst = ring + (size_t)s * kStage;
-        mbar_expect_tx(&full_bar[s], bytes + (uint32_t)BC::kProbBytes);
-        bulk_g2s(dst, Vl + (long long)slot0 * D, bytes, &full_bar[s]);
+        if constexpr (kMma) {
+          // whole boxes of 32 rows in the swizzled layout (rows past the lane's slots: other bytes, zeroed by the consumers)
+          mbar_expect_tx(&full_bar[s], (uint32_t)(BC::kVHalves * BC::kVHalfBytes + BC::kProbBytes));
+#pragma unroll
+          for (int h = 0; h < BC::kVHalves; ++h)
+            tensor_g2s_2d(dst + h * BC::kVHalfBytes, P.vmap, h * 64, (int)(lane * P.cap) + slot0, &full_bar[s]);
+        } else {
+          mbar_expect_tx(&full_bar[s], bytes + (uint32_t)BC::kProbBytes);
+          bulk_g2s(dst, Vl + (long long)slot0 * D, bytes, &full_bar[s]);
+        }
         // the tile's probabilities: 32 slots of every row (entries past the lane's slots are never used)
         for (int r = 0; r < R; ++r)
           bulk_g2s(dst + BC::kTileBytes + r * kTileSlots * 4, pt + (long long)r * P.cap + slot0, kTileSlots * 4, &full_bar[s]);
+      }
+    }
+  } else if constexpr (kMma) {
+    // (V rows)^T [channels x 8 rows] times the block's probabilities [8 rows x R tokens] per warp and tile, in blocks of
+    // 16 channels: mma.m16n8k8 with the value fragments read transposed out of the swizzled tile, each probability as a
+    // bf16 high part plus a bf16 low part (two products into one accumulator).  Warp w owns rows 8w .. 8w+7 of every
+    // tile.  Accumulator of block j: channels 16j + c and 16j + 8 + c (c = lane / 4) of tokens 2q and 2q+1 (q = lane % 4).
+    using SW = Scanner<T, D, 4>;                         // its v_word() addresses the swizzled tile
+    constexpr int NB = D / 16;
+    float oc[NB][4];
+#pragma unroll
+    for (int j = 0; j < NB; ++j) oc[j][0] = oc[j][1] = oc[j][2] = oc[j][3] = 0.f;
+    const int tokn = lane_id >> 2, q2 = (lane_id & 3) * 2;                // B fragment: column (token), first of its two rows
+    for (int i = 0; i < n_tiles; ++i) {
+      const int s = i % NS;
+      mbar_wait(&full_bar[s], (i / NS) & 1, P.status);
+      T* tV = reinterpret_cast<T*>(ring + (size_t)s * kStage);
+      const float* tP = reinterpret_cast<const float*>(ring + (size_t)s * kStage + BC::kTileBytes);
+      const int slot0 = (tile_begin + i) * kTileSlots;
+      if (slot0 + kTileSlots > L) {
+        // ragged tile: rows beyond L hold other bytes, possibly NaN patterns, and 0 * NaN would reach the accumulators
+        for (int w = lane_id; w < 8 * (BC::kRowBytes / 4); w += 32) {
+          const int r = w / (BC::kRowBytes / 4);
+          if (slot0 + warp * 8 + r >= L) *SW::v_word(tV, warp * 8 + r, w % (BC::kRowBytes / 4)) = 0u;
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // before the stage is refilled
+        __syncwarp();
+      }
+      const int row = warp * 8 + q2;
+      float2 p = *reinterpret_cast<const float2*>(tP + tokn * kTileSlots + row);
+      if (slot0 + row >= L) p.x = 0.f;                                    // entries past the lane's slots are stale
+      if (slot0 + row + 1 >= L) p.y = 0.f;
+      const __nv_bfloat162 hi = __floats2bfloat162_rn(p.x, p.y);
+      const float2 hf = __bfloat1622float2(hi);
+      const __nv_bfloat162 lo = __floats2bfloat162_rn(p.x - hf.x, p.y - hf.y);
+      const uint32_t bh = *reinterpret_cast<const uint32_t*>(&hi), bl = *reinterpret_cast<const uint32_t*>(&lo);
+#pragma unroll
+      for (int jj = 0; jj < NB / 2; ++jj) {
+        uint32_t af[4];
+        ldmatrix_x4_trans(af, SW::v_word(tV, warp * 8 + (lane_id & 7), (4 * jj + (lane_id >> 3)) * 4));
+        mma_m16n8k8_bf16(oc[2 * jj], af[0], af[1], bh);
+        mma_m16n8k8_bf16(oc[2 * jj], af[0], af[1], bl);
+        mma_m16n8k8_bf16(oc[2 * jj + 1], af[2], af[3], bh);
+        mma_m16n8k8_bf16(oc[2 * jj + 1], af[2], af[3], bl);
+      }
+      release_stage(&empty_bar[s]);
+    }
+    {
+      const int c = lane_id >> 2;
+      float* wa = warp_part + (warp * R + q2) * D;       // token 2q
+      float* wb = wa + D;                                // token 2q + 1
+#pragma unroll
+      for (int j = 0; j < NB; ++j) {
+        wa[16 * j + c] = oc[j][0];
+        wb[16 * j + c] = oc[j][1];
+        wa[16 * j + 8 + c] = oc[j][2];
+        wb[16 * j + 8 + c] = oc[j][3];
       }
     }
   } else {
@@ -289,17 +362,31 @@ __global__ void __launch_bounds__(D) block_out_kernel(const BlockParams P) {
   const float* pt = P.ptab + ((long long)lane_local * R + row) * P.cap;
   const int32_t* rs = P.rec_slot + (long long)lane_local * P.block_tokens * 2;
   const float* rr = P.rec_rows + (long long)lane_local * P.block_tokens * 2 * D;
+  // A record made at step k (k >= tok) holds the row of its slot as token tok attended it, unless an earlier record
+  // (tok <= k' < k) of the same slot does: the first record of a slot at or after the token's own step counts.  One
+  // thread per record decides that and fetches the token's probability of the slot; the channel threads then go over
+  // the records without a load that depends on another.
+  constexpr int kMaxRec = 16;                            // 2 * block_tokens, block_tokens <= 8
+  __shared__ int rec_slot_s[kMaxRec];
+  __shared__ float rec_p_s[kMaxRec];
+  const int n_rec = 2 * n_act;
+  if (c < kMaxRec) {
+    int slot = -1;
+    if (c >= 2 * tok && c < n_rec) {
+      slot = rs[c];
+      for (int k2 = 2 * tok; k2 < c; ++k2)
+        if (rs[k2] == slot) slot = -1;
+    }
+    rec_slot_s[c] = slot;
+    rec_p_s[c] = slot >= 0 ? pt[slot] : 0.f;
+  }
   float o = 0.f;
   for (int u = 0; u < P.n_units; ++u) o += P.opart[(((long long)lane_local * P.n_units + u) * R + row) * D + c];
-  // A record made at step k (k >= tok) holds the row of its slot as token tok attended it, unless an earlier record
-  // (tok <= k' < k) of the same slot does: the first record of a slot at or after the token's own step counts.
-  for (int k = 2 * tok; k < 2 * n_act; ++k) {
-    const int slot = rs[k];
-    if (slot < 0) continue;
-    bool first = true;
-    for (int k2 = 2 * tok; k2 < k; ++k2) first = first && rs[k2] != slot;
-    if (!first) continue;
-    o += pt[slot] * (rr[(long long)k * D + c] - to_f32(Vl[(long long)slot * D + c]));
+  __syncthreads();
+#pragma unroll 4
+  for (int k = 2 * tok; k < n_rec; ++k) {
+    const int slot = rec_slot_s[k];                      // the same for every thread of the CTA
+    if (slot >= 0) o += rec_p_s[k] * (rr[(long long)k * D + c] - to_f32(Vl[(long long)slot * D + c]));
   }
   T* dst = reinterpret_cast<T*>(P.out) + b * P.out_bs + (long long)(P.tok0 + tok) * P.out_ts + ((long long)hk * P.group + g) * D;
   dst[c] = from_f32<T>(o);
