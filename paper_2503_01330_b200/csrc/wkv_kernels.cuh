@@ -409,6 +409,8 @@ struct LaneView {
   int head, tail;            // chain ends before this step (only the code that finishes the lane reads them)
   int step;                  // set and used only by the kernel that finishes a whole block of a blocked prompt tail (kLoop):
   int row0;                  // the token's index inside its block, and the first row of its logits / probabilities
+  int* st_s;                 // ... shared-memory copy of the state words, kept current from token to token
+  const float* lgx_s;        // ... the lane's logits against the block's own keys [rows][block_tokens], in shared memory
 };
 // Index of the step's token inside its block, and first row of its logits / probabilities among the lane's rows: launch
 // parameters, except in the kernel that loops over a block's tokens (kLoop), where they change from step to step.
@@ -921,7 +923,7 @@ __device__ __forceinline__ void group_sum_u64(unsigned long long (&x)[G], unsign
 template <typename T, int G, bool kLoop = false>
 __device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>& v, float* a_l, int32_t* pos_l, int slot,
                                          const float (&e)[G], const float* Z, float a_old, int pos_i, bool compress,
-                                         unsigned long long& best, int& best_slot) {
+                                         unsigned long long& best, int& best_slot, float* a_s = nullptr) {
   float pg[G];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
@@ -934,6 +936,7 @@ __device__ __forceinline__ void fold_one(const StepParams& P, const LaneView<T>&
   if (G > 1) pbar = __fmul_rn(pbar, 1.0f / (float)G);
   const float a_new = __fadd_rn(a_old, pbar);
   a_l[slot] = a_new;
+  if constexpr (kLoop) a_s[slot] = a_new;              // the staged copy serves the block's next token (and the merge weights)
   if (slot == v.new_slot) pos_l[slot] = v.t;
   if (compress && pos_i >= P.sink && pos_i <= v.t - P.window) {
     const float abar = __fdiv_rn(a_new, __int2float_rn(v.t - pos_i + 1));
@@ -1004,7 +1007,8 @@ __device__ __forceinline__ unsigned long long group_min_key(unsigned long long b
 // neighbour keeps its own key, a and n), merge V[j] into V[next[j]], update the lane state.  One group per lane runs it.
 template <typename T, int D, int G, int NT, bool kLoop = false>
 __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<T>& v, const EpScratch& ep, bool compress,
-                                            unsigned long long bmin, int j_slot) {
+                                            unsigned long long bmin, int j_slot, const float* a_s = nullptr,
+                                            const int* pos_s = nullptr) {
   static_assert(NT >= D, "one thread per channel of the merged row");
   const int tid = threadIdx.x;
   const int t = v.t, new_slot = v.new_slot, L = v.L;
@@ -1045,8 +1049,9 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
       } else {
         const int pv = prev_l[j];
         const float abar_j = __uint_as_float((uint32_t)(bmin >> 32));
-        const int pos_r = r == new_slot ? t : __ldcg(pos_l + r);
-        const float abar_r = __fdiv_rn(__ldcg(a_l + r), __int2float_rn(t - pos_r + 1));
+        // (kLoop: the staged copies are current -- this step's fold wrote them before the pick's barrier)
+        const int pos_r = kLoop ? pos_s[r] : (r == new_slot ? t : __ldcg(pos_l + r));
+        const float abar_r = __fdiv_rn(kLoop ? a_s[r] : __ldcg(a_l + r), __int2float_rn(t - pos_r + 1));
         const float Dn = __fadd_rn(abar_j, abar_r);
         float wj = 0.5f, wr = 0.5f;
         if (Dn != 0.f) { wj = __fdiv_rn(abar_j, Dn); wr = __fdiv_rn(abar_r, Dn); }
@@ -1067,6 +1072,13 @@ __device__ __forceinline__ void finish_lane(const StepParams& P, const LaneView<
     v.st[LS_HEAD] = head;
     v.st[LS_TAIL] = tail;
     v.st[LS_FREE] = new_free;
+    if constexpr (kLoop) {
+      v.st_s[LS_LEN] = new_len;
+      v.st_s[LS_T] = t + 1;
+      v.st_s[LS_HEAD] = head;
+      v.st_s[LS_TAIL] = tail;
+      v.st_s[LS_FREE] = new_free;
+    }
     if (P.evicted) P.evicted[v.b * P.ev_bs + v.hk + (kLoop ? (long long)v.step * P.ev_ts : 0ll)] = ev_pos;
     if (blocked) {
       int32_t* rs = P.rec_slot + ((long long)v.lane_local * P.block_tokens + step_of<kLoop>(P, v)) * 2;
@@ -1179,7 +1191,7 @@ __device__ __forceinline__ void lane_epilogue_from_scratch(const StepParams& P, 
 // where the loop version pays one per few slots and phase.  Same arithmetic, same results.
 template <typename T, int D, int G, int NT, int E, bool kLoop = false>
 __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, const LaneView<T>& v, const EpScratch& ep,
-                                                           const float* a_s, const int* pos_s) {
+                                                           float* a_s, const int* pos_s) {
   const int tid = threadIdx.x, L = v.L;
   const float* lg = P.logits + ((long long)v.lane_local * P.logit_rows + row0_of<kLoop>(P, v)) * P.cap;
   float sx[E][G];
@@ -1199,7 +1211,8 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
       const int i = tid + u * NT;
       if (i < L && pos_s[i] >= t0) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) sx[u][g] = __ldcg(lx + g * P.block_tokens + (pos_s[i] - t0));
+        for (int g = 0; g < G; ++g)
+          sx[u][g] = kLoop ? v.lgx_s[(v.row0 + g) * P.block_tokens + (pos_s[i] - t0)] : __ldcg(lx + g * P.block_tokens + (pos_s[i] - t0));
       }
     }
     // no split partials here: the maximum of every head comes from the logits themselves (exact, order-free)
@@ -1253,13 +1266,13 @@ __device__ __forceinline__ void lane_epilogue_in_registers(const StepParams& P, 
 #pragma unroll
   for (int u = 0; u < E; ++u) {
     const int i = tid + u * NT;
-    if (i < L) fold_one<T, G, kLoop>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot);
+    if (i < L) fold_one<T, G, kLoop>(P, v, a_l, pos_l, i, sx[u], Zr, a_s[i], pos_s[i], compress, best, best_slot, a_s);
   }
   clear_probs_tail<G, NT>(P, v.lane_local, row0_of<kLoop>(P, v), L);
   int j_slot;
   const unsigned long long bmin = group_min_key<NT>(best, best_slot, ep.u64 + 64, j_slot);   // its barrier also publishes a, pos
   // (5), (6)
-  finish_lane<T, D, G, NT, kLoop>(P, v, ep, compress, bmin, j_slot);
+  finish_lane<T, D, G, NT, kLoop>(P, v, ep, compress, bmin, j_slot, a_s, pos_s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1667,18 +1680,32 @@ __device__ __forceinline__ void lane_epilogue_block_body(const StepParams& P) {
   const int b = lane_local / P.n_kv_heads, hk = lane_local % P.n_kv_heads;
   griddep_wait();                                        // the block's logit sweep (and everything before it) is done
   griddep_launch();
+  // What a token's step would otherwise fetch from L2 again is kept in shared memory from token to token: the lane's
+  // state words (thread 0 keeps the copy current), its scores and positions (staged once; every step's fold keeps
+  // the scores current, and the only position that changes is the new token's) and the block's own-key logits.
+  __shared__ int st_s[LS_STRIDE];
+  __shared__ float lgx_s[64];                            // rows * block_tokens = G * B * B <= 64
+  {
+    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;
+    if (threadIdx.x < LS_STRIDE) st_s[threadIdx.x] = __ldcg(st + threadIdx.x);
+    const int n_lgx = min(64, P.logit_rows * P.block_tokens);
+    for (int i = threadIdx.x; i < n_lgx; i += NT) lgx_s[i] = __ldcg(P.lgx + (long long)lane_local * P.logit_rows * P.block_tokens + i);
+  }
+  __syncthreads();
+  bool staged = false;
   for (int step = 0; step < P.block_n; ++step) {
     if (P.seq_lens != nullptr && P.tok_idx + step >= P.seq_lens[b]) {          // the sequence has ended (same for the whole CTA)
       if (threadIdx.x == 0 && P.evicted) P.evicted[b * P.ev_bs + hk + (long long)step * P.ev_ts] = -1;
       continue;
     }
     LaneView<T> v;
-    const int* st = P.lane_state + ((long long)P.lane0 + lane_local) * LS_STRIDE;   // written by thread 0 in the step before
-    fill_view<T, D>(v, P, lane_local, 0, __ldcg(st + LS_LEN), __ldcg(st + LS_T), __ldcg(st + LS_FREE));
-    v.head = __ldcg(st + LS_HEAD);
-    v.tail = __ldcg(st + LS_TAIL);
+    fill_view<T, D>(v, P, lane_local, 0, st_s[LS_LEN], st_s[LS_T], st_s[LS_FREE]);   // written by thread 0 in the step before
+    v.head = st_s[LS_HEAD];
+    v.tail = st_s[LS_TAIL];
     v.step = step;
     v.row0 = step * G;
+    v.st_s = st_s;
+    v.lgx_s = lgx_s;
     v.new_k = v.Kl + (long long)v.new_slot * D;
     v.new_v = v.Vl + (long long)v.new_slot * D;
     {
@@ -1691,12 +1718,18 @@ __device__ __forceinline__ void lane_epilogue_block_body(const StepParams& P) {
       }
     }
     if (E > 0 && v.L <= E * NT && v.L <= P.ep_stage_slots) {
-      const float* a_l = P.a + v.lane * P.cap;
-      const int32_t* pos_l = P.pos + v.lane * P.cap;
-      for (int i = threadIdx.x; i < v.L; i += NT) {
-        const bool old_entry = i != v.new_slot;
-        a_s[i] = old_entry ? __ldcg(a_l + i) : 0.f;
-        pos_s[i] = old_entry ? __ldcg(pos_l + i) : v.t;
+      if (!staged) {
+        const float* a_l = P.a + v.lane * P.cap;
+        const int32_t* pos_l = P.pos + v.lane * P.cap;
+        for (int i = threadIdx.x; i < v.L; i += NT) {
+          const bool old_entry = i != v.new_slot;
+          a_s[i] = old_entry ? __ldcg(a_l + i) : 0.f;
+          pos_s[i] = old_entry ? __ldcg(pos_l + i) : v.t;
+        }
+        staged = true;
+      } else if ((int)threadIdx.x == v.new_slot % NT) {    // the thread that owns the slot: Algorithm 1's [a, 0] at position t
+        a_s[v.new_slot] = 0.f;
+        pos_s[v.new_slot] = v.t;
       }
       if constexpr (E > 0) lane_epilogue_in_registers<T, D, G, NT, E, true>(P, v, ep, a_s, pos_s);
     } else if (threadIdx.x == 0) {
