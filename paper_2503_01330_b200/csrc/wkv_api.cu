@@ -129,7 +129,16 @@ int take(wkv_ctx* c, P** dst, size_t bytes) {
 // Tensor map over the value cache as a [rows][head_dim] bf16 matrix, boxes of 64 elements x one tile of rows, 128-byte
 // swizzle, zero fill past the last row.  The driver's encoder is found through the runtime: the library does not
 // link against the driver.
+int encode_rows_map(wkv_ctx* c, unsigned char* out128, const void* base, unsigned long long row_elems, unsigned long long rows,
+                    unsigned box_rows);
 int encode_value_map(wkv_ctx* c, void* base, unsigned long long rows, int head_dim) {
+  if (rows >= 0x7fffffffULL) return fail(c, WKV_ERR_INVALID, "n_layers * batch * n_kv_heads * (budget + 1) must stay below 2^31 rows with bf16 storage");
+  return encode_rows_map(c, c->vmap, base, (unsigned long long)head_dim, rows, (unsigned)wkv::kTileSlots);
+}
+// bf16 matrix [rows][row_elems] (row-major, rows 16-byte aligned), boxes of 64 elements x box_rows rows, 128-byte swizzle,
+// zero fill outside the matrix.
+int encode_rows_map(wkv_ctx* c, unsigned char* out128, const void* base, unsigned long long row_elems, unsigned long long rows,
+                    unsigned box_rows) {
   typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -139,17 +148,16 @@ int encode_value_map(wkv_ctx* c, void* base, unsigned long long rows, int head_d
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qr);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)");
   if (qr != cudaDriverEntryPointSuccess || !sym) return fail(c, WKV_ERR_CUDA, "the driver has no cuTensorMapEncodeTiled");
-  if (rows >= 0x7fffffffULL) return fail(c, WKV_ERR_INVALID, "n_layers * batch * n_kv_heads * (budget + 1) must stay below 2^31 rows with bf16 storage");
-  const cuuint64_t dims[2] = {(cuuint64_t)head_dim, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)head_dim * 2};
-  const cuuint32_t box[2] = {64u, (cuuint32_t)wkv::kTileSlots};
+  const cuuint64_t dims[2] = {(cuuint64_t)row_elems, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_elems * 2};
+  const cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1u, 1u};
   CUtensorMap m;
-  const CUresult r = reinterpret_cast<encode_fn>(sym)(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+  const CUresult r = reinterpret_cast<encode_fn>(sym)(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(c, WKV_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
-  std::memcpy(c->vmap, &m, sizeof(m));
+  std::memcpy(out128, &m, sizeof(m));
   return WKV_OK;
 }
 
@@ -498,9 +506,9 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
   return WKV_OK;
 }
 
-template <typename T, int D, int KT>
+template <typename T, int D, int KT, bool kTma = false>
 cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
-  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT>();
+  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT, kTma>();
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -508,10 +516,10 @@ cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStrea
     return cudaGetLastError();
   };
   switch (G) {
-    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT>);
-    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT>);
-    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT>);
-    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT>);
+    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT, kTma>);
+    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT, kTma>);
+    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT, kTma>);
+    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT, kTma>);
   }
   return cudaErrorInvalidValue;
 }
@@ -995,8 +1003,9 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
 
 // The dense kernel over `lanes` consecutive lanes starting at lane0 (one layer, or all layers at once: to the kernel the
 // lanes of several layers are just more sequences).  Takes the scratch on first use / when more lanes are needed.
+// fresh: no lane of the launch holds a token yet (every key then comes from this call's K and V).
 static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void* Q, const void* K, const void* V,
-                        const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos) {
+                        const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos, bool fresh) {
   if (c->bulk_S == nullptr || c->bulk_lanes < lanes) {
     c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
     int rc = take(c, &c->bulk_S, (size_t)lanes * wkv::kBulkRows * c->bulk_stride * 4);
@@ -1022,7 +1031,24 @@ static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void
   const int n = (int)lanes;
   if (c->cfg.dtype == WKV_BF16) {
     // 128-key tiles (two CTAs per SM) unless there are more lanes than that keeps busy
-    if (n <= 2 * c->sm_count)
+    const bool wide = n <= 2 * c->sm_count;
+    const unsigned long long rows = (unsigned long long)(lanes / c->cfg.n_kv_heads) * (unsigned long long)T_max;
+    const unsigned long long row_elems = (unsigned long long)c->cfg.n_kv_heads * c->cfg.head_dim;
+    // lanes that hold nothing yet take their tiles through tensor maps over this call's K and V
+    bool tma = fresh && rows < 0x7fffffffULL;
+    if (tma) {
+      int rc = encode_rows_map(c, P.kmap, K, row_elems, rows, wide ? 128u : 64u);
+      if (rc == WKV_OK) rc = encode_rows_map(c, P.vmap, V, row_elems, rows, wide ? 128u : 64u);
+      if (rc != WKV_OK) return rc;
+    }
+    if (tma) {
+      if (wide)
+        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128, true>(c->group, P, n, c->stream)
+                                   : launch_bulk<__nv_bfloat16, 64, 128, true>(c->group, P, n, c->stream);
+      else
+        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64, true>(c->group, P, n, c->stream)
+                                   : launch_bulk<__nv_bfloat16, 64, 64, true>(c->group, P, n, c->stream);
+    } else if (wide)
       e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, n, c->stream)
                                  : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, n, c->stream);
     else
@@ -1055,7 +1081,7 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     // whatever each lane already holds), the rest is streamed behind it on the same stream.
     n0 = (int32_t)std::min<long long>(T_max, room);
     rc = launch_dense(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, Q, K, V, seq_lens, T_max, n0, out,
-                      evicted_pos);
+                      evicted_pos, c->tokens_hi[layer] == 0);
     if (rc != WKV_OK) return rc;
     c->tokens_hi[layer] += n0;
   }
@@ -1088,17 +1114,18 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
   int32_t n0 = 0;
   if (room > 0 && T_max > 0) {
     n0 = (int32_t)std::min<long long>(T_max, room);        // uncompressed in every lane of every layer (see wkv_prefill_bulk)
+    const bool fresh = room == c->cfg.budget;               // no layer holds a token yet
     const int stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
     const size_t need_all = (size_t)c->lanes_total * wkv::kBulkRows * stride * 4;
     if (need_all <= ((size_t)256 << 20)) {
       // every lane of every layer in one launch
-      rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos);
+      rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos, fresh);
       if (rc != WKV_OK) return rc;
     } else {
       for (int l = 0; l < L; ++l) {
         rc = launch_dense(c, (long long)l * c->lanes_per_layer, c->lanes_per_layer, (const char*)Q + l * q_layer,
                           (const char*)K + l * kv_layer, (const char*)V + l * kv_layer, seq_lens, T_max, n0,
-                          out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr);
+                          out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr, fresh);
         if (rc != WKV_OK) return rc;
       }
     }

@@ -51,16 +51,25 @@ struct PrefillParams {
   int s_stride;              // multiple of kBulkKeys, >= n0
   float scale;
   uint32_t* status;          // device status word (bounded waits report here)
+  // kTma kernels only: tensor maps over this call's K and V as [sequences * T_max][n_kv_heads * D] matrices, boxes of
+  // 64 elements x one tile of keys, 128-byte swizzle (encoded by the host per call).
+  alignas(64) unsigned char kmap[128];
+  alignas(64) unsigned char vmap[128];
 };
 
 // Keys per tile (a template parameter of the kernel): 64, or 128 for 2-byte storage.  Two tiles of padded rows live in
 // shared memory.  128-key tiles amortise the per-tile work better (4 x 4 outputs per thread, two CTAs per SM); 64-key
 // tiles let four CTAs share an SM, which wins once a layer has more lanes than two per SM.
 
-template <typename T, int D, int KT>
+// kTma (bf16 rows, lanes that hold nothing yet): a tile arrives as one tensor-map copy per 128-byte half of its rows,
+// in the 128-byte swizzle ([half][key][128 B], 16-byte chunk index XORed with key % 8), instead of one bulk copy per
+// row into padded rows: the copy engine of an SM takes tens of cycles per request whatever its size, and a row per
+// request kept it busier than the arithmetic.  Both layouts are free of bank conflicts for the two access patterns
+// (a thread per key in the logits, transposed fragment loads in P.V).
+template <typename T, int D, int KT, bool kTma = false>
 constexpr int bulk_smem_bytes() {
   return kBulkRows * D * 4                                   // query rows, fp32
-         + 2 * KT * (D * (int)sizeof(T) + 16)                // two tile stages, storage type, padded rows
+         + 2 * KT * (D * (int)sizeof(T) + (kTma ? 0 : 16))   // two tile stages, storage type, padded rows (or swizzled)
          + KT * kBulkPadP * 4                                // probabilities of a tile, fp32
          + (sizeof(T) == 2 ? 2 * kBulkRows * (KT + 8) * 2 : 0)   // bf16 hi and lo parts of the probabilities
          + 64;                                               // mbarriers
@@ -111,20 +120,28 @@ __device__ __forceinline__ void mma_m16n8k16_bf16(float (&c)[4], const uint32_t 
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-template <typename T, int D, int G, int KT>
-__global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_kernel(const PrefillParams P) {
+// Byte offset of element `elem` of key `key` inside a swizzled tile of KT keys (see bulk_smem_bytes).
+template <int KT>
+__device__ __forceinline__ uint32_t swz_off(int key, int elem) {
+  const int chunk = elem >> 3;                           // 16-byte chunk of the row
+  return (uint32_t)((chunk >> 3) * (KT * 128) + key * 128 + ((((chunk & 7) ^ (key & 7)) << 4) | ((elem & 7) << 1)));
+}
+
+template <typename T, int D, int G, int KT, bool kTma = false>
+__global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_kernel(const __grid_constant__ PrefillParams P) {
+  static_assert(!kTma || sizeof(T) == 2, "tensor-map tiles are for 2-byte rows");
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
   constexpr int KPT = KT / 32;                   // keys per thread in the logits phase
-  constexpr int RS = D + 16 / (int)sizeof(T);    // row stride of a tile in elements: 16 bytes of padding, no bank conflicts
+  constexpr int RS = D + (kTma ? 0 : 16 / (int)sizeof(T));   // row stride of a tile in elements: 16 bytes of padding, no bank conflicts (kTma: swizzled instead)
   constexpr int ROWB = D * (int)sizeof(T);       // bytes per row
   constexpr int CPT = D / 32;                    // output channels per thread in the P.V phase (fp32 storage)
   constexpr bool kTensorPV = sizeof(T) == 2;     // bf16 storage: P.V on the tensor cores
   constexpr int PS = KT + 8;                     // bf16 row stride of the hi / lo probability tiles
   constexpr int QV = ROWB / 128;                 // 16-byte pieces of the query block per thread
   static_assert(kBulkRows % G == 0 && kBulkThreads == 8 * kBulkRows && KT <= kBulkThreads && kBulkKeys % KT == 0, "thread maps");
-  extern __shared__ __align__(128) unsigned char bulk_smem[];
+  extern __shared__ __align__(1024) unsigned char bulk_smem[];           // (swizzled tiles start on 1024-byte boundaries)
   float* Qs = reinterpret_cast<float*>(bulk_smem);                       // [16][D] fp32
   T* stage0 = reinterpret_cast<T*>(Qs + kBulkRows * D);                  // 2 x [KT][RS]
   float* Pt = reinterpret_cast<float*>(stage0 + 2 * KT * RS);            // [KT][20]: probabilities, [key][row]
@@ -142,7 +159,8 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // score a_i so far; the host only sends lanes here whose n_old + n0 cannot exceed the budget.  This call adds n_new
   // tokens (input rows 0 .. n_new-1, global token index n_old + row); n = tokens held afterwards.
   const int n_old = P.lane_state[lane * LS_STRIDE + LS_T];
-  const bool consistent = P.lane_state[lane * LS_STRIDE + LS_LEN] == n_old && n_old + P.n0 <= P.s_stride && n_old + P.n0 < P.cap;
+  const bool consistent = P.lane_state[lane * LS_STRIDE + LS_LEN] == n_old && n_old + P.n0 <= P.s_stride && n_old + P.n0 < P.cap &&
+                          (!kTma || n_old == 0);         // kTma: every key comes from this call's tensors
   int n_new = P.n0;
   if (P.seq_lens != nullptr) n_new = min(n_new, max(0, P.seq_lens[b % P.batch]));
   const int n = n_old + n_new;
@@ -164,8 +182,8 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   if (n_new == 0) return;
 
   if (tid == 0) {
-    mbar_init(&full[0], KT);                             // every issuing thread arrives once per fill
-    mbar_init(&full[1], KT);
+    mbar_init(&full[0], kTma ? 1 : KT);                  // every issuing thread arrives once per fill
+    mbar_init(&full[1], kTma ? 1 : KT);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -174,7 +192,17 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   uint32_t parity = 0;                                   // bit s: parity of stage s's next completion
   // Keys / values of tokens before n_old come from the cache (slot = token), the others from this call's input.
   auto issue = [&](bool values, int kt, int s, int nk_) {
-    if (tid < KT) {
+    if constexpr (kTma) {
+      // whole boxes of KT keys: keys past nk_ are other tokens' rows (or zero fill past the end of the tensor); the
+      // causal mask keeps them out of the logits, and the value rows among them are zeroed before they are multiplied
+      if (tid == 0) {
+        mbar_expect_tx(&full[s], (uint32_t)(KT * ROWB));
+#pragma unroll
+        for (int h = 0; h < ROWB / 128; ++h)
+          tensor_g2s_2d(reinterpret_cast<unsigned char*>(stage0) + (size_t)s * KT * ROWB + h * KT * 128, values ? P.vmap : P.kmap,
+                        hk * D + h * 64, b * P.T_max + kt * KT, &full[s]);
+      }
+    } else if (tid < KT) {
       const int r = min(kt * KT + tid, nk_ - 1);
       const T* src = r < n_old ? (values ? Vl : Kl) + (long long)r * D : (values ? Vb : Kb) + (long long)(r - n_old) * Hk * D;
       mbar_expect_tx(&full[s], ROWB);
@@ -277,7 +305,12 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
 #pragma unroll
         for (int i = 0; i < 4; ++i) load_pairs<CP>(Qs + (4 * w + i) * D + blk * CH, qv[i]);
 #pragma unroll
-        for (int j = 0; j < KPT; ++j) load_pairs<CP>(Kt + (ln + 32 * j) * RS + blk * CH, kv[j]);
+        for (int j = 0; j < KPT; ++j) {
+          if constexpr (kTma)
+            load_pairs<CP>(reinterpret_cast<const T*>(reinterpret_cast<const unsigned char*>(Kt) + swz_off<KT>(ln + 32 * j, blk * CH)), kv[j]);
+          else
+            load_pairs<CP>(Kt + (ln + 32 * j) * RS + blk * CH, kv[j]);
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
 #pragma unroll
@@ -377,8 +410,20 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         *reinterpret_cast<float4*>(Pt + kk * kBulkPadP + 4 * w) = make_float4(p[0], p[1], p[2], p[3]);
       }
       wait_stage(s);                                     // the V tile
-      __syncthreads();                                   // the probability tiles
-      const T* Vt = stage0 + s * KT * RS;
+      T* Vt = stage0 + s * KT * RS;
+      if constexpr (kTma) {
+        if (k0 + KT > nk) {
+          // rows past the block's last key are not this block's: zero them (0 * NaN would reach the accumulators)
+          const int r0 = nk - k0;
+          for (int idx = tid; idx < (KT - r0) * (ROWB / 16); idx += kBulkThreads) {
+            const int row = r0 + idx / (ROWB / 16), c16 = idx % (ROWB / 16);
+            *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(Vt) + (c16 >> 3) * (KT * 128) + row * 128 + (c16 & 7) * 16) =
+                make_uint4(0u, 0u, 0u, 0u);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the stage is refilled
+        }
+      }
+      __syncthreads();                                   // the probability tiles (and the zeroed rows)
       fold_columns<G, KT>(Pt, a_l, a_prev, k0, t0, nk, n);
       if constexpr (kTensorPV) {
         // O += P . V on the tensor cores (the outputs are not part of the reproducible chain).  Warp w takes all 16
@@ -389,7 +434,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         const int frow = (ln & 7) + ((ln >> 3) & 1) * 8, fcol = (ln >> 4) * 8;
         const uint32_t a_off = (uint32_t)((frow * PS + fcol) * 2);
         const uint32_t ph_base = smem_u32(Ph) + a_off, pl_base = smem_u32(Pl) + a_off;
-        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((frow * RS + w * (D / 4) + fcol) * 2);
+        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((frow * RS + w * (D / 4) + fcol) * 2);   // (padded rows)
         for (int ks = 0; ks < ksteps; ++ks) {
           uint32_t ah[4], al[4];
           asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -399,9 +444,11 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
 #pragma unroll
           for (int np = 0; np < NTW / 2; ++np) {
             uint32_t bf[4];
+            const uint32_t v_addr = kTma ? smem_u32(Vt) + swz_off<KT>(ks * 16 + frow, w * (D / 4) + fcol + np * 16)
+                                         : v_base + (uint32_t)(ks * 16 * RS * 2 + np * 32);
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                          : "=r"(bf[0]), "=r"(bf[1]), "=r"(bf[2]), "=r"(bf[3])
-                         : "r"(v_base + (uint32_t)(ks * 16 * RS * 2 + np * 32)) : "memory");
+                         : "r"(v_addr) : "memory");
             mma_m16n8k16_bf16(cacc[2 * np], ah, bf[0], bf[1]);
             mma_m16n8k16_bf16(cacc[2 * np], al, bf[0], bf[1]);
             mma_m16n8k16_bf16(cacc[2 * np + 1], ah, bf[2], bf[3]);
