@@ -187,7 +187,10 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
  * wkv_prefill's; outputs and merged values agree within rounding.
  * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider, the first
  * blocked tail about 64 * lanes_per_layer * (budget + 1) bytes more (if the provider refuses those, the tail is streamed);
- * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
+ * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  On bf16 rows a call
+ * whose lanes hold nothing yet has the driver encode two tensor maps over K and V (host work of microseconds, nothing
+ * allocated; WKV_ERR_CUDA if the driver refuses), so K and V must stay valid until the call's work has run, as for every
+ * asynchronous call.  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos);
 

@@ -126,9 +126,8 @@ int take(wkv_ctx* c, P** dst, size_t bytes) {
   return WKV_OK;
 }
 
-// Tensor map over the value cache as a [rows][head_dim] bf16 matrix, boxes of 64 elements x one tile of rows, 128-byte
-// swizzle, zero fill past the last row.  The driver's encoder is found through the runtime: the library does not
-// link against the driver.
+// Tensor maps.  The driver's encoder is found through the runtime: the library does not link against the driver.
+// encode_value_map: the value cache as a [rows][head_dim] bf16 matrix, boxes of 64 elements x one scan tile of rows.
 int encode_rows_map(wkv_ctx* c, unsigned char* out128, const void* base, unsigned long long row_elems, unsigned long long rows,
                     unsigned box_rows);
 int encode_value_map(wkv_ctx* c, void* base, unsigned long long rows, int head_dim) {
