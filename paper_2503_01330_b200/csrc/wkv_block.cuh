@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kThreads) block_logits_kernel(const BlockParam
         const int slot0 = (tile_begin + i) * kTileSlots;
         const uint32_t bytes = (uint32_t)min(kTileSlots, L - slot0) * BC::kRowBytes;
         mbar_expect_tx(&full_bar[s], bytes);
-        bulk_g2s(ring + (size_t)s * BC::kTileBytes, Kl + (long long)slot0 * D, bytes, &full_bar[s]);
+        bulk_g2s_hint(ring + (size_t)s * BC::kTileBytes, Kl + (long long)slot0 * D, bytes, &full_bar[s], l2_policy_evict_first());   // streamed once
       }
     }
     return;
@@ -218,10 +218,10 @@ __global__ void __launch_bounds__(kThreads) block_pv_kernel(const __grid_constan
           mbar_expect_tx(&full_bar[s], (uint32_t)(BC::kVHalves * BC::kVHalfBytes + BC::kProbBytes));
 #pragma unroll
           for (int h = 0; h < BC::kVHalves; ++h)
-            tensor_g2s_2d(dst + h * BC::kVHalfBytes, P.vmap, h * 64, (int)(lane * P.cap) + slot0, &full_bar[s]);
+            tensor_g2s_2d_hint(dst + h * BC::kVHalfBytes, P.vmap, h * 64, (int)(lane * P.cap) + slot0, &full_bar[s], l2_policy_evict_first());
         } else {
           mbar_expect_tx(&full_bar[s], bytes + (uint32_t)BC::kProbBytes);
-          bulk_g2s(dst, Vl + (long long)slot0 * D, bytes, &full_bar[s]);
+          bulk_g2s_hint(dst, Vl + (long long)slot0 * D, bytes, &full_bar[s], l2_policy_evict_first());
         }
         // the tile's probabilities: 32 slots of every row (entries past the lane's slots are never used)
         for (int r = 0; r < R; ++r)

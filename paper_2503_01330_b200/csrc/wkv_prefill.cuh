@@ -190,6 +190,10 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // The ring.  Thread r < KT fetches row r of a tile: one bulk copy, counted in bytes on the stage's barrier.  Rows
   // beyond the last key of the block re-fetch that last key (finite values; their probabilities are exactly zero).
   uint32_t parity = 0;                                   // bit s: parity of stage s's next completion
+  // (kTma) the tiles are streamed -- every block re-reads them, long after they have left L2 -- while the scratch rows
+  // of logits are re-read within the block: the tiles are marked to leave L2 first (measured: 2 to 10 % of the kernel;
+  // marking the scratch rows to stay instead made it slower)
+  const uint64_t stream_policy = kTma ? l2_policy_evict_first() : 0ull;
   // Keys / values of tokens before n_old come from the cache (slot = token), the others from this call's input.
   auto issue = [&](bool values, int kt, int s, int nk_) {
     if constexpr (kTma) {
@@ -199,8 +203,8 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         mbar_expect_tx(&full[s], (uint32_t)(KT * ROWB));
 #pragma unroll
         for (int h = 0; h < ROWB / 128; ++h)
-          tensor_g2s_2d(reinterpret_cast<unsigned char*>(stage0) + (size_t)s * KT * ROWB + h * KT * 128, values ? P.vmap : P.kmap,
-                        hk * D + h * 64, b * P.T_max + kt * KT, &full[s]);
+          tensor_g2s_2d_hint(reinterpret_cast<unsigned char*>(stage0) + (size_t)s * KT * ROWB + h * KT * 128, values ? P.vmap : P.kmap,
+                             hk * D + h * 64, b * P.T_max + kt * KT, &full[s], stream_policy);
       }
     } else if (tid < KT) {
       const int r = min(kt * KT + tid, nk_ - 1);
