@@ -34,7 +34,7 @@ METRIC = "decode steps/sec incl. merge; achieved HBM GB/s vs B200 peak (1 GPU)"
 FALLBACK_HBM_GBS = 6650.0
 # workload -> (dram__bytes_read.sum + dram__bytes_write.sum per layer call, hash of the kernel source when captured);
 # profiles/scan_kernel_and_lane_epilogue_kernel_serving_b16.md
-NCU_TRAFFIC = {"serving_b16": (1090305000 + 12269824 + 27000000 + 0, "15ee060f24e0b939")}
+NCU_TRAFFIC = {"serving_b16": (1090256000 + 3704320 + 27001000 + 4352, "31d998bb0dfd8fd1")}
 
 
 def kernel_source_hash() -> str:
