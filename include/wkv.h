@@ -85,8 +85,8 @@ const char* wkv_config_error(const wkv_config* cfg);
 /* Validates cfg, allocates the cache and bookkeeping for n_layers*batch*n_kv_heads lanes on the current
  * CUDA device through the provider and clears them (Algorithm 1 starts from empty score and count lists).  *out is
  * NULL on failure; when the provider returns NULL for one of the blocks the call returns WKV_ERR_ALLOC after handing
- * every block it had obtained back to `release`.  On bf16 rows the cache scan with four query heads per key and the value sweep of a blocked prompt tail take
- * their value tiles through a tensor map, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
+ * every block it had obtained back to `release`.  On bf16 rows the cache scan with four query heads per key, the value sweep of a blocked prompt tail and the
+ * dense prompt kernel take tiles of the cache through tensor maps, which the driver encodes here (cuTensorMapEncodeTiled, looked up at run time): WKV_ERR_CUDA if
  * the driver lacks it, WKV_ERR_INVALID if the value cache would have 2^31 rows or more. */
 int wkv_create(const wkv_config* cfg, wkv_ctx** out);
 
@@ -187,10 +187,7 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
  * wkv_prefill's; outputs and merged values agree within rounding.
  * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider, the first
  * blocked tail about 64 * lanes_per_layer * (budget + 1) bytes more (if the provider refuses those, the tail is streamed);
- * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  On bf16 rows a call
- * whose lanes hold nothing yet has the driver encode two tensor maps over K and V (host work of microseconds, nothing
- * allocated; WKV_ERR_CUDA if the driver refuses), so K and V must stay valid until the call's work has run, as for every
- * asynchronous call.  Asynchronous. */
+ * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
                      int32_t T_max, void* out, int32_t* evicted_pos);
 

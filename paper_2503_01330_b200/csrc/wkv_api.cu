@@ -58,6 +58,9 @@ struct wkv_ctx {
   uint32_t* status = nullptr;
   // four query heads on bf16 rows: the scan takes its V tiles through this tensor map (see StepParams::vmap)
   alignas(64) unsigned char vmap[128] = {};
+  // bf16 rows: the K and the V cache once more, in boxes of 64 and of 128 rows (the dense prompt kernel's two tile sizes)
+  alignas(64) unsigned char dense_kmap[2][128] = {};
+  alignas(64) unsigned char dense_vmap[2][128] = {};
   // staging for the host-buffer entry point and for discarded prefill outputs
   void* stage_q = nullptr;
   void* stage_k = nullptr;
@@ -505,9 +508,9 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
   return WKV_OK;
 }
 
-template <typename T, int D, int KT, bool kTma = false>
+template <typename T, int D, int KT>
 cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
-  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT, kTma>();
+  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT>();
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
@@ -515,10 +518,10 @@ cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStrea
     return cudaGetLastError();
   };
   switch (G) {
-    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT, kTma>);
-    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT, kTma>);
-    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT, kTma>);
-    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT, kTma>);
+    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT>);
+    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT>);
+    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT>);
+    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT>);
   }
   return cudaErrorInvalidValue;
 }
@@ -622,6 +625,11 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   // bf16 rows: the scan with four query heads per key and the value sweep of a blocked prompt tail take V tiles through it
   if (rc == WKV_OK && cfg->dtype == WKV_BF16)
     rc = encode_value_map(c, c->Vc, (unsigned long long)c->lanes_total * cap, cfg->head_dim);
+  for (int i = 0; i < 2 && rc == WKV_OK && cfg->dtype == WKV_BF16; ++i) {
+    rc = encode_rows_map(c, c->dense_kmap[i], c->Kc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, i ? 128u : 64u);
+    if (rc == WKV_OK)
+      rc = encode_rows_map(c, c->dense_vmap[i], c->Vc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, i ? 128u : 64u);
+  }
   if (rc == WKV_OK) rc = run_reset(c);
   if (rc != WKV_OK) {
     wkv_destroy(c);
@@ -1002,9 +1010,8 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
 
 // The dense kernel over `lanes` consecutive lanes starting at lane0 (one layer, or all layers at once: to the kernel the
 // lanes of several layers are just more sequences).  Takes the scratch on first use / when more lanes are needed.
-// fresh: no lane of the launch holds a token yet (every key then comes from this call's K and V).
 static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void* Q, const void* K, const void* V,
-                        const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos, bool fresh) {
+                        const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos) {
   if (c->bulk_S == nullptr || c->bulk_lanes < lanes) {
     c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
     int rc = take(c, &c->bulk_S, (size_t)lanes * wkv::kBulkRows * c->bulk_stride * 4);
@@ -1031,23 +1038,10 @@ static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void
   if (c->cfg.dtype == WKV_BF16) {
     // 128-key tiles (two CTAs per SM) unless there are more lanes than that keeps busy
     const bool wide = n <= 2 * c->sm_count;
-    const unsigned long long rows = (unsigned long long)(lanes / c->cfg.n_kv_heads) * (unsigned long long)T_max;
-    const unsigned long long row_elems = (unsigned long long)c->cfg.n_kv_heads * c->cfg.head_dim;
-    // lanes that hold nothing yet take their tiles through tensor maps over this call's K and V
-    bool tma = fresh && rows < 0x7fffffffULL;
-    if (tma) {
-      int rc = encode_rows_map(c, P.kmap, K, row_elems, rows, wide ? 128u : 64u);
-      if (rc == WKV_OK) rc = encode_rows_map(c, P.vmap, V, row_elems, rows, wide ? 128u : 64u);
-      if (rc != WKV_OK) return rc;
-    }
-    if (tma) {
-      if (wide)
-        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128, true>(c->group, P, n, c->stream)
-                                   : launch_bulk<__nv_bfloat16, 64, 128, true>(c->group, P, n, c->stream);
-      else
-        e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64, true>(c->group, P, n, c->stream)
-                                   : launch_bulk<__nv_bfloat16, 64, 64, true>(c->group, P, n, c->stream);
-    } else if (wide)
+    // the kernel takes its tiles through the tensor maps over the caches (boxes of one tile of keys)
+    std::memcpy(P.kmap, c->dense_kmap[wide ? 1 : 0], sizeof(P.kmap));
+    std::memcpy(P.vmap, c->dense_vmap[wide ? 1 : 0], sizeof(P.vmap));
+    if (wide)
       e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, n, c->stream)
                                  : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, n, c->stream);
     else
@@ -1080,7 +1074,7 @@ int wkv_prefill_bulk(wkv_ctx* c, int32_t layer, const void* Q, const void* K, co
     // whatever each lane already holds), the rest is streamed behind it on the same stream.
     n0 = (int32_t)std::min<long long>(T_max, room);
     rc = launch_dense(c, (long long)layer * c->lanes_per_layer, c->lanes_per_layer, Q, K, V, seq_lens, T_max, n0, out,
-                      evicted_pos, c->tokens_hi[layer] == 0);
+                      evicted_pos);
     if (rc != WKV_OK) return rc;
     c->tokens_hi[layer] += n0;
   }
@@ -1113,18 +1107,17 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
   int32_t n0 = 0;
   if (room > 0 && T_max > 0) {
     n0 = (int32_t)std::min<long long>(T_max, room);        // uncompressed in every lane of every layer (see wkv_prefill_bulk)
-    const bool fresh = room == c->cfg.budget;               // no layer holds a token yet
     const int stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
     const size_t need_all = (size_t)c->lanes_total * wkv::kBulkRows * stride * 4;
     if (need_all <= ((size_t)256 << 20)) {
       // every lane of every layer in one launch
-      rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos, fresh);
+      rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos);
       if (rc != WKV_OK) return rc;
     } else {
       for (int l = 0; l < L; ++l) {
         rc = launch_dense(c, (long long)l * c->lanes_per_layer, c->lanes_per_layer, (const char*)Q + l * q_layer,
                           (const char*)K + l * kv_layer, (const char*)V + l * kv_layer, seq_lens, T_max, n0,
-                          out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr, fresh);
+                          out ? (char*)out + l * q_layer : nullptr, evicted_pos ? evicted_pos + l * ev_layer : nullptr);
         if (rc != WKV_OK) return rc;
       }
     }

@@ -51,8 +51,8 @@ struct PrefillParams {
   int s_stride;              // multiple of kBulkKeys, >= n0
   float scale;
   uint32_t* status;          // device status word (bounded waits report here)
-  // kTma kernels only: tensor maps over this call's K and V as [sequences * T_max][n_kv_heads * D] matrices, boxes of
-  // 64 elements x one tile of keys, 128-byte swizzle (encoded by the host per call).
+  // 2-byte rows only: tensor maps over the K and the V cache as [lanes_total * cap][D] matrices, boxes of 64 elements x
+  // one tile of keys, 128-byte swizzle (encoded once per context).
   alignas(64) unsigned char kmap[128];
   alignas(64) unsigned char vmap[128];
 };
@@ -61,13 +61,15 @@ struct PrefillParams {
 // shared memory.  128-key tiles amortise the per-tile work better (4 x 4 outputs per thread, two CTAs per SM); 64-key
 // tiles let four CTAs share an SM, which wins once a layer has more lanes than two per SM.
 
-// kTma (bf16 rows, lanes that hold nothing yet): a tile arrives as one tensor-map copy per 128-byte half of its rows,
-// in the 128-byte swizzle ([half][key][128 B], 16-byte chunk index XORed with key % 8), instead of one bulk copy per
-// row into padded rows: the copy engine of an SM takes tens of cycles per request whatever its size, and a row per
-// request kept it busier than the arithmetic.  Both layouts are free of bank conflicts for the two access patterns
-// (a thread per key in the logits, transposed fragment loads in P.V).
-template <typename T, int D, int KT, bool kTma = false>
+// 2-byte rows (kTma): a tile arrives as one tensor-map copy per 128-byte half of its rows, in the 128-byte swizzle
+// ([half][key][128 B], 16-byte chunk index XORed with key % 8), instead of one bulk copy per row into padded rows: the
+// copy engine of an SM takes tens of cycles per request whatever its size, and a row per request kept it busier than
+// the arithmetic.  Both layouts are free of bank conflicts for the two access patterns (a thread per key in the logits,
+// transposed fragment loads in P.V).  The tiles are read from the CACHE, where the kernel has put this call's rows
+// first (token i in slot i), so earlier chunks of a prompt and this one come through the same map.
+template <typename T, int D, int KT>
 constexpr int bulk_smem_bytes() {
+  constexpr bool kTma = sizeof(T) == 2;
   return kBulkRows * D * 4                                   // query rows, fp32
          + 2 * KT * (D * (int)sizeof(T) + (kTma ? 0 : 16))   // two tile stages, storage type, padded rows (or swizzled)
          + KT * kBulkPadP * 4                                // probabilities of a tile, fp32
@@ -127,9 +129,9 @@ __device__ __forceinline__ uint32_t swz_off(int key, int elem) {
   return (uint32_t)((chunk >> 3) * (KT * 128) + key * 128 + ((((chunk & 7) ^ (key & 7)) << 4) | ((elem & 7) << 1)));
 }
 
-template <typename T, int D, int G, int KT, bool kTma = false>
+template <typename T, int D, int G, int KT>
 __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_kernel(const __grid_constant__ PrefillParams P) {
-  static_assert(!kTma || sizeof(T) == 2, "tensor-map tiles are for 2-byte rows");
+  constexpr bool kTma = sizeof(T) == 2;          // tiles through the caches' tensor maps
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
@@ -159,8 +161,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // score a_i so far; the host only sends lanes here whose n_old + n0 cannot exceed the budget.  This call adds n_new
   // tokens (input rows 0 .. n_new-1, global token index n_old + row); n = tokens held afterwards.
   const int n_old = P.lane_state[lane * LS_STRIDE + LS_T];
-  const bool consistent = P.lane_state[lane * LS_STRIDE + LS_LEN] == n_old && n_old + P.n0 <= P.s_stride && n_old + P.n0 < P.cap &&
-                          (!kTma || n_old == 0);         // kTma: every key comes from this call's tensors
+  const bool consistent = P.lane_state[lane * LS_STRIDE + LS_LEN] == n_old && n_old + P.n0 <= P.s_stride && n_old + P.n0 < P.cap;
   int n_new = P.n0;
   if (P.seq_lens != nullptr) n_new = min(n_new, max(0, P.seq_lens[b % P.batch]));
   const int n = n_old + n_new;
@@ -197,14 +198,15 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   // Keys / values of tokens before n_old come from the cache (slot = token), the others from this call's input.
   auto issue = [&](bool values, int kt, int s, int nk_) {
     if constexpr (kTma) {
-      // whole boxes of KT keys: keys past nk_ are other tokens' rows (or zero fill past the end of the tensor); the
-      // causal mask keeps them out of the logits, and the value rows among them are zeroed before they are multiplied
+      // whole boxes of KT keys out of the cache: keys past nk_ are slots not yet filled (or zero fill past the end of
+      // the cache); the causal mask keeps them out of the logits, and the value rows among them are zeroed before they
+      // are multiplied
       if (tid == 0) {
         mbar_expect_tx(&full[s], (uint32_t)(KT * ROWB));
 #pragma unroll
         for (int h = 0; h < ROWB / 128; ++h)
           tensor_g2s_2d_hint(reinterpret_cast<unsigned char*>(stage0) + (size_t)s * KT * ROWB + h * KT * 128, values ? P.vmap : P.kmap,
-                             hk * D + h * 64, b * P.T_max + kt * KT, &full[s], stream_policy);
+                             h * 64, (int)(lane * P.cap) + kt * KT, &full[s], stream_policy);
       }
     } else if (tid < KT) {
       const int r = min(kt * KT + tid, nk_ - 1);
@@ -248,8 +250,10 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
     }
   };
   load_q(n_old);
-  issue(kKeys, 0, 0, min(n_old + BQ, n));
-  if (min(n_old + BQ, n) > KT) issue(kKeys, 1, 1, min(n_old + BQ, n));
+  if constexpr (!kTma) {
+    issue(kKeys, 0, 0, min(n_old + BQ, n));
+    if (min(n_old + BQ, n) > KT) issue(kKeys, 1, 1, min(n_old + BQ, n));
+  }
 
   // the cache after n uncompressed steps: token i in slot i, linked in order (Algorithm 1 appends, nothing is removed)
   {
@@ -276,6 +280,13 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
       st[LS_TAIL] = n - 1;
       st[LS_FREE] = n;                                   // while growing, slots fill in arrival order
     }
+  }
+  if constexpr (kTma) {
+    // the tiles come out of the cache rows just written: make those writes visible to the copy engine first
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __syncthreads();
+    issue(kKeys, 0, 0, min(n_old + BQ, n));
+    if (min(n_old + BQ, n) > KT) issue(kKeys, 1, 1, min(n_old + BQ, n));
   }
 
   for (int t0 = n_old; t0 < n; t0 += BQ) {
