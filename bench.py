@@ -569,6 +569,11 @@ def main():
         line["other_workloads"] = others
     if not args.no_bulk_prefill:
         line["bulk_prefill"] = bulk_prefill_figures(wl, dev, seed)
+        if world == 1 and not args.layers and wl.name == "serving_b16":
+            # a whole prompt past the budget (dense phase + blocked tail) on two layers of the shape, beside the same
+            # prompt streamed as Algorithm 1 prints it
+            import dataclasses
+            line["whole_prompt"] = whole_prompt_figures(dataclasses.replace(wl, n_layers=2), dev, seed, 2 * wl.budget)
     if not args.no_cpu_baseline:
         cores = os.cpu_count() or 1
         n_lanes = min(wl.lanes, 4 * cores)
