@@ -58,9 +58,9 @@ struct wkv_ctx {
   uint32_t* status = nullptr;
   // four query heads on bf16 rows: the scan takes its V tiles through this tensor map (see StepParams::vmap)
   alignas(64) unsigned char vmap[128] = {};
-  // bf16 rows: the K and the V cache once more, in boxes of 64 and of 128 rows (the dense prompt kernel's two tile sizes)
-  alignas(64) unsigned char dense_kmap[2][128] = {};
-  alignas(64) unsigned char dense_vmap[2][128] = {};
+  // bf16 rows: the K and the V cache once more, in boxes of 64 rows (the dense prompt kernel's tile)
+  alignas(64) unsigned char dense_kmap[128] = {};
+  alignas(64) unsigned char dense_vmap[128] = {};
   // staging for the host-buffer entry point and for discarded prefill outputs
   void* stage_q = nullptr;
   void* stage_k = nullptr;
@@ -72,6 +72,7 @@ struct wkv_ctx {
   float* bulk_S = nullptr;
   int bulk_stride = 0;
   long long bulk_lanes = 0;     // lanes the scratch has rows for
+  int bulk_rows = 0;            // ... logit rows per lane (16, or 32 where a launch ran blocks of 32 rows)
   // per layer: an upper bound on the tokens any lane of the layer has consumed since creation / reset; while it is
   // below the budget no lane has compressed and token i of every lane sits in slot i (kCompressed: unknown / beyond)
   // blocked prompt tail (wkv_block.cuh): scratch for `blk_lanes` lanes, taken on first use
@@ -508,20 +509,20 @@ int check_lane(wkv_ctx* c, int layer, int b, int h) {
   return WKV_OK;
 }
 
-template <typename T, int D, int KT>
+template <typename T, int D, int KT, int ROWS = wkv::kBulkRows>
 cudaError_t launch_bulk(int G, const wkv::PrefillParams& P, int lanes, cudaStream_t s) {
-  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT>();
+  constexpr int smem = wkv::bulk_smem_bytes<T, D, KT, ROWS>();
   auto go = [&](auto kern) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    kern<<<lanes, wkv::kBulkThreads, smem, s>>>(P);
+    kern<<<lanes, wkv::bulk_threads(ROWS), smem, s>>>(P);
     return cudaGetLastError();
   };
   switch (G) {
-    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT>);
-    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT>);
-    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT>);
-    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT>);
+    case 1: return go(wkv::prefill_bulk_kernel<T, D, 1, KT, ROWS>);
+    case 2: return go(wkv::prefill_bulk_kernel<T, D, 2, KT, ROWS>);
+    case 4: return go(wkv::prefill_bulk_kernel<T, D, 4, KT, ROWS>);
+    case 8: return go(wkv::prefill_bulk_kernel<T, D, 8, KT, ROWS>);
   }
   return cudaErrorInvalidValue;
 }
@@ -625,11 +626,10 @@ int wkv_create(const wkv_config* cfg, wkv_ctx** out) {
   // bf16 rows: the scan with four query heads per key and the value sweep of a blocked prompt tail take V tiles through it
   if (rc == WKV_OK && cfg->dtype == WKV_BF16)
     rc = encode_value_map(c, c->Vc, (unsigned long long)c->lanes_total * cap, cfg->head_dim);
-  for (int i = 0; i < 2 && rc == WKV_OK && cfg->dtype == WKV_BF16; ++i) {
-    rc = encode_rows_map(c, c->dense_kmap[i], c->Kc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, i ? 128u : 64u);
-    if (rc == WKV_OK)
-      rc = encode_rows_map(c, c->dense_vmap[i], c->Vc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, i ? 128u : 64u);
-  }
+  if (rc == WKV_OK && cfg->dtype == WKV_BF16)
+    rc = encode_rows_map(c, c->dense_kmap, c->Kc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, 64u);
+  if (rc == WKV_OK && cfg->dtype == WKV_BF16)
+    rc = encode_rows_map(c, c->dense_vmap, c->Vc, (unsigned long long)cfg->head_dim, (unsigned long long)c->lanes_total * cap, 64u);
   if (rc == WKV_OK) rc = run_reset(c);
   if (rc != WKV_OK) {
     wkv_destroy(c);
@@ -1010,13 +1010,22 @@ int wkv_prefill(wkv_ctx* c, int32_t layer, const void* Q, const void* K, const v
 
 // The dense kernel over `lanes` consecutive lanes starting at lane0 (one layer, or all layers at once: to the kernel the
 // lanes of several layers are just more sequences).  Takes the scratch on first use / when more lanes are needed.
+// Which geometry the dense prompt kernel runs with for a launch of `lanes` lanes: blocks of 32 query rows (256 threads,
+// two CTAs per SM) while two CTAs per SM hold every lane, else blocks of 16 rows (128 threads, four CTAs per SM).
+static bool dense_rows_wide(const wkv_ctx* c, long long lanes) {
+  return c->cfg.dtype == WKV_BF16 && lanes <= 2LL * c->sm_count;
+}
 static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void* Q, const void* K, const void* V,
                         const int32_t* seq_lens, int32_t T_max, int32_t n0, void* out, int32_t* evicted_pos) {
-  if (c->bulk_S == nullptr || c->bulk_lanes < lanes) {
+  // few lanes (at most two per SM): blocks of 32 query rows on 256 threads; else 16 rows on 128 threads, four CTAs per SM
+  const bool wide = dense_rows_wide(c, lanes);
+  const int rows = wide ? wkv::kBulkRowsWide : wkv::kBulkRows;
+  if (c->bulk_S == nullptr || c->bulk_lanes * c->bulk_rows < lanes * rows) {
     c->bulk_stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
-    int rc = take(c, &c->bulk_S, (size_t)lanes * wkv::kBulkRows * c->bulk_stride * 4);
+    int rc = take(c, &c->bulk_S, (size_t)lanes * rows * c->bulk_stride * 4);
     if (rc != WKV_OK) return rc;
     c->bulk_lanes = lanes;
+    c->bulk_rows = rows;
   }
   wkv::PrefillParams P;
   std::memset(&P, 0, sizeof(P));
@@ -1036,14 +1045,12 @@ static int launch_dense(wkv_ctx* c, long long lane0, long long lanes, const void
   cudaError_t e;
   const int n = (int)lanes;
   if (c->cfg.dtype == WKV_BF16) {
-    // 128-key tiles (two CTAs per SM) unless there are more lanes than that keeps busy
-    const bool wide = n <= 2 * c->sm_count;
-    // the kernel takes its tiles through the tensor maps over the caches (boxes of one tile of keys)
-    std::memcpy(P.kmap, c->dense_kmap[wide ? 1 : 0], sizeof(P.kmap));
-    std::memcpy(P.vmap, c->dense_vmap[wide ? 1 : 0], sizeof(P.vmap));
+    // the kernel takes its tiles through the tensor maps over the caches (boxes of one tile of 64 keys)
+    std::memcpy(P.kmap, c->dense_kmap, sizeof(P.kmap));
+    std::memcpy(P.vmap, c->dense_vmap, sizeof(P.vmap));
     if (wide)
-      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 128>(c->group, P, n, c->stream)
-                                 : launch_bulk<__nv_bfloat16, 64, 128>(c->group, P, n, c->stream);
+      e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64, wkv::kBulkRowsWide>(c->group, P, n, c->stream)
+                                 : launch_bulk<__nv_bfloat16, 64, 64, wkv::kBulkRowsWide>(c->group, P, n, c->stream);
     else
       e = c->cfg.head_dim == 128 ? launch_bulk<__nv_bfloat16, 128, 64>(c->group, P, n, c->stream)
                                  : launch_bulk<__nv_bfloat16, 64, 64>(c->group, P, n, c->stream);
@@ -1108,7 +1115,7 @@ int wkv_prefill_bulk_layers(wkv_ctx* c, const void* Q, const void* K, const void
   if (room > 0 && T_max > 0) {
     n0 = (int32_t)std::min<long long>(T_max, room);        // uncompressed in every lane of every layer (see wkv_prefill_bulk)
     const int stride = (c->cfg.budget + wkv::kBulkKeys - 1) / wkv::kBulkKeys * wkv::kBulkKeys;
-    const size_t need_all = (size_t)c->lanes_total * wkv::kBulkRows * stride * 4;
+    const size_t need_all = (size_t)c->lanes_total * (dense_rows_wide(c, c->lanes_total) ? wkv::kBulkRowsWide : wkv::kBulkRows) * stride * 4;
     if (need_all <= ((size_t)256 << 20)) {
       // every lane of every layer in one launch
       rc = launch_dense(c, 0, c->lanes_total, Q, K, V, seq_lens, T_max, n0, out, evicted_pos);

@@ -25,10 +25,14 @@
 
 namespace wkv {
 
-constexpr int kBulkRows = 16;        // query rows per block: 16 / G tokens x G heads
+constexpr int kBulkRows = 16;        // query rows per block: 16 / G tokens x G heads (kBulkRowsWide: 32, for layers of few lanes)
+constexpr int kBulkRowsWide = 32;
 constexpr int kBulkKeys = 128;       // granularity of the scratch rows (a multiple of every tile size)
-constexpr int kBulkThreads = 128;    // 4 warps; warp w owns query rows 4w .. 4w+3
-constexpr int kBulkPadP = 20;        // floats per key in the probability tile (16 rows + padding)
+// A CTA has 8 threads per query row of its block: warp w owns query rows 4w .. 4w+3.  A layer with at most two lanes per
+// SM runs blocks of 32 rows on 256 threads: twice the warps per SM for the same registers per thread, and every key
+// and value tile is fetched half as often.
+__host__ __device__ constexpr int bulk_threads(int rows) { return 8 * rows; }
+__host__ __device__ constexpr int bulk_pad_p(int rows) { return rows + 4; }   // floats per key in the probability tile (the rows + padding)
 
 struct PrefillParams {
   void* Kc;
@@ -67,13 +71,13 @@ struct PrefillParams {
 // the arithmetic.  Both layouts are free of bank conflicts for the two access patterns (a thread per key in the logits,
 // transposed fragment loads in P.V).  The tiles are read from the CACHE, where the kernel has put this call's rows
 // first (token i in slot i), so earlier chunks of a prompt and this one come through the same map.
-template <typename T, int D, int KT>
+template <typename T, int D, int KT, int ROWS = kBulkRows>
 constexpr int bulk_smem_bytes() {
   constexpr bool kTma = sizeof(T) == 2;
-  return kBulkRows * D * 4                                   // query rows, fp32
+  return ROWS * D * 4                                        // query rows, fp32
          + 2 * KT * (D * (int)sizeof(T) + (kTma ? 0 : 16))   // two tile stages, storage type, padded rows (or swizzled)
-         + KT * kBulkPadP * 4                                // probabilities of a tile, fp32
-         + (sizeof(T) == 2 ? 2 * kBulkRows * (KT + 8) * 2 : 0)   // bf16 hi and lo parts of the probabilities
+         + KT * bulk_pad_p(ROWS) * 4                         // probabilities of a tile, fp32
+         + (sizeof(T) == 2 ? 2 * ROWS * (KT + 8) * 2 : 0)    // bf16 hi and lo parts of the probabilities
          + 64;                                               // mbarriers
 }
 
@@ -97,13 +101,13 @@ __device__ __forceinline__ void store_row_part(__nv_bfloat16* p, const float (&x
 // a_i <- a_i + mean over the group's heads of P[t, g, i], one token after the other (the order Algorithm 1 adds them
 // in).  Thread tid < KT owns key k0 + tid of the tile; Pt is [key][row] with row = token_in_block * G + head; a_prev is
 // the key's score before this block (0 if the key's own token is in the block: it starts from [a, 0]).
-template <int G, int KT>
+template <int G, int KT, int ROWS>
 __device__ __forceinline__ void fold_columns(const float* Pt, float* a_l, float a_prev, int k0, int t0, int nk, int n) {
-  constexpr int BQ = kBulkRows / G;
+  constexpr int BQ = ROWS / G;
   const int key = k0 + (int)threadIdx.x;
   if ((int)threadIdx.x >= KT || key >= nk) return;
   float a_i = a_prev;
-  const float* pr = Pt + threadIdx.x * kBulkPadP;
+  const float* pr = Pt + threadIdx.x * bulk_pad_p(ROWS);
 #pragma unroll
   for (int tok = 0; tok < BQ; ++tok) {
     float pbar = pr[tok * G];
@@ -129,9 +133,13 @@ __device__ __forceinline__ uint32_t swz_off(int key, int elem) {
   return (uint32_t)((chunk >> 3) * (KT * 128) + key * 128 + ((((chunk & 7) ^ (key & 7)) << 4) | ((elem & 7) << 1)));
 }
 
-template <typename T, int D, int G, int KT>
-__global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_kernel(const __grid_constant__ PrefillParams P) {
+template <typename T, int D, int G, int KT, int ROWS = kBulkRows>
+__global__ void __launch_bounds__(bulk_threads(ROWS), ROWS == 32 ? 2 : (KT == 64 ? 4 : 2))
+prefill_bulk_kernel(const __grid_constant__ PrefillParams P) {
   constexpr bool kTma = sizeof(T) == 2;          // tiles through the caches' tensor maps
+  constexpr int kBulkRows = ROWS;                // (shadows the namespace constants: this instantiation's geometry)
+  constexpr int kBulkThreads = bulk_threads(ROWS);
+  constexpr int kBulkPadP = bulk_pad_p(ROWS);
   constexpr int BQ = kBulkRows / G;              // tokens per row block
   constexpr int CH = D / 16;                     // channels per partial sum of the reproducible dot
   constexpr int CP = CH / 2;                     // ... as (even, odd) pairs
@@ -144,10 +152,10 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
   constexpr int QV = ROWB / 128;                 // 16-byte pieces of the query block per thread
   static_assert(kBulkRows % G == 0 && kBulkThreads == 8 * kBulkRows && KT <= kBulkThreads && kBulkKeys % KT == 0, "thread maps");
   extern __shared__ __align__(1024) unsigned char bulk_smem[];           // (swizzled tiles start on 1024-byte boundaries)
-  float* Qs = reinterpret_cast<float*>(bulk_smem);                       // [16][D] fp32
+  float* Qs = reinterpret_cast<float*>(bulk_smem);                       // [rows][D] fp32
   T* stage0 = reinterpret_cast<T*>(Qs + kBulkRows * D);                  // 2 x [KT][RS]
   float* Pt = reinterpret_cast<float*>(stage0 + 2 * KT * RS);            // [KT][20]: probabilities, [key][row]
-  __nv_bfloat16* Ph = reinterpret_cast<__nv_bfloat16*>(Pt + KT * kBulkPadP);   // [16][KT + 8] (bf16 storage only)
+  __nv_bfloat16* Ph = reinterpret_cast<__nv_bfloat16*>(Pt + KT * kBulkPadP);   // [rows][KT + 8] (bf16 storage only)
   __nv_bfloat16* Pl = Ph + kBulkRows * PS;
   uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(Pt + KT * kBulkPadP) +
                                                (kTensorPV ? 2 * kBulkRows * PS * 2 : 0));
@@ -439,17 +447,19 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         }
       }
       __syncthreads();                                   // the probability tiles (and the zeroed rows)
-      fold_columns<G, KT>(Pt, a_l, a_prev, k0, t0, nk, n);
+      fold_columns<G, KT, ROWS>(Pt, a_l, a_prev, k0, t0, nk, n);
       if constexpr (kTensorPV) {
         // O += P . V on the tensor cores (the outputs are not part of the reproducible chain).  Warp w takes all 16
         // rows and channels [w*D/4, (w+1)*D/4).  Fragment addresses: A (P, row-major [row][key]): thread i -> row
         // (i%8) + 8*((i/8)&1), key 8*(i/16); B (V, [key][channel], read transposed): thread i -> key (i%8) +
         // 8*((i/8)&1), channel 8*(i/16).
+        // (blocks of 32 rows: warps 4 .. 7 do the same for rows 16 .. 31)
         const int ksteps = (min(KT, nk - k0) + 15) / 16;
+        const int wq = w & 3, wr = (w >> 2) * 16;        // the warp's channel quarter and first row
         const int frow = (ln & 7) + ((ln >> 3) & 1) * 8, fcol = (ln >> 4) * 8;
-        const uint32_t a_off = (uint32_t)((frow * PS + fcol) * 2);
+        const uint32_t a_off = (uint32_t)(((wr + frow) * PS + fcol) * 2);
         const uint32_t ph_base = smem_u32(Ph) + a_off, pl_base = smem_u32(Pl) + a_off;
-        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((frow * RS + w * (D / 4) + fcol) * 2);   // (padded rows)
+        const uint32_t v_base = smem_u32(Vt) + (uint32_t)((frow * RS + wq * (D / 4) + fcol) * 2);   // (padded rows)
         for (int ks = 0; ks < ksteps; ++ks) {
           uint32_t ah[4], al[4];
           asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -459,7 +469,7 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
 #pragma unroll
           for (int np = 0; np < NTW / 2; ++np) {
             uint32_t bf[4];
-            const uint32_t v_addr = kTma ? smem_u32(Vt) + swz_off<KT>(ks * 16 + frow, w * (D / 4) + fcol + np * 16)
+            const uint32_t v_addr = kTma ? smem_u32(Vt) + swz_off<KT>(ks * 16 + frow, wq * (D / 4) + fcol + np * 16)
                                          : v_base + (uint32_t)(ks * 16 * RS * 2 + np * 32);
             asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
                          : "=r"(bf[0]), "=r"(bf[1]), "=r"(bf[2]), "=r"(bf[3])
@@ -516,10 +526,10 @@ __global__ void __launch_bounds__(kBulkThreads, KT == 64 ? 4 : 2) prefill_bulk_k
         // accumulator fragment: rows ln/4 and ln/4 + 8, channels (ln%4)*2, +1 of each n-tile
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const int rho = (ln >> 2) + 8 * h;
+          const int rho = (w >> 2) * 16 + (ln >> 2) + 8 * h;
           const int t = t0 + rho / G, g = rho % G;
           if (t >= n) continue;
-          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + (t - n_old)) * Hq + (long long)hk * G + g) * D + w * (D / 4) + (ln & 3) * 2;
+          T* dst = reinterpret_cast<T*>(P.out) + (((long long)b * P.T_max + (t - n_old)) * Hq + (long long)hk * G + g) * D + (w & 3) * (D / 4) + (ln & 3) * 2;
 #pragma unroll
           for (int nt = 0; nt < NTW; ++nt) {
             const float x[2] = {cacc[nt][2 * h], cacc[nt][2 * h + 1]};
