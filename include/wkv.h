@@ -185,7 +185,8 @@ int wkv_prefill(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const
  * score fold, pick, merge) then runs on them token after token exactly as when streaming, and one sweep over the value
  * rows gives all outputs; elsewhere they are streamed as in wkv_prefill.  So a prompt may come in one call or in chunks.  K, positions, accumulated scores and removed positions are bit-identical to
  * wkv_prefill's; outputs and merged values agree within rounding.
- * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider, the first
+ * The first call takes 64 * lanes_per_layer * round_up(budget, 128) bytes of scratch from the memory provider (twice that for
+ * bf16 layers of at most two lanes per SM, which run blocks of 32 query rows), the first
  * blocked tail about 64 * lanes_per_layer * (budget + 1) bytes more (if the provider refuses those, the tail is streamed);
  * both are kept until wkv_destroy.  Q, K, V, out must be 16-byte aligned (WKV_ERR_INVALID otherwise).  Asynchronous. */
 int wkv_prefill_bulk(wkv_ctx* ctx, int32_t layer, const void* Q, const void* K, const void* V, const int32_t* seq_lens,
